@@ -1,0 +1,317 @@
+// GaussWS sampling oracle: a plain, slow, single-threaded CPU statement of the
+// weight-sampling pass of Gaussian weight sampling (Eq. 3 forward, Eq. 4
+// backward, Section 3.4 noise law of Eq. 9 / Eq. 10, packed format of
+// Section 3.4's last paragraph).
+//
+// THIS FILE IS TEST INFRASTRUCTURE.  It exists to be checked by eye against
+// the paper and to check the CUDA library.  It shares no code with the CUDA
+// path, nothing in the product imports it, and it is never tuned for speed.
+// Only the test suite, the smoke check and the CPU-baseline leg of the
+// benchmark may call it.
+//
+// Build: g++ -std=c++17 -O2 -ffp-contract=off -fno-fast-math -shared -fPIC
+// (no FMA contraction, so every float operation below rounds exactly once).
+//
+// Conventions (the paper leaves them open; both sides implement this list):
+//   * A tensor is row-major [rows, cols] BF16 with `ld` elements between rows.
+//   * A group is group_rows x group_cols elements (group_cols == 0: the whole
+//     row).  Groups are numbered row-major over the ceil(rows/group_rows) x
+//     ceil(cols/group_cols) grid, the shape the paper gives b_t below Eq. 3.
+//   * PRNG: Philox4x32 with 10 rounds (the paper names Philox in Section 3.4).
+//     Element (i, j) has the logical index e = elem_offset + i*cols + j.  The
+//     Philox counter is (lo32(e>>3), hi32(e>>3), lo32(step), hi32(step)), the
+//     key is (lo32(seed), hi32(seed)).  One call serves 8 consecutive
+//     elements; element e uses the 16-bit field number (e & 7) of the 128
+//     output bits, fields counted from the least significant bits of word 0.
+//   * Noise decode (Eq. 9 / Eq. 10), field bits x0 (LSB) .. x15:
+//       m2 = x0 & x1 & ... & x7 & (x8 | x9)          Pr = 2^-8 * 3/4
+//       m1 = (x10 | x11) & (x12 | x13) & x14         Pr = (3/4)^2 * 1/2
+//       |R| = 2 if m2, else 1 if m1, else 0;  R = -|R| if x15 else +|R|.
+//   * scale s_g = fl32(absmax_g * 2^(1 - b_g)); 2^(1-b) is computed in
+//     double and rounded to float (exact for integer b).
+//   * sample: y = fl32(float(w) + float(R) * s_g)  (the product is exact),
+//     w_hat = BF16 round-to-nearest-even of y.  R == 0 adds +0.0f.
+//   * backward: grad_w = upstream gradient unchanged; grad_b_g =
+//     float(-ln 2 * s_g * sum_g(float(g) * R)), the sum taken in double in
+//     row-major order inside the group.
+//
+// Pins (tests/test_oracle_*.py): Philox known-answer vectors; exhaustive
+// decode counts against Eq. 10; closed-form moments; KS / chi-square over
+// 10^7 draws; hand-computed add-then-cast cases; library BF16 casts;
+// finite-difference gradients; the Lemma 1 and Proposition 2 invariants.
+// The only thing left unpinned is which of the equally valid bit assignments
+// the authors' own kernels used; their stream cannot be reproduced.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+namespace {
+
+// ---- BF16 <-> FP32 by bit manipulation ------------------------------------
+
+float bf16_to_f32(uint16_t h) {
+  uint32_t u = static_cast<uint32_t>(h) << 16;
+  float f;
+  std::memcpy(&f, &u, sizeof f);
+  return f;
+}
+
+// IEEE round-to-nearest, ties-to-even, onto the upper 16 bits of a float.
+uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, sizeof u);
+  const uint32_t exponent = (u >> 23) & 0xFFu;
+  const uint32_t fraction = u & 0x007FFFFFu;
+  if (exponent == 0xFFu && fraction != 0) {
+    // NaN: keep it a NaN after truncation.
+    return static_cast<uint16_t>((u >> 16) | 0x0040u);
+  }
+  uint32_t kept = u >> 16;            // sign, exponent, 7 fraction bits
+  const uint32_t dropped = u & 0xFFFFu;  // the 16 bits that are cut off
+  const uint32_t half = 0x8000u;
+  if (dropped > half) {
+    kept += 1;                        // above the midpoint: round away
+  } else if (dropped == half) {
+    if (kept & 1u) kept += 1;         // exactly the midpoint: to even
+  }
+  // A carry out of the fraction moves into the exponent, which is the right
+  // result (next binade, or infinity at the top).
+  return static_cast<uint16_t>(kept);
+}
+
+// ---- Philox4x32-10 ----------------------------------------------------------
+
+constexpr uint32_t PHILOX_M0 = 0xD2511F53u;
+constexpr uint32_t PHILOX_M1 = 0xCD9E8D57u;
+constexpr uint32_t PHILOX_W0 = 0x9E3779B9u;
+constexpr uint32_t PHILOX_W1 = 0xBB67AE85u;
+
+void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    const uint64_t p0 = static_cast<uint64_t>(PHILOX_M0) * c0;
+    const uint64_t p1 = static_cast<uint64_t>(PHILOX_M1) * c2;
+    const uint32_t hi0 = static_cast<uint32_t>(p0 >> 32), lo0 = static_cast<uint32_t>(p0);
+    const uint32_t hi1 = static_cast<uint32_t>(p1 >> 32), lo1 = static_cast<uint32_t>(p1);
+    const uint32_t n0 = hi1 ^ c1 ^ k0;
+    const uint32_t n1 = lo1;
+    const uint32_t n2 = hi0 ^ c3 ^ k1;
+    const uint32_t n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += PHILOX_W0;
+    k1 += PHILOX_W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// The four output words for the 8-element vector number `vec`.
+void philox_for_vector(uint64_t seed, uint64_t step, uint64_t vec, uint32_t out[4]) {
+  const uint32_t ctr[4] = {static_cast<uint32_t>(vec), static_cast<uint32_t>(vec >> 32),
+                           static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32)};
+  const uint32_t key[2] = {static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32)};
+  philox4x32_10(ctr, key, out);
+}
+
+// ---- noise decode (Eq. 9 / Eq. 10) -----------------------------------------
+
+int decode_field(uint32_t field) {
+  int x[16];
+  for (int k = 0; k < 16; ++k) x[k] = static_cast<int>((field >> k) & 1u);
+  int low_byte_all_ones = 1;
+  for (int k = 0; k < 8; ++k) low_byte_all_ones &= x[k];
+  const int m2 = low_byte_all_ones & (x[8] | x[9]);
+  const int m1 = (x[10] | x[11]) & (x[12] | x[13]) & x[14];
+  const int magnitude = m2 ? 2 : (m1 ? 1 : 0);
+  return x[15] ? -magnitude : magnitude;
+}
+
+// Noise of the element with logical index e.
+int noise_of_element(uint64_t seed, uint64_t step, uint64_t e) {
+  uint32_t o[4];
+  philox_for_vector(seed, step, e >> 3, o);
+  const unsigned t = static_cast<unsigned>(e & 7u);
+  const uint32_t field = (o[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu;
+  return decode_field(field);
+}
+
+// ---- group geometry ----------------------------------------------------------
+
+struct Geometry {
+  int64_t rows, cols, ld, group_rows, group_cols, groups_per_row_band, n_groups;
+};
+
+Geometry make_geometry(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols) {
+  Geometry g;
+  g.rows = rows;
+  g.cols = cols;
+  g.ld = ld;
+  g.group_rows = group_rows;
+  g.group_cols = (group_cols == 0) ? cols : group_cols;
+  g.groups_per_row_band = (cols + g.group_cols - 1) / g.group_cols;
+  g.n_groups = ((rows + group_rows - 1) / group_rows) * g.groups_per_row_band;
+  return g;
+}
+
+int64_t group_of(const Geometry& g, int64_t i, int64_t j) {
+  return (i / g.group_rows) * g.groups_per_row_band + (j / g.group_cols);
+}
+
+float scale_of(float absmax, float bits) {
+  const float pow2 = static_cast<float>(std::exp2(1.0 - static_cast<double>(bits)));
+  return absmax * pow2;
+}
+
+}  // namespace
+
+extern "C" {
+
+float gwso_bf16_to_f32(uint16_t h) { return bf16_to_f32(h); }
+uint16_t gwso_f32_to_bf16_rne(float f) { return f32_to_bf16_rne(f); }
+
+void gwso_philox4x32_10(const uint32_t* ctr4, const uint32_t* key2, uint32_t* out4) {
+  philox4x32_10(ctr4, key2, out4);
+}
+
+// out4 receives 4 words for each of the n_vec vectors first_vec, first_vec+1, ...
+void gwso_philox_words(uint64_t seed, uint64_t step, uint64_t first_vec, int64_t n_vec, uint32_t* out4) {
+  for (int64_t k = 0; k < n_vec; ++k) philox_for_vector(seed, step, first_vec + static_cast<uint64_t>(k), out4 + 4 * k);
+}
+
+int gwso_decode_field(uint32_t field16) { return decode_field(field16 & 0xFFFFu); }
+
+int64_t gwso_n_groups(int64_t rows, int64_t cols, int64_t group_rows, int64_t group_cols) {
+  return make_geometry(rows, cols, cols, group_rows, group_cols).n_groups;
+}
+
+// R for the n elements with logical indices first_elem, first_elem+1, ...
+void gwso_noise_r(uint64_t seed, uint64_t step, uint64_t first_elem, int64_t n, int8_t* r) {
+  for (int64_t k = 0; k < n; ++k)
+    r[k] = static_cast<int8_t>(noise_of_element(seed, step, first_elem + static_cast<uint64_t>(k)));
+}
+
+// Packed sign-magnitude nibbles, 8 elements per 32-bit word: element k of the
+// run sits in word k>>3 at bits [4*(k&7), 4*(k&7)+3]; nibble = sign<<3 | |R|,
+// and R == 0 is always stored as 0 (no negative zero).  first_elem must be a
+// multiple of 8; a final partial word has its unused nibbles zero.
+void gwso_noise_packed(uint64_t seed, uint64_t step, uint64_t first_elem, int64_t n, uint32_t* packed) {
+  const int64_t n_words = (n + 7) / 8;
+  for (int64_t v = 0; v < n_words; ++v) packed[v] = 0;
+  for (int64_t k = 0; k < n; ++k) {
+    const int r = noise_of_element(seed, step, first_elem + static_cast<uint64_t>(k));
+    const uint32_t magnitude = static_cast<uint32_t>(r < 0 ? -r : r);
+    const uint32_t nibble = (r < 0 ? 8u : 0u) | magnitude;
+    packed[k >> 3] |= nibble << (4 * (k & 7));
+  }
+}
+
+// absmax[g] = max over group g of |w| (exact: BF16 magnitudes widen to FP32 exactly).
+void gwso_group_absmax(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols,
+                       const uint16_t* w, float* absmax) {
+  const Geometry geo = make_geometry(rows, cols, ld, group_rows, group_cols);
+  for (int64_t g = 0; g < geo.n_groups; ++g) absmax[g] = 0.0f;
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const float a = std::fabs(bf16_to_f32(w[i * ld + j]));
+      const int64_t g = group_of(geo, i, j);
+      if (a > absmax[g]) absmax[g] = a;
+    }
+}
+
+void gwso_scale(int64_t n_groups, const float* absmax, const float* bt, float* scale) {
+  for (int64_t g = 0; g < n_groups; ++g) scale[g] = scale_of(absmax[g], bt[g]);
+}
+
+// Eq. 3 followed by the BF16 cast, with R supplied by the caller
+// (r[i*cols + j], values in -2..2).  scale_out may be null.
+void gwso_sample_fwd_injected(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols,
+                              const uint16_t* w, const float* bt, const int8_t* r, uint16_t* w_hat,
+                              float* scale_out, float* absmax_scratch) {
+  const Geometry geo = make_geometry(rows, cols, ld, group_rows, group_cols);
+  gwso_group_absmax(rows, cols, ld, group_rows, group_cols, w, absmax_scratch);
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const int64_t g = group_of(geo, i, j);
+      const float s = scale_of(absmax_scratch[g], bt[g]);
+      const float pqn = static_cast<float>(r[i * cols + j]) * s;
+      const float y = bf16_to_f32(w[i * ld + j]) + pqn;
+      w_hat[i * ld + j] = f32_to_bf16_rne(y);
+    }
+  if (scale_out)
+    for (int64_t g = 0; g < geo.n_groups; ++g) scale_out[g] = scale_of(absmax_scratch[g], bt[g]);
+}
+
+// Eq. 3 + cast with R drawn from the counter-based generator.
+void gwso_sample_fwd(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols,
+                     uint64_t seed, uint64_t step, uint64_t elem_offset, const uint16_t* w, const float* bt,
+                     uint16_t* w_hat, float* scale_out, float* absmax_scratch) {
+  const Geometry geo = make_geometry(rows, cols, ld, group_rows, group_cols);
+  gwso_group_absmax(rows, cols, ld, group_rows, group_cols, w, absmax_scratch);
+  uint64_t cached_vec = ~static_cast<uint64_t>(0);
+  uint32_t o[4] = {0, 0, 0, 0};
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const uint64_t e = elem_offset + static_cast<uint64_t>(i * cols + j);
+      if ((e >> 3) != cached_vec) {  // same call as noise_of_element, made once per vector
+        cached_vec = e >> 3;
+        philox_for_vector(seed, step, cached_vec, o);
+      }
+      const unsigned t = static_cast<unsigned>(e & 7u);
+      const int r = decode_field((o[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu);
+      const int64_t g = group_of(geo, i, j);
+      const float s = scale_of(absmax_scratch[g], bt[g]);
+      const float pqn = static_cast<float>(r) * s;
+      const float y = bf16_to_f32(w[i * ld + j]) + pqn;
+      w_hat[i * ld + j] = f32_to_bf16_rne(y);
+    }
+  if (scale_out)
+    for (int64_t g = 0; g < geo.n_groups; ++g) scale_out[g] = scale_of(absmax_scratch[g], bt[g]);
+}
+
+// Eq. 4 with R supplied.  grad_w (may be null) receives the upstream gradient
+// unchanged; grad_bt[g] = -ln2 * scale[g] * sum_g(grad * R).
+void gwso_sample_bwd_injected(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols,
+                              const uint16_t* grad_w_hat, const float* scale, const int8_t* r,
+                              uint16_t* grad_w, float* grad_bt, double* acc_scratch) {
+  const Geometry geo = make_geometry(rows, cols, ld, group_rows, group_cols);
+  for (int64_t g = 0; g < geo.n_groups; ++g) acc_scratch[g] = 0.0;
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const uint16_t gbits = grad_w_hat[i * ld + j];
+      if (grad_w) grad_w[i * ld + j] = gbits;
+      acc_scratch[group_of(geo, i, j)] +=
+          static_cast<double>(bf16_to_f32(gbits)) * static_cast<double>(r[i * cols + j]);
+    }
+  const double ln2 = 0.6931471805599453;
+  for (int64_t g = 0; g < geo.n_groups; ++g)
+    grad_bt[g] = static_cast<float>(-ln2 * static_cast<double>(scale[g]) * acc_scratch[g]);
+}
+
+// Eq. 4 with R regenerated from (seed, step, element index).
+void gwso_sample_bwd(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols,
+                     uint64_t seed, uint64_t step, uint64_t elem_offset, const uint16_t* grad_w_hat,
+                     const float* scale, uint16_t* grad_w, float* grad_bt, double* acc_scratch) {
+  const Geometry geo = make_geometry(rows, cols, ld, group_rows, group_cols);
+  for (int64_t g = 0; g < geo.n_groups; ++g) acc_scratch[g] = 0.0;
+  uint64_t cached_vec = ~static_cast<uint64_t>(0);
+  uint32_t o[4] = {0, 0, 0, 0};
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const uint64_t e = elem_offset + static_cast<uint64_t>(i * cols + j);
+      if ((e >> 3) != cached_vec) {
+        cached_vec = e >> 3;
+        philox_for_vector(seed, step, cached_vec, o);
+      }
+      const unsigned t = static_cast<unsigned>(e & 7u);
+      const int r = decode_field((o[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu);
+      const uint16_t gbits = grad_w_hat[i * ld + j];
+      if (grad_w) grad_w[i * ld + j] = gbits;
+      acc_scratch[group_of(geo, i, j)] += static_cast<double>(bf16_to_f32(gbits)) * static_cast<double>(r);
+    }
+  const double ln2 = 0.6931471805599453;
+  for (int64_t g = 0; g < geo.n_groups; ++g)
+    grad_bt[g] = static_cast<float>(-ln2 * static_cast<double>(scale[g]) * acc_scratch[g]);
+}
+
+}  // extern "C"

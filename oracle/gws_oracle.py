@@ -1,0 +1,204 @@
+"""ctypes front end of the GaussWS CPU oracle (``gws_oracle.cpp``).
+
+TEST INFRASTRUCTURE ONLY: the oracle is the slow, single-threaded statement of
+Eq. 3 / Eq. 4 / Eq. 10 that the CUDA library is checked against.  The product
+package never imports this module; only the tests, the smoke check and the
+CPU-baseline leg of the benchmark do.
+
+All arrays are numpy.  BF16 tensors travel as ``uint16`` bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from ctypes import POINTER, c_double, c_float, c_int, c_int8, c_int64, c_uint16, c_uint32, c_uint64
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gws_oracle.cpp")
+_LIB = os.path.join(_HERE, "libgws_oracle.so")
+
+CXXFLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ if the shared object is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.run(["g++", *CXXFLAGS, "-o", tmp, _SRC], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        u16p, u32p, f32p, i8p, f64p = (POINTER(c_uint16), POINTER(c_uint32), POINTER(c_float), POINTER(c_int8),
+                                       POINTER(c_double))
+        L.gwso_bf16_to_f32.argtypes = [c_uint16]
+        L.gwso_bf16_to_f32.restype = c_float
+        L.gwso_f32_to_bf16_rne.argtypes = [c_float]
+        L.gwso_f32_to_bf16_rne.restype = c_uint16
+        L.gwso_philox4x32_10.argtypes = [u32p, u32p, u32p]
+        L.gwso_philox4x32_10.restype = None
+        L.gwso_philox_words.argtypes = [c_uint64, c_uint64, c_uint64, c_int64, u32p]
+        L.gwso_philox_words.restype = None
+        L.gwso_decode_field.argtypes = [c_uint32]
+        L.gwso_decode_field.restype = c_int
+        L.gwso_n_groups.argtypes = [c_int64] * 4
+        L.gwso_n_groups.restype = c_int64
+        L.gwso_noise_r.argtypes = [c_uint64, c_uint64, c_uint64, c_int64, i8p]
+        L.gwso_noise_r.restype = None
+        L.gwso_noise_packed.argtypes = [c_uint64, c_uint64, c_uint64, c_int64, u32p]
+        L.gwso_noise_packed.restype = None
+        L.gwso_group_absmax.argtypes = [c_int64] * 5 + [u16p, f32p]
+        L.gwso_group_absmax.restype = None
+        L.gwso_scale.argtypes = [c_int64, f32p, f32p, f32p]
+        L.gwso_scale.restype = None
+        L.gwso_sample_fwd_injected.argtypes = [c_int64] * 5 + [u16p, f32p, i8p, u16p, f32p, f32p]
+        L.gwso_sample_fwd_injected.restype = None
+        L.gwso_sample_fwd.argtypes = [c_int64] * 5 + [c_uint64] * 3 + [u16p, f32p, u16p, f32p, f32p]
+        L.gwso_sample_fwd.restype = None
+        L.gwso_sample_bwd_injected.argtypes = [c_int64] * 5 + [u16p, f32p, i8p, u16p, f32p, f64p]
+        L.gwso_sample_bwd_injected.restype = None
+        L.gwso_sample_bwd.argtypes = [c_int64] * 5 + [c_uint64] * 3 + [u16p, f32p, u16p, f32p, f64p]
+        L.gwso_sample_bwd.restype = None
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray, ctype):
+    return a.ctypes.data_as(POINTER(ctype))
+
+
+def _c(a, dtype) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+# ---- scalar helpers -------------------------------------------------------------
+
+def bf16_to_f32(bits: int) -> float:
+    return float(lib().gwso_bf16_to_f32(int(bits) & 0xFFFF))
+
+
+def f32_to_bf16_rne(x: float) -> int:
+    return int(lib().gwso_f32_to_bf16_rne(c_float(x)))
+
+
+def f32_array_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Elementwise oracle cast of a float32 array to BF16 bit patterns."""
+    x = _c(x, np.float32).ravel()
+    out = np.empty(x.shape, np.uint16)
+    f = lib().gwso_f32_to_bf16_rne
+    for k in range(x.size):
+        out[k] = f(c_float(float(x[k])))
+    return out
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    c, k, o = _c(ctr, np.uint32), _c(key, np.uint32), np.empty(4, np.uint32)
+    assert c.size == 4 and k.size == 2
+    lib().gwso_philox4x32_10(_p(c, c_uint32), _p(k, c_uint32), _p(o, c_uint32))
+    return o
+
+
+def philox_words(seed: int, step: int, first_vec: int, n_vec: int) -> np.ndarray:
+    out = np.empty((n_vec, 4), np.uint32)
+    lib().gwso_philox_words(seed, step, first_vec, n_vec, _p(out, c_uint32))
+    return out
+
+
+def decode_field(field16: int) -> int:
+    return int(lib().gwso_decode_field(field16))
+
+
+def n_groups(rows: int, cols: int, group_rows: int, group_cols: int) -> int:
+    return int(lib().gwso_n_groups(rows, cols, group_rows, group_cols))
+
+
+# ---- array entry points -----------------------------------------------------------
+
+def noise_r(seed: int, step: int, first_elem: int, n: int) -> np.ndarray:
+    """R in {-2..2} (int8) for the logical element indices first_elem .. first_elem+n-1."""
+    r = np.empty(n, np.int8)
+    lib().gwso_noise_r(seed, step, first_elem, n, _p(r, c_int8))
+    return r
+
+
+def noise_packed(seed: int, step: int, first_elem: int, n: int) -> np.ndarray:
+    assert first_elem % 8 == 0
+    out = np.empty((n + 7) // 8, np.uint32)
+    lib().gwso_noise_packed(seed, step, first_elem, n, _p(out, c_uint32))
+    return out
+
+
+def _check_w(w: np.ndarray, rows: int, cols: int, ld: int) -> np.ndarray:
+    w = _c(w, np.uint16).ravel()
+    assert w.size >= (rows - 1) * ld + cols, "buffer smaller than (rows-1)*ld + cols"
+    return w
+
+
+def group_absmax(w, rows, cols, group_rows=1, group_cols=0, ld=None) -> np.ndarray:
+    ld = cols if ld is None else ld
+    w = _check_w(w, rows, cols, ld)
+    out = np.empty(n_groups(rows, cols, group_rows, group_cols), np.float32)
+    lib().gwso_group_absmax(rows, cols, ld, group_rows, group_cols, _p(w, c_uint16), _p(out, c_float))
+    return out
+
+
+def scale(absmax, bt) -> np.ndarray:
+    a, b = _c(absmax, np.float32), _c(bt, np.float32)
+    assert a.size == b.size
+    out = np.empty(a.size, np.float32)
+    lib().gwso_scale(a.size, _p(a, c_float), _p(b, c_float), _p(out, c_float))
+    return out
+
+
+def sample_fwd(w, bt, rows, cols, group_rows=1, group_cols=0, seed=0, step=0, elem_offset=0, ld=None, r=None):
+    """Returns (w_hat uint16 [same buffer shape as w], scale float32 [n_groups]).
+
+    With ``r`` (int8 [rows*cols], logical order) the noise is injected instead of generated."""
+    ld = cols if ld is None else ld
+    w = _check_w(w, rows, cols, ld)
+    ng = n_groups(rows, cols, group_rows, group_cols)
+    bt = _c(bt, np.float32)
+    assert bt.size == ng
+    w_hat = w.copy()  # padding (ld > cols) keeps the input bits
+    sc = np.empty(ng, np.float32)
+    scratch = np.empty(ng, np.float32)
+    if r is None:
+        lib().gwso_sample_fwd(rows, cols, ld, group_rows, group_cols, seed, step, elem_offset, _p(w, c_uint16),
+                              _p(bt, c_float), _p(w_hat, c_uint16), _p(sc, c_float), _p(scratch, c_float))
+    else:
+        r = _c(r, np.int8)
+        assert r.size == rows * cols
+        lib().gwso_sample_fwd_injected(rows, cols, ld, group_rows, group_cols, _p(w, c_uint16), _p(bt, c_float),
+                                       _p(r, c_int8), _p(w_hat, c_uint16), _p(sc, c_float), _p(scratch, c_float))
+    return w_hat, sc
+
+
+def sample_bwd(g, scale_, rows, cols, group_rows=1, group_cols=0, seed=0, step=0, elem_offset=0, ld=None, r=None):
+    """Returns (grad_w uint16, grad_bt float32 [n_groups])."""
+    ld = cols if ld is None else ld
+    g = _check_w(g, rows, cols, ld)
+    ng = n_groups(rows, cols, group_rows, group_cols)
+    sc = _c(scale_, np.float32)
+    assert sc.size == ng
+    gw = g.copy()
+    gbt = np.empty(ng, np.float32)
+    acc = np.empty(ng, np.float64)
+    if r is None:
+        lib().gwso_sample_bwd(rows, cols, ld, group_rows, group_cols, seed, step, elem_offset, _p(g, c_uint16),
+                              _p(sc, c_float), _p(gw, c_uint16), _p(gbt, c_float), _p(acc, c_double))
+    else:
+        r = _c(r, np.int8)
+        assert r.size == rows * cols
+        lib().gwso_sample_bwd_injected(rows, cols, ld, group_rows, group_cols, _p(g, c_uint16), _p(sc, c_float),
+                                       _p(r, c_int8), _p(gw, c_uint16), _p(gbt, c_float), _p(acc, c_double))
+    return gw, gbt
