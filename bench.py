@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the GaussWS weight-sampling pass on B200.
+
+One "step" = one forward pass (Eq. 3 + BF16 cast) plus one backward pass (Eq. 4, noise
+regenerated) over the whole Llama2-1B-shaped linear weight set (154 tensors, 1,130,364,928 BF16
+elements, groups of 128 along the input dimension, b_t uniform on {4..9}), each pass one launch.
+Inputs are synthetic (seeded N(0, 0.02^2) weights, N(0, 1e-4^2) upstream gradients) and resident
+in HBM when the timed region starts; every pass streams 2.26 GB per tensor set, far beyond L2.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sampling fwd+bwd GB/s and Gelem/s at 1 B200; fraction of HBM peak"
+WORKLOAD = "llama2_1b_linear_set_g128"
+FWD_BYTES_PER_ELEM = 2 + 2 + 8 / 128      # read w, write w_hat, read b_t + write scale per 128 elements
+BWD_BYTES_PER_ELEM = 2 + 8 / 128          # read dL/dw_hat, read scale + write dL/db_t per 128 elements
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def ncu_traffic():
+    """Per-launch DRAM bytes of the forward kernel from the committed ncu summary, if there is one."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f)
+    return {}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        rows = [s for (t, s) in self.samples if t0 - 0.05 <= t <= t1 + 0.15] or [s for (_, s) in self.samples]
+        mhz, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                mhz.append(float(f[0]))
+                mx = float(f[1])
+            except Exception:
+                continue
+            for name, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        mhz.sort()
+        return {"sm_mhz": mhz[len(mhz) // 2] if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(mhz)}
+
+
+def run_reference(args, rank: int, world: int):
+    """The CPU oracle, as it stands, on a bounded sample of the workload (rank 0 only)."""
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import gws_oracle as orc
+    from paper_2505_11170_b200 import synthetic as syn
+    specs = syn.llama2_1b()
+    sample = [0, 4]                       # l0.q (2048x2048) and l0.gate (5632x2048): 15.7 M elements
+    data = []
+    for i in sample:
+        s = specs[i]
+        as_bits = lambda t: t.view(torch.int16).numpy().view(np.uint16)
+        data.append((s, syn.layer_seed(0, i), as_bits(syn.weights(s, i)), syn.bitwidths(s, i).numpy(),
+                     as_bits(syn.upstream_grad(s, i))))
+    elems = sum(d[0].numel for d in data)
+
+    def step(k):
+        for s, seed, w, bt, g in data:
+            _, sc = orc.sample_fwd(w, bt, s.rows, s.cols, 1, s.group_cols, seed=seed, step=k)
+            orc.sample_bwd(g, sc, s.rows, s.cols, 1, s.group_cols, seed=seed, step=k)
+
+    for k in range(args.warmup):
+        step(k)
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        step(args.warmup + k)
+    dt = time.perf_counter() - t0
+    gbs = elems * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM) * args.steps / dt / 1e9
+    sample_text = "tensors l0.q and l0.gate of the 154 (15,728,640 of 1,130,364,928 elements) per step, fwd+bwd"
+    line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic (f64 gradient sum)", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample_text},
+            "gelem_per_s": elems * args.steps / dt / 1e9,
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample_text},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def cpu_baseline(specs):
+    """Oracle timed on the host cores: three Llama blocks, forward + backward, one thread."""
+    import numpy as np
+    from oracle import gws_oracle as orc
+    from paper_2505_11170_b200 import synthetic as syn
+    as_bits = lambda t: t.view(torch.int16).numpy().view(np.uint16)
+    idx = list(range(0, 14))             # blocks 0 and 1
+    elems, t = 0, 0.0
+    for i in idx:
+        s = specs[i]
+        w, bt, g = as_bits(syn.weights(s, i)), syn.bitwidths(s, i).numpy(), as_bits(syn.upstream_grad(s, i))
+        t0 = time.perf_counter()
+        _, sc = orc.sample_fwd(w, bt, s.rows, s.cols, 1, s.group_cols, seed=syn.layer_seed(0, i), step=0)
+        orc.sample_bwd(g, sc, s.rows, s.cols, 1, s.group_cols, seed=syn.layer_seed(0, i), step=0)
+        t += time.perf_counter() - t0
+        elems += s.numel
+    return {"value": elems * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM) / t / 1e9, "unit": "GB/s", "cores": 1,
+            "kind": "oracle", "gelem_per_s": elems / t / 1e9, "seconds": t, "host_cores": os.cpu_count(),
+            "sample": "blocks 0-1 of 22 (14 tensors, 102,760,448 elements), one forward + backward step"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--blocks", type=int, default=22, help="Llama blocks in the set (22 = the full workload)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import paper_2505_11170_b200 as gws
+    from paper_2505_11170_b200 import synthetic as syn
+    from paper_2505_11170_b200.binding import Desc
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the sampling pass has no CPU path")
+    gws.load_library()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # Every rank holds a full replica of the weight set (the pass has no exchange step): weak scaling.
+    specs = syn.llama2_1b(n_blocks=args.blocks)
+    n_elem = syn.total_elements(specs)
+    descs = [Desc.make(s.rows, s.cols, 1, s.group_cols, seed=syn.layer_seed(rank, i)) for i, s in enumerate(specs)]
+    W = [syn.weights(s, i, device=dev) for i, s in enumerate(specs)]
+    BT = [syn.bitwidths(s, i, device=dev) for i, s in enumerate(specs)]
+    G = [syn.upstream_grad(s, i, device=dev) for i, s in enumerate(specs)]
+    WH = [torch.empty_like(t) for t in W]
+    SC = [torch.empty(s.n_groups, device=dev) for s in specs]
+    GBT = [torch.empty(s.n_groups, device=dev) for s in specs]
+    plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=WH, scale=SC, grad_w_hat=G, grad_bt=GBT)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    step_no = 0
+    for _ in range(args.warmup):
+        plan.sample_fwd_multi(step_no)
+        plan.sample_bwd_multi(step_no)
+        step_no += 1
+    barrier()
+
+    # ---- device-resident timing: K steps, an event after every launch ----
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches0 = gws.launch_count()
+    barrier()
+    t_wall0 = time.time()
+    for k in range(args.steps):
+        ev[k][0].record(stream)
+        plan.sample_fwd_multi(step_no, stream)
+        ev[k][1].record(stream)
+        plan.sample_bwd_multi(step_no, stream)
+        ev[k][2].record(stream)
+        step_no += 1
+    barrier()
+    t_wall1 = time.time()
+    launches = gws.launch_count() - launches0
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    fwd_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    bwd_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    t = torch.tensor([total_ms, fwd_ms, bwd_ms], device=dev, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, fwd_ms, bwd_ms = (float(x) for x in t.tolist())
+    ms_per_step = total_ms / args.steps
+    bytes_per_step = n_elem * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM)
+    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    gelem = world * n_elem / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end through the host-buffer entry point: pinned host tensors in, results out ----
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda x: x.cpu().pin_memory()
+        block = list(range(min(7, len(specs))))            # one transformer block of pinned host buffers, reused
+        hW, hBT, hG = [pin(W[i]) for i in block], [pin(BT[i]) for i in block], [pin(G[i]) for i in block]
+        hWH = [torch.empty_like(x).pin_memory() for x in hW]
+        hSC = [torch.empty_like(x).pin_memory() for x in hBT]
+        hGBT = [torch.empty_like(x).pin_memory() for x in hBT]
+
+        def host_step(k):
+            for i in range(len(specs)):
+                j = i % len(block)
+                gws.sample_step_host(descs[i].with_step(k), hW[j], hBT[j], hG[j], hWH[j], hSC[j], hGBT[j], W[i], WH[i], G[i],
+                                     BT[i], SC[i], GBT[i], stream)
+
+        host_step(0)
+        barrier()
+        e2e_steps = 3
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for k in range(e2e_steps):
+            host_step(1 + k)
+        e1.record(stream)
+        barrier()
+        e2e_ms = torch.tensor([e0.elapsed_time(e1) / e2e_steps], device=dev, dtype=torch.float64)
+        if dist is not None:
+            dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+        n_groups = sum(s.n_groups for s in specs)
+        e2e = {"value": world * bytes_per_step / (float(e2e_ms) * 1e-3) / 1e9, "unit": "GB/s",
+               "h2d_bytes_per_step": int(n_elem * 4 + n_groups * 4), "d2h_bytes_per_step": int(n_elem * 2 + n_groups * 8),
+               "ms_per_step": float(e2e_ms), "steps": e2e_steps,
+               "note": "gws_sample_step_host per tensor; pinned host buffers of one transformer block reused for all 22"}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    traffic = ncu_traffic()
+    fwd_bytes = n_elem * FWD_BYTES_PER_ELEM
+    bwd_bytes = n_elem * BWD_BYTES_PER_ELEM
+    fwd_gbs = fwd_bytes / (fwd_ms * 1e-3) / 1e9
+    bwd_gbs = bwd_bytes / (bwd_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "tensors": len(specs), "elements": n_elem, "group": "1x128",
+                   "bits": "uniform integers 4..9", "passes": "forward + backward (identity grad_w), one launch each",
+                   "l2": "inputs larger than L2: each pass streams %.2f GB" % (n_elem * 2 / 1e9),
+                   "multi_gpu": "replicas only (no exchange step in the path)"},
+        "gelem_per_s": gelem, "hbm_frac": value / world / peak,
+        "roofline": {"bound": "hbm", "kernel": "k_flat<fwd> (gws_sample_fwd_multi)", "achieved": fwd_gbs, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": fwd_gbs / peak, "ms_per_launch": fwd_ms,
+                     "algorithmic_bytes_per_launch": fwd_bytes, "traffic": traffic.get("fwd_bytes_per_launch")},
+        "roofline_bwd": {"bound": "hbm", "kernel": "k_flat<bwd> (gws_sample_bwd_multi)", "achieved": bwd_gbs, "peak": peak,
+                         "unit": "GB/s", "frac": bwd_gbs / peak, "ms_per_launch": bwd_ms,
+                         "algorithmic_bytes_per_launch": bwd_bytes, "traffic": traffic.get("bwd_bytes_per_launch")},
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(syn.llama2_1b())
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

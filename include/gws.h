@@ -1,0 +1,218 @@
+/*
+ * gws.h - C ABI of the B200 (sm_100a) Gaussian-weight-sampling library.
+ *
+ * The library runs the per-step weight-sampling pass of GaussWS pseudo-quantization
+ * training on one GPU:
+ *
+ *   forward  (Eq. 3 + the BF16 cast of Section 3.3):
+ *       w_hat = bf16_rne( w + R * broadcast( max_group|w| * 2^(1 - b_t) ) )
+ *   backward (Eq. 4):
+ *       dL/dw = dL/dw_hat,   dL/db_t = -ln2 * max_group|w| * 2^(1-b_t) * sum_group( dL/dw_hat * R )
+ *   noise    (Section 3.4, Eq. 9 / Eq. 10): R in {-2,-1,0,1,2}, built from AND / OR of
+ *       independent random bits, regenerated in backward from the same counter (Section 3.5,
+ *       "GPU memory"; Section 3.6, "Managing seed") instead of being stored.
+ *
+ * Conventions shared by every entry point
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".  The caller owns
+ *     every buffer; the library allocates nothing, frees nothing, never synchronises the
+ *     device and only enqueues work on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream).  Inputs are never written.
+ *   - A tensor is row-major [rows, cols] of BF16 with `ld` elements between rows (ld >= cols).
+ *   - A group is group_rows x group_cols elements; group_cols == 0 means "the whole row".
+ *     Groups are numbered row-major over the ceil(rows/group_rows) x ceil(cols/group_cols)
+ *     grid, the shape the paper gives b_t under Eq. 3.  Per-group arrays (b_t, scale, absmax,
+ *     grad_bt) are dense FP32 in that order.  Edge groups may be ragged.
+ *   - Random bits: Philox4x32 with 10 rounds (Section 3.4 names Philox).  Element (i, j) has
+ *     the logical index e = elem_offset + i*cols + j (independent of ld).  Counter =
+ *     (lo32(e>>3), hi32(e>>3), lo32(step), hi32(step)), key = (lo32(seed), hi32(seed)).  One
+ *     call yields 128 bits = eight 16-bit fields; element e uses field e & 7, counted from
+ *     the least significant bits of output word 0.
+ *   - Field bits x0 (LSB) .. x15:  m2 = x0&...&x7&(x8|x9);  m1 = (x10|x11)&(x12|x13)&x14;
+ *     |R| = 2 if m2 else 1 if m1 else 0;  R is negative iff x15 is set and |R| != 0.
+ *     This gives exactly Eq. 10: Pr(+-2) = 3/4 * 2^-9 each, Pr(+-1) = (3/4)^2 * 2^-2 *
+ *     (1 - 3/1024) each.
+ *   - scale_g = fl32( absmax_g * 2^(1 - b_g) ); 2^(1-b) is exact for integer-valued b and is
+ *     computed in double then rounded to float otherwise.
+ *   - sample: y = fl32( float(w) + float(R) * scale_g ) (the product is exact, no FMA
+ *     contraction), w_hat = IEEE round-to-nearest-even of y to BF16.  R == 0 adds +0.0.
+ *   - Fast kernels need: 16-byte aligned tensor pointers, cols % 8 == 0, ld == cols,
+ *     elem_offset % 8 == 0, group_rows == 1 and group_cols in {8,16,32,64,128,256} dividing
+ *     cols, or whole-row groups with cols <= 65536.  Every other legal shape (ragged groups,
+ *     ld > cols, the paper's 32x32 square blocks, odd cols) runs on a slower general kernel
+ *     with identical results.
+ *   - NaN / Inf in the inputs give unspecified values but never a fault.
+ *
+ * Every function returns 0 (GWS_OK) or a negative gws_status.  Arguments are validated on
+ * the host before anything is launched; a failed call has enqueued nothing.
+ */
+#ifndef GWS_H_
+#define GWS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gws_status {
+  GWS_OK = 0,
+  GWS_ERR_NULL = -1,      /* a required pointer is NULL                                        */
+  GWS_ERR_SHAPE = -2,     /* rows/cols < 0, ld < cols, elem_offset % 8 != 0, n < 0             */
+  GWS_ERR_GROUP = -3,     /* group_rows < 1 or group_cols < 0                                  */
+  GWS_ERR_ALIGN = -4,     /* BF16 pointer not 2-byte aligned / FP32 or u32 pointer not 4-byte  */
+  GWS_ERR_ALIAS = -5,     /* output overlaps an input it must not overlap                      */
+  GWS_ERR_WORKSPACE = -6, /* workspace NULL, misaligned (256 B) or too small                   */
+  GWS_ERR_CUDA = -7,      /* a CUDA runtime call failed; see gws_last_cuda_error()             */
+  GWS_ERR_LIMIT = -8      /* size beyond a documented maximum                                  */
+} gws_status;
+
+/* One tensor and its noise stream. */
+typedef struct gws_desc {
+  int64_t rows, cols;   /* logical shape; cols contiguous; 0 rows or cols = nothing to do      */
+  int64_t ld;           /* elements between consecutive rows, >= cols                          */
+  int32_t group_rows;   /* >= 1; the paper's square block is 32 (Eq. 3, b_l = 32)              */
+  int32_t group_cols;   /* >= 1, or 0 for "whole row"                                          */
+  uint64_t seed;        /* per-layer seed (output of the layer PRNG of Section 3.6)            */
+  uint64_t step;        /* gradient-update counter; same value in forward and backward         */
+  uint64_t elem_offset; /* logical index of element (0,0); multiple of 8; 0 unless the tensor
+                           is a shard of a larger one whose noise stream it must reproduce     */
+} gws_desc;
+
+/* Number of groups of a descriptor (0 if rows or cols is 0, negative gws_status on error). */
+int64_t gws_n_groups(const gws_desc* desc);
+
+/*
+ * Group absolute maximum, the max_{b_l}(|w|) of Eq. 3.
+ *   w       device, BF16 [rows, ld], read only
+ *   absmax  device, FP32 [n_groups], written; exact (a BF16 magnitude widened to FP32)
+ */
+int gws_group_absmax(const gws_desc* desc, const void* w, float* absmax, void* stream);
+
+/*
+ * The noise R of Section 3.4 in the packed format of that section's last paragraph:
+ * sign-magnitude, 4 bits per element, 8 elements per 32-bit word (0.5 byte per element).
+ *   r_packed  device, u32 [ceil(rows*cols/8)], written.  Element k (logical order, no ld)
+ *             sits in word k>>3 at bits [4*(k&7), 4*(k&7)+3]; nibble = sign<<3 | |R|; zero is
+ *             never negative; unused nibbles of a last partial word are 0.
+ * Uses rows, cols, seed, step, elem_offset of the descriptor; ld and the group shape are ignored.
+ */
+int gws_noise(const gws_desc* desc, uint32_t* r_packed, void* stream);
+
+/*
+ * Forward sampling, Eq. 3 followed by the BF16 cast, in one pass over W.
+ *   w          device, BF16 [rows, ld], read only
+ *   bt         device, FP32 [n_groups], the bit-width b_t of each group, read only
+ *   w_hat      device, BF16 [rows, ld], written (padding columns ld > cols are not touched);
+ *              must not overlap w
+ *   scale_out  device, FP32 [n_groups] or NULL; receives absmax * 2^(1-b_t), the factor the
+ *              backward pass needs (W does not change between the two)
+ */
+int gws_sample_fwd(const gws_desc* desc, const void* w, const float* bt, void* w_hat, float* scale_out,
+                   void* stream);
+
+/*
+ * Backward, Eq. 4, with R regenerated from (seed, step, element index).
+ *   grad_w_hat  device, BF16 [rows, ld], dL/dw_hat, read only
+ *   scale       device, FP32 [n_groups], as written by gws_sample_fwd for the same step
+ *   grad_w      device, BF16 [rows, ld], NULL or == grad_w_hat: dL/dw is dL/dw_hat itself and
+ *               nothing is copied; any other (non-overlapping) pointer receives a bit copy
+ *   grad_bt     device, FP32 [n_groups], written: -ln2 * scale * sum_group(grad * R).  The sum
+ *               is accumulated in FP32 in a fixed order (run-to-run identical bits).
+ */
+int gws_sample_bwd(const gws_desc* desc, const void* grad_w_hat, const float* scale, void* grad_w,
+                   float* grad_bt, void* stream);
+
+/* ---- many tensors per launch ---------------------------------------------------------------
+ * One linear layer of a 1B-parameter model is a few microseconds of HBM time, so a training
+ * step samples all layers with one launch per kernel class.  The tensor set is described
+ * once (gws_multi_prepare uploads a table into caller-owned device workspace); each step then
+ * calls gws_sample_fwd_multi / gws_sample_bwd_multi with only the step counter changing.
+ */
+
+/* Host arrays of n device pointers each; the meaning of every pointer is that of the
+ * single-tensor call.  scale is written by forward and read by backward.  grad_w_hat, grad_w and
+ * grad_bt may be NULL arrays if backward is never called; w, bt, w_hat if forward is not. */
+typedef struct gws_multi_ptrs {
+  const void* const* w;
+  const float* const* bt;
+  void* const* w_hat;
+  float* const* scale;
+  const void* const* grad_w_hat;
+  void* const* grad_w; /* array may be NULL, and so may each entry: identity, no copy */
+  float* const* grad_bt;
+} gws_multi_ptrs;
+
+/* Caller-owned, filled by gws_multi_prepare, read by the *_multi calls.  Plain data. */
+typedef struct gws_multi_plan {
+  void* workspace;
+  int32_t n_tensors;
+  int32_t has_fwd, has_bwd;
+  int32_t count[4];     /* tensors per kernel class: flat groups, warp-per-row, CTA-per-row, general */
+  int64_t tiles[4];     /* thread-block tiles per class                                             */
+  int64_t fwd_offset[4], bwd_offset[4]; /* byte offsets of the class tables inside workspace         */
+  int64_t total_elements;
+} gws_multi_plan;
+
+/* Bytes of device workspace gws_multi_prepare needs for n tensors (256-byte aligned base). */
+size_t gws_workspace_bytes(int n_tensors);
+
+/*
+ * Validate n descriptors and pointer sets, build the tile tables and copy them into
+ * `workspace` on `stream` (from pageable host memory: the call may wait for earlier work
+ * on the stream, so call it outside the training loop).  desc[i].step is ignored.
+ * The workspace must stay untouched for as long as the plan is used.
+ */
+int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace,
+                      size_t workspace_bytes, gws_multi_plan* plan_out, void* stream);
+
+/* Forward / backward of every tensor of the plan for gradient-update counter `step`. */
+int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
+int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
+
+/* ---- host-buffer step (end-to-end path) --------------------------------------------------------
+ * One forward + backward of one tensor whose data lives in HOST memory (pinned memory makes the
+ * copies asynchronous).  Copies w, bt, grad_w_hat to the device staging buffers, runs
+ * gws_sample_fwd and gws_sample_bwd, copies w_hat, scale and grad_bt back, all on `stream`;
+ * returns without synchronising.
+ *   h_w, h_bt, h_grad_w_hat   host inputs  (BF16 [rows, ld], FP32 [n_groups], BF16 [rows, ld])
+ *   h_w_hat, h_scale, h_grad_bt  host outputs
+ *   d_w, d_w_hat, d_grad      device staging, each rows*ld BF16; d_bt, d_scale, d_grad_bt device
+ *                             staging, each n_groups FP32
+ */
+int gws_sample_step_host(const gws_desc* desc, const void* h_w, const float* h_bt, const void* h_grad_w_hat,
+                         void* h_w_hat, float* h_scale, float* h_grad_bt, void* d_w, void* d_w_hat, void* d_grad,
+                         float* d_bt, float* d_scale, float* d_grad_bt, void* stream);
+
+/* ---- diagnostics -----------------------------------------------------------------------------*/
+
+/* Raw Philox4x32-10 output words for vectors first_vec .. first_vec+n_vec-1 (4 words each):
+ * the random bits of Section 3.4 before decoding.  out4: device, u32 [4*n_vec]. */
+int gws_philox_words(uint64_t seed, uint64_t step, uint64_t first_vec, int64_t n_vec, uint32_t* out4,
+                     void* stream);
+
+/* Generates and decodes the noise of the descriptor exactly like gws_noise but stores only one
+ * word per thread block (an XOR of the packed words it produced): the arithmetic ceiling of noise
+ * generation without its memory traffic.  sink: device, u32 [gws_noise_alu_probe_words(desc)]. */
+int gws_noise_alu_probe(const gws_desc* desc, uint32_t* sink, void* stream);
+int64_t gws_noise_alu_probe_words(const gws_desc* desc);
+
+/* Host-side evaluation of the same inline decode / Philox code the kernels use (no GPU needed):
+ * r8 receives R for the 8 fields of the 4 words; packed receives the nibble word. */
+void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed);
+void gws_host_philox(uint64_t seed, uint64_t step, uint64_t vec, uint32_t* out4);
+
+/* Which kernel class a descriptor with fully aligned pointers would use:
+ * 0 flat groups, 1 warp per row, 2 thread block per row, 3 general; negative gws_status on error. */
+int gws_kernel_class(const gws_desc* desc);
+
+const char* gws_status_string(int status);
+/* Text of the last CUDA error this thread saw inside the library ("" if none). */
+const char* gws_last_cuda_error(void);
+/* Count of kernel launches the library has enqueued since load (all threads). */
+uint64_t gws_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GWS_H_ */

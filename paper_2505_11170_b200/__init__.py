@@ -1,0 +1,9 @@
+"""B200 (sm_100a) implementation of the weight-sampling pass of Gaussian weight sampling.
+
+``binding`` mirrors the C ABI of ``include/gws.h`` one to one (argument marshalling only);
+``synthetic`` draws seeded inputs shaped like the paper's workloads.  There is no CPU fallback:
+every call goes to the CUDA library and raises if it cannot be loaded.
+"""
+from . import synthetic  # noqa: F401
+from .binding import (GwsError, Desc, MultiPlan, group_absmax, kernel_class, launch_count, load_library, n_groups,  # noqa: F401
+                      noise, noise_alu_probe, philox_words, sample_bwd, sample_fwd, sample_step_host, status_string)

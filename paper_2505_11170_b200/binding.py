@@ -1,0 +1,274 @@
+"""Thin ctypes binding of ``include/gws.h``: one Python function per C entry point.
+
+Only argument marshalling happens here (tensor -> device pointer, current stream -> cudaStream_t,
+output allocation through torch); every step of the sampling pass runs in the CUDA library.
+If the library is missing or cannot be loaded the functions raise: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_char_p, c_float, c_int, c_int8, c_int32, c_int64, c_size_t, c_uint32, c_uint64, c_void_p
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import _build
+
+
+class GwsError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        msg = f"gws status {status}: {status_string(status)}"
+        if detail:
+            msg += f" [{detail}]"
+        super().__init__(msg)
+
+
+OK, ERR_NULL, ERR_SHAPE, ERR_GROUP, ERR_ALIGN, ERR_ALIAS, ERR_WORKSPACE, ERR_CUDA, ERR_LIMIT = 0, -1, -2, -3, -4, -5, -6, -7, -8
+
+
+class Desc(Structure):
+    """Mirror of ``gws_desc``."""
+    _fields_ = [("rows", c_int64), ("cols", c_int64), ("ld", c_int64), ("group_rows", c_int32), ("group_cols", c_int32),
+                ("seed", c_uint64), ("step", c_uint64), ("elem_offset", c_uint64)]
+
+    @staticmethod
+    def make(rows: int, cols: int, group_rows: int = 1, group_cols: int = 0, seed: int = 0, step: int = 0,
+             elem_offset: int = 0, ld: Optional[int] = None) -> "Desc":
+        return Desc(rows, cols, cols if ld is None else ld, group_rows, group_cols, seed & 0xFFFFFFFFFFFFFFFF,
+                    step & 0xFFFFFFFFFFFFFFFF, elem_offset)
+
+    def with_step(self, step: int) -> "Desc":
+        return Desc(self.rows, self.cols, self.ld, self.group_rows, self.group_cols, self.seed, step, self.elem_offset)
+
+
+class _MultiPtrs(Structure):
+    _fields_ = [("w", POINTER(c_void_p)), ("bt", POINTER(c_void_p)), ("w_hat", POINTER(c_void_p)),
+                ("scale", POINTER(c_void_p)), ("grad_w_hat", POINTER(c_void_p)), ("grad_w", POINTER(c_void_p)),
+                ("grad_bt", POINTER(c_void_p))]
+
+
+class _MultiPlan(Structure):
+    _fields_ = [("workspace", c_void_p), ("n_tensors", c_int32), ("has_fwd", c_int32), ("has_bwd", c_int32),
+                ("count", c_int32 * 4), ("tiles", c_int64 * 4), ("fwd_offset", c_int64 * 4), ("bwd_offset", c_int64 * 4),
+                ("total_elements", c_int64)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+_SIGNATURES = {
+    "gws_n_groups": (c_int64, [POINTER(Desc)]),
+    "gws_kernel_class": (c_int, [POINTER(Desc)]),
+    "gws_group_absmax": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p]),
+    "gws_noise": (c_int, [POINTER(Desc), c_void_p, c_void_p]),
+    "gws_sample_fwd": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gws_sample_bwd": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gws_workspace_bytes": (c_size_t, [c_int]),
+    "gws_multi_prepare": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, POINTER(_MultiPlan), c_void_p]),
+    "gws_sample_fwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
+    "gws_sample_bwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
+    "gws_sample_step_host": (c_int, [POINTER(Desc)] + [c_void_p] * 13),
+    "gws_philox_words": (c_int, [c_uint64, c_uint64, c_uint64, c_int64, c_void_p, c_void_p]),
+    "gws_noise_alu_probe": (c_int, [POINTER(Desc), c_void_p, c_void_p]),
+    "gws_noise_alu_probe_words": (c_int64, [POINTER(Desc)]),
+    "gws_host_decode8": (None, [POINTER(c_uint32), POINTER(c_int8), POINTER(c_uint32)]),
+    "gws_host_philox": (None, [c_uint64, c_uint64, c_uint64, POINTER(c_uint32)]),
+    "gws_status_string": (c_char_p, [c_int]),
+    "gws_last_cuda_error": (c_char_p, []),
+    "gws_launch_count": (c_uint64, []),
+}
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Load ``libgws.so`` (built in-tree by ``_build.build``) and declare its signatures."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or _build.LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(f"CUDA library {path} is missing: run `python -c 'import __graft_entry__ as g; g.build()'` "
+                           "(there is no CPU fallback)")
+    lib = ctypes.CDLL(path)
+    for name, (restype, argtypes) in _SIGNATURES.items():
+        fn = getattr(lib, name)   # AttributeError if the library does not export it
+        fn.restype = restype
+        fn.argtypes = argtypes
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().gws_status_string(status).decode()
+
+
+def _check(status: int) -> None:
+    if status != OK:
+        detail = load_library().gws_last_cuda_error().decode() if status == ERR_CUDA else ""
+        raise GwsError(status, detail)
+
+
+def _stream(stream) -> c_void_p:
+    if stream is None:
+        if not torch.cuda.is_available():
+            return c_void_p(None)    # validation-only calls on a machine without a GPU
+        stream = torch.cuda.current_stream()
+    return c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> c_void_p:
+    return c_void_p(None) if t is None else c_void_p(t.data_ptr())
+
+
+def _require_cuda(*tensors: Optional[torch.Tensor]) -> None:
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise ValueError("gws: device pointers expected (tensor is on %s)" % t.device)
+
+
+def n_groups(desc: Desc) -> int:
+    n = load_library().gws_n_groups(ctypes.byref(desc))
+    if n < 0:
+        raise GwsError(int(n))
+    return int(n)
+
+
+def kernel_class(desc: Desc) -> int:
+    c = load_library().gws_kernel_class(ctypes.byref(desc))
+    if c < 0:
+        raise GwsError(int(c))
+    return int(c)
+
+
+def launch_count() -> int:
+    return int(load_library().gws_launch_count())
+
+
+def group_absmax(desc: Desc, w: torch.Tensor, absmax: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    _require_cuda(w, absmax)
+    if absmax is None:
+        absmax = torch.empty(n_groups(desc), dtype=torch.float32, device=w.device)
+    _check(load_library().gws_group_absmax(ctypes.byref(desc), _ptr(w), _ptr(absmax), _stream(stream)))
+    return absmax
+
+
+def noise(desc: Desc, r_packed: Optional[torch.Tensor] = None, device="cuda", stream=None) -> torch.Tensor:
+    """Packed 4-bit sign-magnitude noise, int32 tensor of ceil(rows*cols/8) words."""
+    if r_packed is None:
+        r_packed = torch.empty((desc.rows * desc.cols + 7) // 8, dtype=torch.int32, device=device)
+    _require_cuda(r_packed)
+    _check(load_library().gws_noise(ctypes.byref(desc), _ptr(r_packed), _stream(stream)))
+    return r_packed
+
+
+def sample_fwd(desc: Desc, w: torch.Tensor, bt: torch.Tensor, w_hat: Optional[torch.Tensor] = None,
+               scale_out: Optional[torch.Tensor] = None, want_scale: bool = True, stream=None):
+    """Returns (w_hat, scale_out)."""
+    _require_cuda(w, bt, w_hat, scale_out)
+    if w_hat is None:
+        w_hat = torch.empty_like(w)
+    if scale_out is None and want_scale:
+        scale_out = torch.empty(n_groups(desc), dtype=torch.float32, device=w.device)
+    _check(load_library().gws_sample_fwd(ctypes.byref(desc), _ptr(w), _ptr(bt), _ptr(w_hat), _ptr(scale_out), _stream(stream)))
+    return w_hat, scale_out
+
+
+def sample_bwd(desc: Desc, grad_w_hat: torch.Tensor, scale: torch.Tensor, grad_w: Optional[torch.Tensor] = None,
+               grad_bt: Optional[torch.Tensor] = None, stream=None):
+    """Returns (grad_w, grad_bt); grad_w is ``grad_w_hat`` itself when no copy was requested."""
+    _require_cuda(grad_w_hat, scale, grad_w, grad_bt)
+    if grad_bt is None:
+        grad_bt = torch.empty(n_groups(desc), dtype=torch.float32, device=grad_w_hat.device)
+    _check(load_library().gws_sample_bwd(ctypes.byref(desc), _ptr(grad_w_hat), _ptr(scale), _ptr(grad_w), _ptr(grad_bt),
+                                         _stream(stream)))
+    return (grad_w_hat if grad_w is None else grad_w), grad_bt
+
+
+def philox_words(seed: int, step: int, first_vec: int, n_vec: int, out: Optional[torch.Tensor] = None, device="cuda",
+                 stream=None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty((n_vec, 4), dtype=torch.int32, device=device)
+    _require_cuda(out)
+    _check(load_library().gws_philox_words(seed, step, first_vec, n_vec, _ptr(out), _stream(stream)))
+    return out
+
+
+def noise_alu_probe(desc: Desc, sink: Optional[torch.Tensor] = None, device="cuda", stream=None) -> torch.Tensor:
+    lib = load_library()
+    if sink is None:
+        sink = torch.empty(max(1, int(lib.gws_noise_alu_probe_words(ctypes.byref(desc)))), dtype=torch.int32, device=device)
+    _require_cuda(sink)
+    _check(lib.gws_noise_alu_probe(ctypes.byref(desc), _ptr(sink), _stream(stream)))
+    return sink
+
+
+def _ptr_array(tensors: Optional[Sequence[Optional[torch.Tensor]]], n: int):
+    if tensors is None:
+        return None
+    assert len(tensors) == n
+    return (c_void_p * n)(*[None if t is None else t.data_ptr() for t in tensors])
+
+
+class MultiPlan:
+    """``gws_multi_prepare`` + the two ``*_multi`` launches for a fixed set of tensors."""
+
+    def __init__(self, descs: Sequence[Desc], w=None, bt=None, w_hat=None, scale=None, grad_w_hat=None, grad_w=None,
+                 grad_bt=None, stream=None):
+        lib = load_library()
+        n = len(descs)
+        anyt = next(t for group in (w, grad_w_hat) if group is not None for t in group if t is not None)
+        _require_cuda(anyt)
+        self._keep = [w, bt, w_hat, scale, grad_w_hat, grad_w, grad_bt]    # the plan holds raw pointers
+        self._descs = (Desc * n)(*descs)
+        arrays = [_ptr_array(g, n) for g in self._keep]
+        cast = lambda a: ctypes.cast(a, POINTER(c_void_p)) if a is not None else None
+        self._ptrs = _MultiPtrs(*[cast(a) for a in arrays])
+        nbytes = int(lib.gws_workspace_bytes(n))
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=anyt.device)
+        self.plan = _MultiPlan()
+        _check(lib.gws_multi_prepare(n, self._descs, ctypes.byref(self._ptrs), _ptr(self.workspace), nbytes,
+                                     ctypes.byref(self.plan), _stream(stream)))
+
+    @property
+    def total_elements(self) -> int:
+        return int(self.plan.total_elements)
+
+    @property
+    def launches_per_pass(self) -> int:
+        c = list(self.plan.count)
+        return sum(1 for k in range(3) if c[k]) + c[3]
+
+    def sample_fwd_multi(self, step: int, stream=None) -> None:
+        _check(load_library().gws_sample_fwd_multi(ctypes.byref(self.plan), step, _stream(stream)))
+
+    def sample_bwd_multi(self, step: int, stream=None) -> None:
+        _check(load_library().gws_sample_bwd_multi(ctypes.byref(self.plan), step, _stream(stream)))
+
+
+def sample_step_host(desc: Desc, h_w, h_bt, h_grad, h_w_hat, h_scale, h_grad_bt, d_w, d_w_hat, d_grad, d_bt, d_scale,
+                     d_grad_bt, stream=None) -> None:
+    """Forward + backward of one tensor held in host memory (pinned tensors make the copies asynchronous)."""
+    for t in (h_w, h_bt, h_grad, h_w_hat, h_scale, h_grad_bt):
+        if t.is_cuda:
+            raise ValueError("gws: host tensors expected")
+    _require_cuda(d_w, d_w_hat, d_grad, d_bt, d_scale, d_grad_bt)
+    _check(load_library().gws_sample_step_host(ctypes.byref(desc), _ptr(h_w), _ptr(h_bt), _ptr(h_grad), _ptr(h_w_hat),
+                                               _ptr(h_scale), _ptr(h_grad_bt), _ptr(d_w), _ptr(d_w_hat), _ptr(d_grad),
+                                               _ptr(d_bt), _ptr(d_scale), _ptr(d_grad_bt), _stream(stream)))
+
+
+# ---- host-side diagnostics (no GPU needed) ------------------------------------------------------------
+
+def host_decode8(words4: Sequence[int]):
+    """(R[8], packed nibble word) computed on the CPU by the same inline code the kernels use."""
+    w = (c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in words4])
+    r = (c_int8 * 8)()
+    p = c_uint32(0)
+    load_library().gws_host_decode8(w, r, ctypes.byref(p))
+    return list(r), int(p.value)
+
+
+def host_philox(seed: int, step: int, vec: int) -> List[int]:
+    o = (c_uint32 * 4)()
+    load_library().gws_host_philox(seed, step, vec, o)
+    return list(o)

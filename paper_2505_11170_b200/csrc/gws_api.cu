@@ -1,0 +1,461 @@
+// Host side of the C ABI declared in gws.h: argument validation, choice of kernel class,
+// launch geometry, the multi-tensor table.  No device memory is allocated here.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "gws.h"
+#include "gws_kernels.cuh"
+
+namespace {
+
+using gws::Entry;
+
+thread_local std::string g_last_cuda_error;
+std::atomic<uint64_t> g_launches{0};
+
+constexpr int64_t kMaxGrid = 2147483647LL;
+constexpr int kGeneralGrid = 148 * 8;
+
+int cuda_fail(cudaError_t err, const char* what) {
+  g_last_cuda_error = std::string(what) + ": " + cudaGetErrorString(err);
+  return GWS_ERR_CUDA;
+}
+
+int check_launch(const char* what) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  const cudaError_t err = cudaGetLastError();
+  return err == cudaSuccess ? GWS_OK : cuda_fail(err, what);
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int validate_desc(const gws_desc* d) {
+  if (d == nullptr) return GWS_ERR_NULL;
+  if (d->rows < 0 || d->cols < 0) return GWS_ERR_SHAPE;
+  if (d->rows > 0 && d->cols > 0 && d->ld < d->cols) return GWS_ERR_SHAPE;
+  if (d->elem_offset % 8 != 0) return GWS_ERR_SHAPE;
+  if (d->group_rows < 1 || d->group_cols < 0) return GWS_ERR_GROUP;
+  if (d->rows > 0 && d->cols > 0 && (d->rows > (INT64_MAX / 4) / d->cols || d->rows > (INT64_MAX / 4) / d->ld))
+    return GWS_ERR_LIMIT;
+  return GWS_OK;
+}
+
+bool is_empty(const gws_desc* d) { return d->rows == 0 || d->cols == 0; }
+
+int64_t resolved_group_cols(const gws_desc* d) { return d->group_cols == 0 ? d->cols : d->group_cols; }
+
+int64_t n_groups_of(const gws_desc* d) {
+  if (is_empty(d)) return 0;
+  const int64_t gc = resolved_group_cols(d);
+  return ((d->rows + d->group_rows - 1) / d->group_rows) * ((d->cols + gc - 1) / gc);
+}
+
+// Bytes spanned by a [rows, ld] BF16 tensor with `cols` used columns.
+size_t span_bytes(const gws_desc* d) { return static_cast<size_t>((d->rows - 1) * d->ld + d->cols) * 2u; }
+
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+  return x < y + nb && y < x + na;
+}
+
+// Kernel class for a descriptor; `vec_ok` says whether every tensor pointer is 16-byte aligned.
+int classify(const gws_desc* d, bool vec_ok) {
+  const int64_t gc = resolved_group_cols(d);
+  const bool dense = vec_ok && d->ld == d->cols && d->cols % 8 == 0 && d->group_rows == 1;
+  if (!dense) return gws::kGeneral;
+  if (gc <= 256 && gc >= 8 && (gc & (gc - 1)) == 0 && d->cols % gc == 0) return gws::kFlat;
+  if (gc == d->cols) {
+    const int64_t vpr = d->cols / 8;
+    if (vpr <= 32 * gws::kRowWarpVecs) return gws::kRowWarp;
+    if (vpr <= static_cast<int64_t>(gws::kRowCtaThreads) * gws::kRowCtaVecs) return gws::kRowCta;
+  }
+  return gws::kGeneral;
+}
+
+int64_t tiles_of(const gws_desc* d, int cls) {
+  switch (cls) {
+    case gws::kFlat: {
+      const int64_t n_vec = d->rows * d->cols / 8;
+      const int64_t per = static_cast<int64_t>(gws::kFlatThreads) * gws::kFlatVecs;
+      return (n_vec + per - 1) / per;
+    }
+    case gws::kRowWarp:
+      return (d->rows + (gws::kRowWarpThreads / 32) - 1) / (gws::kRowWarpThreads / 32);
+    case gws::kRowCta:
+      return d->rows;
+    default: {
+      const int64_t ng = n_groups_of(d);
+      return ng < kGeneralGrid ? ng : kGeneralGrid;
+    }
+  }
+}
+
+Entry make_entry(const gws_desc* d, int cls, const void* in, void* out, const float* gin, float* gout) {
+  Entry e;
+  std::memset(&e, 0, sizeof e);
+  e.in = in;
+  e.out = out;
+  e.gin = gin;
+  e.gout = gout;
+  e.rows = d->rows;
+  e.cols = d->cols;
+  e.ld = d->ld;
+  e.group_rows = d->group_rows;
+  e.group_cols = static_cast<int32_t>(resolved_group_cols(d) > INT32_MAX ? INT32_MAX : resolved_group_cols(d));
+  e.elem_offset = d->elem_offset;
+  e.n_vec = static_cast<uint64_t>(d->rows * d->cols / 8);
+  e.seed_lo = static_cast<uint32_t>(d->seed);
+  e.seed_hi = static_cast<uint32_t>(d->seed >> 32);
+  e.vpr = static_cast<uint32_t>(d->cols / 8);
+  e.lanes_log2 = 0;
+  if (cls == gws::kFlat) {
+    int64_t lanes = resolved_group_cols(d) / 8;
+    while (lanes > 1) { lanes >>= 1; ++e.lanes_log2; }
+  }
+  e.tile_begin = 0;
+  return e;
+}
+
+template <int MODE>
+int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int64_t tiles, uint64_t step,
+           cudaStream_t stream) {
+  if (tiles <= 0) return GWS_OK;
+  if (tiles > kMaxGrid) return GWS_ERR_LIMIT;
+  const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
+  const unsigned grid = static_cast<unsigned>(tiles);
+  switch (cls) {
+    case gws::kFlat:
+      gws::k_flat<MODE><<<grid, gws::kFlatThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      return check_launch("flat-group kernel");
+    case gws::kRowWarp:
+      gws::k_row_warp<MODE><<<grid, gws::kRowWarpThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      return check_launch("warp-per-row kernel");
+    case gws::kRowCta:
+      gws::k_row_cta<MODE><<<grid, gws::kRowCtaThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      return check_launch("block-per-row kernel");
+    default:
+      gws::k_general<MODE><<<grid, gws::kGeneralThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      return check_launch("general kernel");
+  }
+}
+
+// Shared checks of the single-tensor calls.  Returns 1 if there is nothing to do.
+int precheck(const gws_desc* d) {
+  const int st = validate_desc(d);
+  if (st != GWS_OK) return st;
+  return is_empty(d) ? 1 : GWS_OK;
+}
+
+struct ClassTables {
+  std::vector<Entry> fwd[4], bwd[4];
+};
+
+}  // namespace
+
+extern "C" {
+
+int64_t gws_n_groups(const gws_desc* desc) {
+  const int st = validate_desc(desc);
+  if (st != GWS_OK) return st;
+  return n_groups_of(desc);
+}
+
+int gws_kernel_class(const gws_desc* desc) {
+  const int st = validate_desc(desc);
+  if (st != GWS_OK) return st;
+  return classify(desc, true);
+}
+
+int gws_group_absmax(const gws_desc* desc, const void* w, float* absmax, void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (w == nullptr || absmax == nullptr) return GWS_ERR_NULL;
+  if (!aligned(w, 2) || !aligned(absmax, 4)) return GWS_ERR_ALIGN;
+  const int cls = classify(desc, aligned(w, 16));
+  const Entry e = make_entry(desc, cls, w, nullptr, nullptr, absmax);
+  return launch<gws::kAbsmax>(cls, e, nullptr, 0, tiles_of(desc, cls), desc->step, static_cast<cudaStream_t>(stream));
+}
+
+int gws_sample_fwd(const gws_desc* desc, const void* w, const float* bt, void* w_hat, float* scale_out, void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (w == nullptr || bt == nullptr || w_hat == nullptr) return GWS_ERR_NULL;
+  if (!aligned(w, 2) || !aligned(w_hat, 2) || !aligned(bt, 4) || !aligned(scale_out, 4)) return GWS_ERR_ALIGN;
+  if (overlaps(w, span_bytes(desc), w_hat, span_bytes(desc))) return GWS_ERR_ALIAS;
+  const int cls = classify(desc, aligned(w, 16) && aligned(w_hat, 16));
+  const Entry e = make_entry(desc, cls, w, w_hat, bt, scale_out);
+  return launch<gws::kFwd>(cls, e, nullptr, 0, tiles_of(desc, cls), desc->step, static_cast<cudaStream_t>(stream));
+}
+
+int gws_sample_bwd(const gws_desc* desc, const void* grad_w_hat, const float* scale, void* grad_w, float* grad_bt,
+                   void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (grad_w_hat == nullptr || scale == nullptr || grad_bt == nullptr) return GWS_ERR_NULL;
+  if (!aligned(grad_w_hat, 2) || !aligned(grad_w, 2) || !aligned(scale, 4) || !aligned(grad_bt, 4)) return GWS_ERR_ALIGN;
+  if (grad_w == grad_w_hat) grad_w = nullptr;  // identity: nothing to copy
+  if (grad_w != nullptr && overlaps(grad_w_hat, span_bytes(desc), grad_w, span_bytes(desc))) return GWS_ERR_ALIAS;
+  const int cls = classify(desc, aligned(grad_w_hat, 16) && aligned(grad_w, 16));
+  const Entry e = make_entry(desc, cls, grad_w_hat, grad_w, scale, grad_bt);
+  return launch<gws::kBwd>(cls, e, nullptr, 0, tiles_of(desc, cls), desc->step, static_cast<cudaStream_t>(stream));
+}
+
+int gws_noise(const gws_desc* desc, uint32_t* r_packed, void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (r_packed == nullptr) return GWS_ERR_NULL;
+  if (!aligned(r_packed, 4)) return GWS_ERR_ALIGN;
+  const uint64_t n_elems = static_cast<uint64_t>(desc->rows * desc->cols);
+  const uint64_t n_words = (n_elems + 7u) / 8u;
+  const uint64_t blocks = (n_words + 255u) / 256u;
+  if (blocks > static_cast<uint64_t>(kMaxGrid)) return GWS_ERR_LIMIT;
+  gws::k_noise<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      r_packed, n_words, n_elems, desc->elem_offset >> 3, static_cast<uint32_t>(desc->seed),
+      static_cast<uint32_t>(desc->seed >> 32), static_cast<uint32_t>(desc->step), static_cast<uint32_t>(desc->step >> 32));
+  return check_launch("noise kernel");
+}
+
+int64_t gws_noise_alu_probe_words(const gws_desc* desc) {
+  const int st = validate_desc(desc);
+  if (st != GWS_OK) return st;
+  const uint64_t n_words = (static_cast<uint64_t>(desc->rows * desc->cols) + 7u) / 8u;
+  return static_cast<int64_t>((n_words + 2047u) / 2048u);
+}
+
+int gws_noise_alu_probe(const gws_desc* desc, uint32_t* sink, void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (sink == nullptr) return GWS_ERR_NULL;
+  if (!aligned(sink, 4)) return GWS_ERR_ALIGN;
+  const uint64_t n_words = (static_cast<uint64_t>(desc->rows * desc->cols) + 7u) / 8u;
+  const uint64_t blocks = (n_words + 2047u) / 2048u;
+  if (blocks > static_cast<uint64_t>(kMaxGrid)) return GWS_ERR_LIMIT;
+  gws::k_noise_probe<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      sink, n_words, desc->elem_offset >> 3, static_cast<uint32_t>(desc->seed), static_cast<uint32_t>(desc->seed >> 32),
+      static_cast<uint32_t>(desc->step), static_cast<uint32_t>(desc->step >> 32));
+  return check_launch("noise arithmetic probe");
+}
+
+int gws_philox_words(uint64_t seed, uint64_t step, uint64_t first_vec, int64_t n_vec, uint32_t* out4, void* stream) {
+  if (n_vec < 0) return GWS_ERR_SHAPE;
+  if (n_vec == 0) return GWS_OK;
+  if (out4 == nullptr) return GWS_ERR_NULL;
+  if (!aligned(out4, 16)) return GWS_ERR_ALIGN;
+  const uint64_t blocks = (static_cast<uint64_t>(n_vec) + 255u) / 256u;
+  if (blocks > static_cast<uint64_t>(kMaxGrid)) return GWS_ERR_LIMIT;
+  gws::k_philox_words<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<uint4*>(out4), static_cast<uint64_t>(n_vec), first_vec, static_cast<uint32_t>(seed),
+      static_cast<uint32_t>(seed >> 32), static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32));
+  return check_launch("philox words kernel");
+}
+
+// ---- many tensors -------------------------------------------------------------------------------
+
+size_t gws_workspace_bytes(int n_tensors) {
+  if (n_tensors < 0) return 0;
+  // two tables (forward, backward) of at most n entries, each of the 8 class tables 256-byte aligned
+  return static_cast<size_t>(n_tensors) * 2u * sizeof(Entry) + 8u * 256u;
+}
+
+int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace, size_t workspace_bytes,
+                      gws_multi_plan* plan_out, void* stream) {
+  if (n < 0) return GWS_ERR_SHAPE;
+  if (descs == nullptr || ptrs == nullptr || plan_out == nullptr) return GWS_ERR_NULL;
+  const bool has_fwd = ptrs->w != nullptr;
+  const bool has_bwd = ptrs->grad_w_hat != nullptr;
+  if (!has_fwd && !has_bwd) return GWS_ERR_NULL;
+  if (has_fwd && (ptrs->bt == nullptr || ptrs->w_hat == nullptr)) return GWS_ERR_NULL;
+  if (has_bwd && (ptrs->scale == nullptr || ptrs->grad_bt == nullptr)) return GWS_ERR_NULL;
+  if (workspace == nullptr || !aligned(workspace, 256) || workspace_bytes < gws_workspace_bytes(n)) return GWS_ERR_WORKSPACE;
+
+  ClassTables t;
+  int64_t total = 0;
+  for (int i = 0; i < n; ++i) {
+    const gws_desc* d = &descs[i];
+    const int st = validate_desc(d);
+    if (st != GWS_OK) return st;
+    if (is_empty(d)) continue;
+    bool vec_ok = true;
+    float* scale = ptrs->scale ? ptrs->scale[i] : nullptr;
+    if (has_fwd) {
+      const void* w = ptrs->w[i];
+      void* w_hat = ptrs->w_hat[i];
+      const float* bt = ptrs->bt[i];
+      if (w == nullptr || w_hat == nullptr || bt == nullptr) return GWS_ERR_NULL;
+      if (!aligned(w, 2) || !aligned(w_hat, 2) || !aligned(bt, 4) || !aligned(scale, 4)) return GWS_ERR_ALIGN;
+      if (overlaps(w, span_bytes(d), w_hat, span_bytes(d))) return GWS_ERR_ALIAS;
+      vec_ok = vec_ok && aligned(w, 16) && aligned(w_hat, 16);
+    }
+    void* gw = nullptr;
+    if (has_bwd) {
+      const void* g = ptrs->grad_w_hat[i];
+      gw = ptrs->grad_w ? ptrs->grad_w[i] : nullptr;
+      float* gbt = ptrs->grad_bt[i];
+      if (g == nullptr || scale == nullptr || gbt == nullptr) return GWS_ERR_NULL;
+      if (!aligned(g, 2) || !aligned(gw, 2) || !aligned(scale, 4) || !aligned(gbt, 4)) return GWS_ERR_ALIGN;
+      if (gw == g) gw = nullptr;
+      if (gw != nullptr && overlaps(g, span_bytes(d), gw, span_bytes(d))) return GWS_ERR_ALIAS;
+      vec_ok = vec_ok && aligned(g, 16) && aligned(gw, 16);
+    }
+    const int cls = classify(d, vec_ok);
+    const int64_t tiles = tiles_of(d, cls);
+    total += d->rows * d->cols;
+    if (has_fwd) {
+      Entry e = make_entry(d, cls, ptrs->w[i], ptrs->w_hat[i], ptrs->bt[i], scale);
+      e.tile_begin = tiles;  // turned into a prefix sum below
+      t.fwd[cls].push_back(e);
+    }
+    if (has_bwd) {
+      Entry e = make_entry(d, cls, ptrs->grad_w_hat[i], gw, scale, ptrs->grad_bt[i]);
+      e.tile_begin = tiles;
+      t.bwd[cls].push_back(e);
+    }
+  }
+
+  gws_multi_plan plan;
+  std::memset(&plan, 0, sizeof plan);
+  plan.workspace = workspace;
+  plan.n_tensors = n;
+  plan.has_fwd = has_fwd ? 1 : 0;
+  plan.has_bwd = has_bwd ? 1 : 0;
+  plan.total_elements = total;
+  size_t offset = 0;
+  auto place = [&](std::vector<Entry>& v, int cls, int64_t* where, bool general) -> int {
+    int64_t running = 0;
+    for (Entry& e : v) {
+      const int64_t tiles = e.tile_begin;
+      e.tile_begin = running;
+      running += tiles;
+    }
+    if (!general && running > kMaxGrid) return GWS_ERR_LIMIT;
+    plan.count[cls] = static_cast<int32_t>(v.size());
+    plan.tiles[cls] = running;
+    *where = static_cast<int64_t>(offset);
+    if (!v.empty()) {
+      const size_t bytes = v.size() * sizeof(Entry);
+      const cudaError_t err = cudaMemcpyAsync(static_cast<char*>(workspace) + offset, v.data(), bytes,
+                                              cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream));
+      if (err != cudaSuccess) return cuda_fail(err, "table upload");
+      offset += (bytes + 255u) & ~static_cast<size_t>(255u);
+    }
+    return GWS_OK;
+  };
+  for (int cls = 0; cls < 4; ++cls) {
+    int st = GWS_OK;
+    if (has_fwd) st = place(t.fwd[cls], cls, &plan.fwd_offset[cls], cls == gws::kGeneral);
+    if (st != GWS_OK) return st;
+    if (has_bwd) st = place(t.bwd[cls], cls, &plan.bwd_offset[cls], cls == gws::kGeneral);
+    if (st != GWS_OK) return st;
+  }
+  // The uploads read pageable host memory that dies with this call: wait for them.
+  const cudaError_t err = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) return cuda_fail(err, "table upload");
+  *plan_out = plan;
+  return GWS_OK;
+}
+
+static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream, bool backward) {
+  if (plan == nullptr) return GWS_ERR_NULL;
+  if (plan->workspace == nullptr) return GWS_ERR_WORKSPACE;
+  if (backward ? !plan->has_bwd : !plan->has_fwd) return GWS_ERR_NULL;
+  const Entry none{};
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  for (int cls = 0; cls < 4; ++cls) {
+    const int count = plan->count[cls];
+    if (count == 0) continue;
+    const Entry* table = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->workspace) +
+                                                        (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
+    if (cls != gws::kGeneral) {
+      const int st = backward ? launch<gws::kBwd>(cls, none, table, count, plan->tiles[cls], step, s)
+                              : launch<gws::kFwd>(cls, none, table, count, plan->tiles[cls], step, s);
+      if (st != GWS_OK) return st;
+    } else {
+      for (int i = 0; i < count; ++i) {
+        const int st = backward ? launch<gws::kBwd>(cls, none, table, i, kGeneralGrid, step, s)
+                                : launch<gws::kFwd>(cls, none, table, i, kGeneralGrid, step, s);
+        if (st != GWS_OK) return st;
+      }
+    }
+  }
+  return GWS_OK;
+}
+
+int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
+  return run_multi(plan, step, stream, false);
+}
+
+int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
+  return run_multi(plan, step, stream, true);
+}
+
+// ---- host-buffer step ---------------------------------------------------------------------------
+
+int gws_sample_step_host(const gws_desc* desc, const void* h_w, const float* h_bt, const void* h_grad_w_hat,
+                         void* h_w_hat, float* h_scale, float* h_grad_bt, void* d_w, void* d_w_hat, void* d_grad,
+                         float* d_bt, float* d_scale, float* d_grad_bt, void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (!h_w || !h_bt || !h_grad_w_hat || !h_w_hat || !h_scale || !h_grad_bt || !d_w || !d_w_hat || !d_grad || !d_bt ||
+      !d_scale || !d_grad_bt)
+    return GWS_ERR_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t tb = span_bytes(desc), gb = static_cast<size_t>(n_groups_of(desc)) * sizeof(float);
+  cudaError_t err;
+  if ((err = cudaMemcpyAsync(d_w, h_w, tb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(err, "copy w");
+  if ((err = cudaMemcpyAsync(d_bt, h_bt, gb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(err, "copy bt");
+  if ((err = cudaMemcpyAsync(d_grad, h_grad_w_hat, tb, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+    return cuda_fail(err, "copy grad");
+  int r = gws_sample_fwd(desc, d_w, d_bt, d_w_hat, d_scale, stream);
+  if (r != GWS_OK) return r;
+  r = gws_sample_bwd(desc, d_grad, d_scale, nullptr, d_grad_bt, stream);
+  if (r != GWS_OK) return r;
+  if ((err = cudaMemcpyAsync(h_w_hat, d_w_hat, tb, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+    return cuda_fail(err, "copy w_hat");
+  if ((err = cudaMemcpyAsync(h_scale, d_scale, gb, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+    return cuda_fail(err, "copy scale");
+  if ((err = cudaMemcpyAsync(h_grad_bt, d_grad_bt, gb, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+    return cuda_fail(err, "copy grad_bt");
+  return GWS_OK;
+}
+
+// ---- diagnostics ----------------------------------------------------------------------------------
+
+void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed) {
+  gws::Words4 w;
+  for (int k = 0; k < 4; ++k) w.o[k] = words4[k];
+  uint32_t p[4];
+  gws::decode4(w.o[0], w.o[1], p[0], p[1]);
+  gws::decode4(w.o[2], w.o[3], p[2], p[3]);
+  for (unsigned t = 0; t < 8; ++t) r8[t] = static_cast<int8_t>(gws::r_from_pair(p[t >> 1], t & 1u));
+  if (packed) *packed = gws::pack_nibbles(w);
+}
+
+void gws_host_philox(uint64_t seed, uint64_t step, uint64_t vec, uint32_t* out4) {
+  const gws::Words4 w = gws::philox_for_vector(vec, static_cast<uint32_t>(step), static_cast<uint32_t>(step >> 32),
+                                               static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32));
+  for (int k = 0; k < 4; ++k) out4[k] = w.o[k];
+}
+
+const char* gws_status_string(int status) {
+  switch (status) {
+    case GWS_OK: return "ok";
+    case GWS_ERR_NULL: return "a required pointer is NULL";
+    case GWS_ERR_SHAPE: return "bad shape: negative size, ld < cols, or elem_offset not a multiple of 8";
+    case GWS_ERR_GROUP: return "bad group shape: group_rows < 1 or group_cols < 0";
+    case GWS_ERR_ALIGN: return "pointer not aligned to its element type";
+    case GWS_ERR_ALIAS: return "output overlaps an input";
+    case GWS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case GWS_ERR_CUDA: return "CUDA runtime error (see gws_last_cuda_error)";
+    case GWS_ERR_LIMIT: return "size beyond a documented maximum";
+    default: return "unknown status";
+  }
+}
+
+const char* gws_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+uint64_t gws_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

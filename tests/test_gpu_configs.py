@@ -1,0 +1,139 @@
+"""The benchmark configurations at full size, in the launch configuration the benchmark times
+(one multi-tensor launch per kernel class), against the oracle: completely where the oracle
+finishes in seconds, on sampled tensors / row slices otherwise (every group is independent, and
+a row slice with elem_offset = first_row * cols reproduces the noise stream of the full tensor)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2505_11170_b200 as gws
+from oracle import gws_oracle as orc
+from paper_2505_11170_b200 import synthetic as syn
+from paper_2505_11170_b200.binding import Desc
+from util import bits_of
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+REL = 1e-5
+
+
+def _slice_check(spec, desc_seed, step, w, bt, w_hat, scale, g, gbt, r0, nrows):
+    """Oracle on rows [r0, r0+nrows) of one tensor (groups must not straddle the slice)."""
+    cols = spec.cols
+    gc = cols if spec.group_cols == 0 else spec.group_cols
+    gpr = cols // gc
+    sl = slice(r0, r0 + nrows)
+    gsl = slice(r0 * gpr, (r0 + nrows) * gpr)
+    hat, sc = orc.sample_fwd(bits_of(w[sl]), bt[gsl].cpu().numpy(), nrows, cols, 1, spec.group_cols, seed=desc_seed,
+                             step=step, elem_offset=r0 * cols)
+    assert (bits_of(w_hat[sl]).ravel() == hat).all(), (spec.name, step, r0)
+    assert (scale[gsl].cpu().numpy().view(np.uint32) == sc.view(np.uint32)).all()
+    if g is not None:
+        _, want = orc.sample_bwd(bits_of(g[sl]), sc, nrows, cols, 1, spec.group_cols, seed=desc_seed, step=step,
+                                 elem_offset=r0 * cols)
+        got = gbt[gsl].cpu().numpy().astype(np.float64)
+        r = orc.noise_r(desc_seed, step, r0 * cols, nrows * cols).astype(np.float64)
+        gf = g[sl].float().cpu().numpy().astype(np.float64).reshape(-1)
+        sums = np.abs(gf * r).reshape(nrows * gpr, gc).sum(axis=1)
+        bound = REL * np.log(2.0) * sc.astype(np.float64) * sums
+        assert (np.abs(got - want) <= bound + 1e-45).all(), (spec.name, step, r0)
+        assert np.abs(got - want).max() <= REL * np.abs(want).max() + 1e-45
+
+
+@pytest.mark.parametrize("literal", [False, True])
+def test_config1_gpt2_single_mlp_weight(literal):
+    spec = syn.gpt2_124m_single(literal)[0]
+    w = syn.weights(spec, 0)
+    bt = syn.bitwidths(spec, 0, fixed=6.0)
+    d = Desc.make(spec.rows, spec.cols, 1, 0, seed=syn.layer_seed(0, 0), step=0)
+    w_hat, sc = gws.sample_fwd(d, w.to(DEV), bt.to(DEV))
+    hat, want_sc = orc.sample_fwd(bits_of(w), bt.numpy(), spec.rows, spec.cols, 1, 0, seed=d.seed, step=0)
+    assert (bits_of(w_hat).ravel() == hat).all()
+    assert (sc.cpu().numpy().view(np.uint32) == want_sc.view(np.uint32)).all()
+    packed = gws.noise(d).cpu().numpy().view(np.uint32)
+    assert (packed == orc.noise_packed(d.seed, 0, 0, spec.numel)).all()
+
+
+def _device_set(specs, device=DEV):
+    W = [syn.weights(s, i, device=device) for i, s in enumerate(specs)]
+    BT = [syn.bitwidths(s, i, device=device) for i, s in enumerate(specs)]
+    G = [syn.upstream_grad(s, i, device=device) for i, s in enumerate(specs)]
+    WH = [torch.empty_like(t) for t in W]
+    SC = [torch.empty(s.n_groups, device=device) for s in specs]
+    GBT = [torch.empty(s.n_groups, device=device) for s in specs]
+    descs = [Desc.make(s.rows, s.cols, s.group_rows, s.group_cols, seed=syn.layer_seed(0, i)) for i, s in enumerate(specs)]
+    return descs, W, BT, G, WH, SC, GBT
+
+
+def test_config2_gpt2_all_linear_weights_forward_backward():
+    specs = syn.gpt2_124m_all()
+    assert syn.total_elements(specs) == 84934656 and sum(s.n_groups for s in specs) == 82944
+    descs, W, BT, G, WH, SC, GBT = _device_set(specs)
+    plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=WH, scale=SC, grad_w_hat=G, grad_bt=GBT)
+    assert plan.launches_per_pass == 1                     # every tensor is a warp-per-row tensor
+    plan.sample_fwd_multi(0)
+    plan.sample_bwd_multi(0)
+    torch.cuda.synchronize()
+    # whole tensors of block 0 and block 11, row slices of the rest
+    for i, s in enumerate(specs):
+        if i < 4 or i >= 44:
+            _slice_check(s, descs[i].seed, 0, W[i], BT[i], WH[i], SC[i], G[i], GBT[i], 0, s.rows)
+        else:
+            r0 = (i * 97) % (s.rows - 16)
+            _slice_check(s, descs[i].seed, 0, W[i], BT[i], WH[i], SC[i], G[i], GBT[i], r0, 16)
+
+
+def test_config3_llama2_1b_ten_steps():
+    specs = syn.llama2_1b()
+    assert syn.total_elements(specs) == 1130364928 and sum(s.n_groups for s in specs) == 8830976
+    descs, W, BT, G, WH, SC, GBT = _device_set(specs)
+    plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=WH, scale=SC, grad_w_hat=G, grad_bt=GBT)
+    assert plan.launches_per_pass == 1
+    rng = np.random.default_rng(3)
+    for step in range(10):
+        plan.sample_fwd_multi(step)
+        plan.sample_bwd_multi(step)
+        torch.cuda.synchronize()
+        if step in (0, 9):
+            # two whole tensors (one square, one wide) plus a slice of every tensor
+            for i in (0, 6) if step == 0 else (4, 153):
+                _slice_check(specs[i], descs[i].seed, step, W[i], BT[i], WH[i], SC[i], G[i], GBT[i], 0, specs[i].rows)
+            for i, s in enumerate(specs):
+                r0 = int(rng.integers(0, s.rows - 8))
+                _slice_check(s, descs[i].seed, step, W[i], BT[i], WH[i], SC[i], G[i], GBT[i], r0, 8)
+        else:
+            for i in rng.choice(len(specs), 6, replace=False):
+                s = specs[int(i)]
+                r0 = int(rng.integers(0, s.rows - 8))
+                _slice_check(s, descs[int(i)].seed, step, W[int(i)], BT[int(i)], WH[int(i)], SC[int(i)], G[int(i)],
+                             GBT[int(i)], r0, 8)
+    # the last rows (tail tile) of the last tensor
+    s = specs[-1]
+    _slice_check(s, descs[-1].seed, 9, W[-1], BT[-1], WH[-1], SC[-1], G[-1], GBT[-1], s.rows - 8, 8)
+
+
+@pytest.mark.parametrize("shape", syn.STRESS_SHAPES)
+def test_config4_stress_sweep(shape):
+    rows, cols = shape
+    rng = np.random.default_rng(rows)
+    case = 0
+    for sigma in syn.STRESS_SIGMAS:
+        base = syn.TensorSpec("stress", rows, cols, 1, 0)
+        w = syn.add_outliers(syn.weights(base, case, sigma=sigma, device=DEV), case, sigma)
+        g = syn.upstream_grad(base, case, device=DEV)
+        w_hat = torch.empty_like(w)
+        for gc in syn.STRESS_GROUPS:
+            spec = syn.stress_case(rows, cols, gc)
+            for bits in syn.STRESS_BITS:
+                case += 1
+                d = Desc.make(rows, cols, 1, gc, seed=syn.layer_seed(4, case), step=case)
+                bt = syn.bitwidths(spec, 0, fixed=bits, device=DEV)
+                _, sc = gws.sample_fwd(d, w, bt, w_hat=w_hat)
+                _, gbt = gws.sample_bwd(d, g, sc)
+                torch.cuda.synchronize()
+                nrows = 8 if rows * cols > (1 << 25) else 32
+                for r0 in (0, rows - nrows, int(rng.integers(0, rows - nrows))):
+                    _slice_check(spec, d.seed, case, w, bt, w_hat, sc, g, gbt, r0, nrows)
+                # the outliers are there and the absmax sees them
+                am = gws.group_absmax(d, w)
+                assert float(am.max()) >= 7.9 * sigma
