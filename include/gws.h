@@ -16,7 +16,8 @@
  *   - All data pointers are DEVICE pointers unless a parameter says "host".  The caller owns
  *     every buffer; the library allocates nothing, frees nothing, never synchronises the
  *     device and only enqueues work on `stream` (a cudaStream_t passed as void*; NULL is the
- *     legacy default stream).  Inputs are never written.
+ *     legacy default stream); the one exception is gws_multi_prepare, which waits for its own
+ *     table upload.  Inputs are never written.
  *   - A tensor is row-major [rows, cols] of BF16 with `ld` elements between rows (ld >= cols).
  *   - A group is group_rows x group_cols elements; group_cols == 0 means "the whole row".
  *     Groups are numbered row-major over the ceil(rows/group_rows) x ceil(cols/group_cols)
@@ -64,7 +65,8 @@ typedef enum gws_status {
   GWS_ERR_ALIAS = -5,     /* output overlaps an input it must not overlap                      */
   GWS_ERR_WORKSPACE = -6, /* workspace NULL, misaligned (256 B) or too small                   */
   GWS_ERR_CUDA = -7,      /* a CUDA runtime call failed; see gws_last_cuda_error()             */
-  GWS_ERR_LIMIT = -8      /* size beyond a documented maximum                                  */
+  GWS_ERR_LIMIT = -8,     /* size beyond a documented maximum                                  */
+  GWS_ERR_UNSUPPORTED = -9 /* the call needs a different build of the library                  */
 } gws_status;
 
 /* One tensor and its noise stream. */
@@ -166,6 +168,23 @@ size_t gws_workspace_bytes(int n_tensors);
 int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace,
                       size_t workspace_bytes, gws_multi_plan* plan_out, void* stream);
 
+/* The bytes gws_multi_prepare would upload, written to HOST memory instead (nothing touches the
+ * GPU): lets a caller or a test inspect the tables.  Returns the image size in bytes (pass
+ * host_image = NULL to query it) or a negative gws_status.  The image holds, at the byte offsets
+ * recorded in the plan, arrays of 112-byte records: in, out, gin, gout (pointers), rows, cols, ld
+ * (int64), group_rows, group_cols (int32), elem_offset, n_vec (uint64), seed_lo, seed_hi,
+ * vectors_per_row, log2(lanes per group) (uint32), first tile of the tensor in its launch (int64). */
+int64_t gws_multi_table_image(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace,
+                              size_t workspace_bytes, gws_multi_plan* plan_out, void* host_image,
+                              size_t host_image_bytes);
+
+/* Diagnostic: resolves n_tiles thread-block indices of one launch (kernel_class 0..2, forward or
+ * backward table) to their tensors on the device.  tiles: device, int64 [n_tiles], each inside
+ * [0, plan->tiles[kernel_class]).  out: device, u64 [6*n_tiles] = {in, out, gin, gout pointers,
+ * tile index inside the tensor, rows of the tensor} per tile.  Reads the tables only. */
+int gws_multi_locate_probe(const gws_multi_plan* plan, int backward, int kernel_class, const int64_t* tiles,
+                           int n_tiles, uint64_t* out, void* stream);
+
 /* Forward / backward of every tensor of the plan for gradient-update counter `step`. */
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
 int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
@@ -201,6 +220,16 @@ int64_t gws_noise_alu_probe_words(const gws_desc* desc);
  * r8 receives R for the 8 fields of the 4 words; packed receives the nibble word. */
 void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed);
 void gws_host_philox(uint64_t seed, uint64_t step, uint64_t vec, uint32_t* out4);
+
+/* Self-checking build (compiled with -DGWS_SELF_CHECK; gws_selfcheck_enabled() returns 1): every
+ * kernel access to caller memory is tested against the window [base, base+bytes) declared here; an
+ * access outside it is counted, the first one recorded, and skipped instead of performed.  Both calls
+ * synchronise the device.  report: out5 (host) = {violations, kind of the first (1 vector load,
+ * 2 vector store, 3 float load, 4 float store, 5 element load, 6 element store), its address, block,
+ * thread}.  In the normal build both return GWS_ERR_UNSUPPORTED. */
+int gws_selfcheck_enabled(void);
+int gws_selfcheck_set_window(const void* base, size_t bytes);
+int gws_selfcheck_report(uint64_t* out5);
 
 /* Which kernel class a descriptor with fully aligned pointers would use:
  * 0 flat groups, 1 warp per row, 2 thread block per row, 3 general; negative gws_status on error. */

@@ -24,21 +24,27 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+CHECK_LIB_PATH = os.path.join(_PKG, "libgws_check.so")   # the self-checking variant (-DGWS_SELF_CHECK)
+
+
+def is_stale(path: str = LIB_PATH) -> bool:
+    if not os.path.exists(path):
         return True
-    built = os.path.getmtime(LIB_PATH)
+    built = os.path.getmtime(path)
     return any(os.path.getmtime(p) > built for p in SOURCES + HEADERS)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile ``libgws.so`` next to the package if it is missing or older than its sources."""
-    if force or is_stale():
-        tmp = LIB_PATH + ".tmp.%d" % os.getpid()
-        cmd = [_nvcc(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp, *SOURCES]
+def build(force: bool = False, verbose: bool = False, self_check: bool = False) -> str:
+    """Compile ``libgws.so`` (or the self-checking ``libgws_check.so``) next to the package if it is missing
+    or older than its sources."""
+    path = CHECK_LIB_PATH if self_check else LIB_PATH
+    if force or is_stale(path):
+        tmp = path + ".tmp.%d" % os.getpid()
+        cmd = [_nvcc(), *NVCC_FLAGS, *(["-DGWS_SELF_CHECK"] if self_check else []),
+               *(["-Xptxas", "-v"] if verbose else []), "-o", tmp, *SOURCES]
         subprocess.run(cmd, check=True)
-        os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+        os.replace(tmp, path)
+    return path
 
 
 if __name__ == "__main__":

@@ -25,7 +25,7 @@ class GwsError(RuntimeError):
         super().__init__(msg)
 
 
-OK, ERR_NULL, ERR_SHAPE, ERR_GROUP, ERR_ALIGN, ERR_ALIAS, ERR_WORKSPACE, ERR_CUDA, ERR_LIMIT = 0, -1, -2, -3, -4, -5, -6, -7, -8
+OK, ERR_NULL, ERR_SHAPE, ERR_GROUP, ERR_ALIGN, ERR_ALIAS, ERR_WORKSPACE, ERR_CUDA, ERR_LIMIT, ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6, -7, -8, -9
 
 
 class Desc(Structure):
@@ -66,6 +66,8 @@ _SIGNATURES = {
     "gws_sample_bwd": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gws_workspace_bytes": (c_size_t, [c_int]),
     "gws_multi_prepare": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, POINTER(_MultiPlan), c_void_p]),
+    "gws_multi_table_image": (c_int64, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, POINTER(_MultiPlan), c_void_p, c_size_t]),
+    "gws_multi_locate_probe": (c_int, [POINTER(_MultiPlan), c_int, c_int, c_void_p, c_int, c_void_p, c_void_p]),
     "gws_sample_fwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_sample_bwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_sample_step_host": (c_int, [POINTER(Desc)] + [c_void_p] * 13),
@@ -74,6 +76,9 @@ _SIGNATURES = {
     "gws_noise_alu_probe_words": (c_int64, [POINTER(Desc)]),
     "gws_host_decode8": (None, [POINTER(c_uint32), POINTER(c_int8), POINTER(c_uint32)]),
     "gws_host_philox": (None, [c_uint64, c_uint64, c_uint64, POINTER(c_uint32)]),
+    "gws_selfcheck_enabled": (c_int, []),
+    "gws_selfcheck_set_window": (c_int, [c_void_p, c_size_t]),
+    "gws_selfcheck_report": (c_int, [POINTER(c_uint64)]),
     "gws_status_string": (c_char_p, [c_int]),
     "gws_last_cuda_error": (c_char_p, []),
     "gws_launch_count": (c_uint64, []),
@@ -238,6 +243,15 @@ class MultiPlan:
         c = list(self.plan.count)
         return sum(1 for k in range(3) if c[k]) + c[3]
 
+    def locate_probe(self, backward: bool, kernel_class: int, tiles: torch.Tensor, stream=None) -> torch.Tensor:
+        """Diagnostic: (n_tiles, 6) int64 rows {in, out, gin, gout, tile inside tensor, rows} resolved on the device."""
+        _require_cuda(tiles)
+        assert tiles.dtype == torch.int64 and tiles.is_contiguous()
+        out = torch.zeros((tiles.numel(), 6), dtype=torch.int64, device=tiles.device)
+        _check(load_library().gws_multi_locate_probe(ctypes.byref(self.plan), int(backward), kernel_class, _ptr(tiles),
+                                                     tiles.numel(), _ptr(out), _stream(stream)))
+        return out
+
     def sample_fwd_multi(self, step: int, stream=None) -> None:
         _check(load_library().gws_sample_fwd_multi(ctypes.byref(self.plan), step, _stream(stream)))
 
@@ -255,6 +269,22 @@ def sample_step_host(desc: Desc, h_w, h_bt, h_grad, h_w_hat, h_scale, h_grad_bt,
     _check(load_library().gws_sample_step_host(ctypes.byref(desc), _ptr(h_w), _ptr(h_bt), _ptr(h_grad), _ptr(h_w_hat),
                                                _ptr(h_scale), _ptr(h_grad_bt), _ptr(d_w), _ptr(d_w_hat), _ptr(d_grad),
                                                _ptr(d_bt), _ptr(d_scale), _ptr(d_grad_bt), _stream(stream)))
+
+
+def selfcheck_enabled() -> bool:
+    return bool(load_library().gws_selfcheck_enabled())
+
+
+def selfcheck_set_window(buffer: torch.Tensor) -> None:
+    """Self-checking build only: declare ``buffer`` as the only memory the kernels may touch."""
+    _check(load_library().gws_selfcheck_set_window(_ptr(buffer), buffer.numel() * buffer.element_size()))
+
+
+def selfcheck_report():
+    """Self-checking build only: (violations, kind, address, block, thread) since the window was set."""
+    out = (c_uint64 * 5)()
+    _check(load_library().gws_selfcheck_report(out))
+    return tuple(int(x) for x in out)
 
 
 # ---- host-side diagnostics (no GPU needed) ------------------------------------------------------------

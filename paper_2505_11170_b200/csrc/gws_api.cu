@@ -119,6 +119,27 @@ Entry make_entry(const gws_desc* d, int cls, const void* in, void* out, const fl
   return e;
 }
 
+template <int MODE, bool MULTI>
+int launch_as(int cls, const Entry& single, const Entry* table, int n_or_index, unsigned grid, uint32_t lo, uint32_t hi,
+              cudaStream_t stream) {
+  switch (cls) {
+    case gws::kFlat:
+      gws::k_flat<MODE, MULTI><<<grid, gws::kFlatThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      return check_launch("flat-group kernel");
+    case gws::kRowWarp:
+      gws::k_row_warp<MODE, MULTI><<<grid, gws::kRowWarpThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      return check_launch("warp-per-row kernel");
+    case gws::kRowCta:
+      gws::k_row_cta<MODE, MULTI><<<grid, gws::kRowCtaThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      return check_launch("block-per-row kernel");
+    default:
+      gws::k_general<MODE, MULTI><<<grid, gws::kGeneralThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      return check_launch("general kernel");
+  }
+}
+
+// table == nullptr: one tensor, described by `single`; otherwise entry n_or_index (general class) or the
+// n_or_index entries (other classes) of `table`.
 template <int MODE>
 int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int64_t tiles, uint64_t step,
            cudaStream_t stream) {
@@ -126,20 +147,8 @@ int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int
   if (tiles > kMaxGrid) return GWS_ERR_LIMIT;
   const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
   const unsigned grid = static_cast<unsigned>(tiles);
-  switch (cls) {
-    case gws::kFlat:
-      gws::k_flat<MODE><<<grid, gws::kFlatThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
-      return check_launch("flat-group kernel");
-    case gws::kRowWarp:
-      gws::k_row_warp<MODE><<<grid, gws::kRowWarpThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
-      return check_launch("warp-per-row kernel");
-    case gws::kRowCta:
-      gws::k_row_cta<MODE><<<grid, gws::kRowCtaThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
-      return check_launch("block-per-row kernel");
-    default:
-      gws::k_general<MODE><<<grid, gws::kGeneralThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
-      return check_launch("general kernel");
-  }
+  return table == nullptr ? launch_as<MODE, false>(cls, single, table, n_or_index, grid, lo, hi, stream)
+                          : launch_as<MODE, true>(cls, single, table, n_or_index, grid, lo, hi, stream);
 }
 
 // Shared checks of the single-tensor calls.  Returns 1 if there is nothing to do.
@@ -260,8 +269,10 @@ size_t gws_workspace_bytes(int n_tensors) {
   return static_cast<size_t>(n_tensors) * 2u * sizeof(Entry) + 8u * 256u;
 }
 
-int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace, size_t workspace_bytes,
-                      gws_multi_plan* plan_out, void* stream) {
+// Builds the table image (all class tables, forward then backward, each 256-byte aligned) in host
+// memory and fills the plan.  `workspace` is only recorded, never dereferenced.
+static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace, size_t workspace_bytes,
+                        gws_multi_plan* plan_out, std::vector<char>& image) {
   if (n < 0) return GWS_ERR_SHAPE;
   if (descs == nullptr || ptrs == nullptr || plan_out == nullptr) return GWS_ERR_NULL;
   const bool has_fwd = ptrs->w != nullptr;
@@ -322,39 +333,64 @@ int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, 
   plan.has_fwd = has_fwd ? 1 : 0;
   plan.has_bwd = has_bwd ? 1 : 0;
   plan.total_elements = total;
-  size_t offset = 0;
-  auto place = [&](std::vector<Entry>& v, int cls, int64_t* where, bool general) -> int {
+  image.clear();
+  auto place = [&](std::vector<Entry>& v, int cls, int64_t* where) -> int {
     int64_t running = 0;
     for (Entry& e : v) {
       const int64_t tiles = e.tile_begin;
       e.tile_begin = running;
       running += tiles;
     }
-    if (!general && running > kMaxGrid) return GWS_ERR_LIMIT;
+    if (cls != gws::kGeneral && running > kMaxGrid) return GWS_ERR_LIMIT;
     plan.count[cls] = static_cast<int32_t>(v.size());
     plan.tiles[cls] = running;
-    *where = static_cast<int64_t>(offset);
-    if (!v.empty()) {
-      const size_t bytes = v.size() * sizeof(Entry);
-      const cudaError_t err = cudaMemcpyAsync(static_cast<char*>(workspace) + offset, v.data(), bytes,
-                                              cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream));
-      if (err != cudaSuccess) return cuda_fail(err, "table upload");
-      offset += (bytes + 255u) & ~static_cast<size_t>(255u);
-    }
+    *where = static_cast<int64_t>(image.size());
+    const size_t bytes = v.size() * sizeof(Entry);
+    const size_t padded = (bytes + 255u) & ~static_cast<size_t>(255u);
+    image.resize(image.size() + padded, 0);
+    if (bytes) std::memcpy(image.data() + *where, v.data(), bytes);
     return GWS_OK;
   };
   for (int cls = 0; cls < 4; ++cls) {
     int st = GWS_OK;
-    if (has_fwd) st = place(t.fwd[cls], cls, &plan.fwd_offset[cls], cls == gws::kGeneral);
+    if (has_fwd) st = place(t.fwd[cls], cls, &plan.fwd_offset[cls]);
     if (st != GWS_OK) return st;
-    if (has_bwd) st = place(t.bwd[cls], cls, &plan.bwd_offset[cls], cls == gws::kGeneral);
+    if (has_bwd) st = place(t.bwd[cls], cls, &plan.bwd_offset[cls]);
     if (st != GWS_OK) return st;
   }
-  // The uploads read pageable host memory that dies with this call: wait for them.
-  const cudaError_t err = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
-  if (err != cudaSuccess) return cuda_fail(err, "table upload");
+  if (image.size() > workspace_bytes) return GWS_ERR_WORKSPACE;
   *plan_out = plan;
   return GWS_OK;
+}
+
+int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace, size_t workspace_bytes,
+                      gws_multi_plan* plan_out, void* stream) {
+  std::vector<char> image;
+  gws_multi_plan plan;
+  const int st = build_tables(n, descs, ptrs, workspace, workspace_bytes, &plan, image);
+  if (st != GWS_OK) return st;
+  if (!image.empty()) {
+    cudaError_t err = cudaMemcpyAsync(workspace, image.data(), image.size(), cudaMemcpyHostToDevice,
+                                      static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return cuda_fail(err, "table upload");
+    // The upload reads pageable host memory that dies with this call: wait for it.
+    err = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return cuda_fail(err, "table upload");
+  }
+  *plan_out = plan;
+  return GWS_OK;
+}
+
+int64_t gws_multi_table_image(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace,
+                              size_t workspace_bytes, gws_multi_plan* plan_out, void* host_image, size_t host_image_bytes) {
+  std::vector<char> image;
+  const int st = build_tables(n, descs, ptrs, workspace, workspace_bytes, plan_out, image);
+  if (st != GWS_OK) return st;
+  if (host_image != nullptr) {
+    if (host_image_bytes < image.size()) return GWS_ERR_WORKSPACE;
+    std::memcpy(host_image, image.data(), image.size());
+  }
+  return static_cast<int64_t>(image.size());
 }
 
 static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream, bool backward) {
@@ -389,6 +425,58 @@ int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream
 
 int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
   return run_multi(plan, step, stream, true);
+}
+
+int gws_multi_locate_probe(const gws_multi_plan* plan, int backward, int kernel_class, const int64_t* tiles, int n_tiles,
+                           uint64_t* out, void* stream) {
+  if (plan == nullptr || tiles == nullptr || out == nullptr) return GWS_ERR_NULL;
+  if (kernel_class < 0 || kernel_class > 2 || n_tiles < 0) return GWS_ERR_SHAPE;
+  if (plan->workspace == nullptr) return GWS_ERR_WORKSPACE;
+  if (n_tiles == 0 || plan->count[kernel_class] == 0) return GWS_OK;
+  const Entry* table = reinterpret_cast<const Entry*>(
+      static_cast<const char*>(plan->workspace) + (backward ? plan->bwd_offset[kernel_class] : plan->fwd_offset[kernel_class]));
+  gws::k_locate_probe<<<(n_tiles + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+      table, plan->count[kernel_class], tiles, n_tiles, out);
+  return check_launch("locate probe");
+}
+
+// ---- self-checking build ----------------------------------------------------------------------------
+
+int gws_selfcheck_enabled(void) {
+#ifdef GWS_SELF_CHECK
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+int gws_selfcheck_set_window(const void* base, size_t bytes) {
+#ifdef GWS_SELF_CHECK
+  gws::CheckState st;
+  std::memset(&st, 0, sizeof st);
+  st.lo = reinterpret_cast<unsigned long long>(base);
+  st.hi = st.lo + bytes;
+  const cudaError_t err = cudaMemcpyToSymbol(gws::g_check, &st, sizeof st);
+  return err == cudaSuccess ? GWS_OK : cuda_fail(err, "self-check window");
+#else
+  (void)base; (void)bytes;
+  return GWS_ERR_UNSUPPORTED;
+#endif
+}
+
+int gws_selfcheck_report(uint64_t* out5) {
+#ifdef GWS_SELF_CHECK
+  if (out5 == nullptr) return GWS_ERR_NULL;
+  gws::CheckState st;
+  const cudaError_t err = cudaMemcpyFromSymbol(&st, gws::g_check, sizeof st);
+  if (err != cudaSuccess) return cuda_fail(err, "self-check report");
+  out5[0] = st.violations;
+  for (int k = 0; k < 4; ++k) out5[1 + k] = st.first[k];
+  return GWS_OK;
+#else
+  (void)out5;
+  return GWS_ERR_UNSUPPORTED;
+#endif
 }
 
 // ---- host-buffer step ---------------------------------------------------------------------------
@@ -450,6 +538,7 @@ const char* gws_status_string(int status) {
     case GWS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case GWS_ERR_CUDA: return "CUDA runtime error (see gws_last_cuda_error)";
     case GWS_ERR_LIMIT: return "size beyond a documented maximum";
+    case GWS_ERR_UNSUPPORTED: return "not available in this build of the library";
     default: return "unknown status";
   }
 }

@@ -52,13 +52,62 @@ constexpr int kRowCtaThreads = 512, kRowCtaVecs = 16;   // 1 row per tile, <= 81
 constexpr int kGeneralThreads = 128;
 constexpr float kLn2 = 0.693147180559945309f;
 
-// ---- small device helpers ------------------------------------------------------------------
+// ---- global memory accessors ---------------------------------------------------------------------
+// Every access to caller memory goes through these.  In the self-checking build
+// (-DGWS_SELF_CHECK) each address is first tested against a caller-declared window; an address
+// outside it is recorded (first violation wins: kind, address, block, thread) and the access is
+// skipped, so a wrong pointer or index shows up as a report instead of a fault.
+
+#ifdef GWS_SELF_CHECK
+struct CheckState {
+  unsigned long long lo, hi;        // allowed window [lo, hi)
+  unsigned long long violations;    // count
+  unsigned long long first[4];      // kind, address, blockIdx.x, threadIdx.x of the first one
+};
+__device__ CheckState g_check;
+
+__device__ __noinline__ bool check_access(const void* p, unsigned bytes, unsigned kind) {
+  const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+  if (a >= g_check.lo && a + bytes <= g_check.hi) return true;
+  if (atomicAdd(&g_check.violations, 1ull) == 0ull) {
+    g_check.first[0] = kind;
+    g_check.first[1] = a;
+    g_check.first[2] = blockIdx.x;
+    g_check.first[3] = threadIdx.x;
+  }
+  return false;
+}
+#define GWS_CHECK(p, bytes, kind, fallback) \
+  if (!check_access((p), (bytes), (kind))) return fallback
+#else
+#define GWS_CHECK(p, bytes, kind, fallback)
+#endif
 
 __device__ __forceinline__ uint4 ld_vec(const void* base, uint64_t v) {
-  return __ldg(reinterpret_cast<const uint4*>(base) + v);
+  const uint4* p = reinterpret_cast<const uint4*>(base) + v;
+  GWS_CHECK(p, 16, 1, make_uint4(0, 0, 0, 0));
+  return __ldg(p);
 }
 __device__ __forceinline__ void st_vec(void* base, uint64_t v, const uint4& x) {
-  *(reinterpret_cast<uint4*>(base) + v) = x;
+  uint4* p = reinterpret_cast<uint4*>(base) + v;
+  GWS_CHECK(p, 16, 2, );
+  *p = x;
+}
+__device__ __forceinline__ float ld_f32(const float* base, uint64_t i) {
+  GWS_CHECK(base + i, 4, 3, 0.0f);
+  return __ldg(base + i);
+}
+__device__ __forceinline__ void st_f32(float* base, uint64_t i, float x) {
+  GWS_CHECK(base + i, 4, 4, );
+  base[i] = x;
+}
+__device__ __forceinline__ uint16_t ld_u16(const uint16_t* base, int64_t i) {
+  GWS_CHECK(base + i, 2, 5, 0);
+  return base[i];
+}
+__device__ __forceinline__ void st_u16(uint16_t* base, int64_t i, uint16_t x) {
+  GWS_CHECK(base + i, 2, 6, );
+  base[i] = x;
 }
 
 __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
@@ -138,33 +187,53 @@ __device__ __forceinline__ Words4 philox_vec(const Entry& e, uint64_t vec_in_ten
   return philox_for_vector((e.elem_offset >> 3) + vec_in_tensor, step_lo, step_hi, e.seed_lo, e.seed_hi);
 }
 
-// Finds the tensor that owns tile `tile` of a launch (tile_begin is increasing).
-__device__ __forceinline__ void locate(const Entry& single, const Entry* __restrict__ table, int n, int64_t tile,
-                                       Entry& e, int64_t& local_tile) {
-  if (table == nullptr) {
-    e = single;
-    local_tile = tile;
-    return;
-  }
+// Finds the tensor that owns tile `tile` of a multi-tensor launch (tile_begin is increasing).
+__device__ __forceinline__ int locate(const Entry* __restrict__ table, int n, int64_t tile) {
   int lo = 0, hi = n - 1;
   while (lo < hi) {
     const int mid = (lo + hi + 1) >> 1;
-    if (__ldg(&table[mid].tile_begin) <= tile) lo = mid; else hi = mid - 1;
+    if (table[mid].tile_begin <= tile) lo = mid; else hi = mid - 1;
   }
-  e = table[lo];
-  local_tile = tile - e.tile_begin;
+  return lo;
+}
+
+// The tensor of this thread block.  MULTI is a compile-time switch: a single-tensor launch reads its
+// entry from the kernel parameters, a multi-tensor launch from the table in global memory.  (A run-time
+// choice between the two sources inside one kernel produced entries mixed from both on sm_100a.)
+#define GWS_RESOLVE_ENTRY(e, tile)                                   \
+  Entry e;                                                           \
+  int64_t tile = static_cast<int64_t>(blockIdx.x);                   \
+  if (MULTI) {                                                       \
+    e = table[locate(table, n, tile)];                               \
+    tile -= e.tile_begin;                                            \
+  } else {                                                           \
+    e = single;                                                      \
+  }
+
+// Diagnostic: what locate() resolves for a list of tile indices.  Reads the table only.
+// out[6*k ..] = {in, out, gin, gout, local tile, tensor rows} for tiles[k].
+__global__ void k_locate_probe(const Entry* __restrict__ table, int n, const int64_t* __restrict__ tiles, int n_tiles,
+                               uint64_t* __restrict__ out) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= n_tiles) return;
+  const Entry e = table[locate(table, n, tiles[k])];
+  const int64_t local = tiles[k] - e.tile_begin;
+  out[6 * k + 0] = reinterpret_cast<uint64_t>(e.in);
+  out[6 * k + 1] = reinterpret_cast<uint64_t>(e.out);
+  out[6 * k + 2] = reinterpret_cast<uint64_t>(e.gin);
+  out[6 * k + 3] = reinterpret_cast<uint64_t>(e.gout);
+  out[6 * k + 4] = static_cast<uint64_t>(local);
+  out[6 * k + 5] = static_cast<uint64_t>(e.rows);
 }
 
 // ---- flat groups ------------------------------------------------------------------------------
 
-template <int MODE>
+template <int MODE, bool MULTI>
 __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ Entry single,
                                                        const Entry* __restrict__ table, int n, uint32_t step_lo,
                                                        uint32_t step_hi) {
   constexpr int T = kFlatThreads, V = kFlatVecs;
-  Entry e;
-  int64_t tile;
-  locate(single, table, n, static_cast<int64_t>(blockIdx.x), e, tile);
+  GWS_RESOLVE_ENTRY(e, tile)
   const uint32_t ll = e.lanes_log2;
   const uint32_t L = 1u << ll;
   const uint32_t lane_in_group = threadIdx.x & (L - 1u);
@@ -179,7 +248,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ E
     ok[k] = v < e.n_vec;
     x[k] = ok[k] ? ld_vec(e.in, v) : make_uint4(0, 0, 0, 0);
     gv[k] = 0.0f;
-    if (MODE != kAbsmax && ok[k]) gv[k] = __ldg(e.gin + (v >> ll));
+    if (MODE != kAbsmax && ok[k]) gv[k] = ld_f32(e.gin, v >> ll);
   }
 #pragma unroll
   for (int k = 0; k < V; ++k) {
@@ -189,7 +258,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ E
       float acc = dot_vec(x[k], philox_vec(e, v, step_lo, step_hi));
       for (uint32_t o = 1; o < L; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
       if (ok[k]) {
-        if (lane_in_group == 0) e.gout[g] = __fmul_rn(__fmul_rn(-kLn2, gv[k]), acc);
+        if (lane_in_group == 0) st_f32(e.gout, g, __fmul_rn(__fmul_rn(-kLn2, gv[k]), acc));
         if (e.out != nullptr) st_vec(e.out, v, x[k]);
       }
     } else {
@@ -197,13 +266,13 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ E
       for (uint32_t o = 1; o < L; o <<= 1) m = bmax2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
       const float a = absmax_finish(m);
       if (MODE == kAbsmax) {
-        if (ok[k] && lane_in_group == 0) e.gout[g] = a;
+        if (ok[k] && lane_in_group == 0) st_f32(e.gout, g, a);
       } else {
         const float s = __fmul_rn(a, pow2_one_minus(gv[k]));
         const uint4 y = sample_vec(x[k], philox_vec(e, v, step_lo, step_hi), s);
         if (ok[k]) {
           st_vec(e.out, v, y);
-          if (e.gout != nullptr && lane_in_group == 0) e.gout[g] = s;
+          if (e.gout != nullptr && lane_in_group == 0) st_f32(e.gout, g, s);
         }
       }
     }
@@ -212,14 +281,12 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ E
 
 // ---- one warp per row ---------------------------------------------------------------------------
 
-template <int MODE>
+template <int MODE, bool MULTI>
 __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_constant__ Entry single,
                                                               const Entry* __restrict__ table, int n,
                                                               uint32_t step_lo, uint32_t step_hi) {
   constexpr int V = kRowWarpVecs, ROWS = kRowWarpThreads / 32;
-  Entry e;
-  int64_t tile;
-  locate(single, table, n, static_cast<int64_t>(blockIdx.x), e, tile);
+  GWS_RESOLVE_ENTRY(e, tile)
   const uint32_t lane = threadIdx.x & 31u;
   const int64_t row = tile * ROWS + (threadIdx.x >> 5);
   const bool okr = row < e.rows;
@@ -235,7 +302,7 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
       if (okr && j < vpr) x[k] = ld_vec(e.in, vbase + j);
     }
   }
-  const float gvr = (MODE != kAbsmax && okr) ? __ldg(e.gin + row) : 0.0f;
+  const float gvr = (MODE != kAbsmax && okr) ? ld_f32(e.gin, row) : 0.0f;
 
   if (MODE == kBwd) {
     float acc = 0.0f;
@@ -253,7 +320,7 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
     }
 #pragma unroll
     for (uint32_t o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-    if (okr && lane == 0) e.gout[row] = __fmul_rn(__fmul_rn(-kLn2, gvr), acc);
+    if (okr && lane == 0) st_f32(e.gout, row, __fmul_rn(__fmul_rn(-kLn2, gvr), acc));
   } else {
     uint32_t m = 0;
 #pragma unroll
@@ -263,7 +330,7 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
     for (uint32_t o = 16; o > 0; o >>= 1) m = bmax2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     const float a = absmax_finish(m);
     if (MODE == kAbsmax) {
-      if (okr && lane == 0) e.gout[row] = a;
+      if (okr && lane == 0) st_f32(e.gout, row, a);
     } else {
       const float s = __fmul_rn(a, pow2_one_minus(gvr));
 #pragma unroll
@@ -274,23 +341,21 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
           if (okr && j < vpr) st_vec(e.out, vbase + j, y);
         }
       }
-      if (okr && lane == 0 && e.gout != nullptr) e.gout[row] = s;
+      if (okr && lane == 0 && e.gout != nullptr) st_f32(e.gout, row, s);
     }
   }
 }
 
 // ---- one thread block per row ---------------------------------------------------------------------
 
-template <int MODE>
+template <int MODE, bool MULTI>
 __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constant__ Entry single,
                                                             const Entry* __restrict__ table, int n,
                                                             uint32_t step_lo, uint32_t step_hi) {
   constexpr int T = kRowCtaThreads, V = kRowCtaVecs, WARPS = T / 32;
   __shared__ uint32_t red_u[WARPS];
   __shared__ float red_f[WARPS];
-  Entry e;
-  int64_t tile;
-  locate(single, table, n, static_cast<int64_t>(blockIdx.x), e, tile);
+  GWS_RESOLVE_ENTRY(e, tile)
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const int64_t row = tile;
   const uint32_t vpr = e.vpr;
@@ -305,7 +370,7 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
       if (j < vpr) x[k] = ld_vec(e.in, vbase + j);
     }
   }
-  const float gvr = (MODE != kAbsmax) ? __ldg(e.gin + row) : 0.0f;
+  const float gvr = (MODE != kAbsmax) ? ld_f32(e.gin, row) : 0.0f;
 
   if (MODE == kBwd) {
     float acc = 0.0f;
@@ -327,7 +392,7 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
     if (threadIdx.x == 0) {
       float total = 0.0f;
       for (int w = 0; w < WARPS; ++w) total += red_f[w];  // fixed order
-      e.gout[row] = __fmul_rn(__fmul_rn(-kLn2, gvr), total);
+      st_f32(e.gout, row, __fmul_rn(__fmul_rn(-kLn2, gvr), total));
     }
   } else {
     uint32_t m = 0;
@@ -343,7 +408,7 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
     for (int w = 1; w < WARPS; ++w) mm = bmax2(mm, red_u[w]);
     const float a = absmax_finish(mm);
     if (MODE == kAbsmax) {
-      if (threadIdx.x == 0) e.gout[row] = a;
+      if (threadIdx.x == 0) st_f32(e.gout, row, a);
     } else {
       const float s = __fmul_rn(a, pow2_one_minus(gvr));
 #pragma unroll
@@ -354,21 +419,22 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
           if (j < vpr) st_vec(e.out, vbase + j, y);
         }
       }
-      if (threadIdx.x == 0 && e.gout != nullptr) e.gout[row] = s;
+      if (threadIdx.x == 0 && e.gout != nullptr) st_f32(e.gout, row, s);
     }
   }
 }
 
 // ---- general shapes: one thread block per group, scalar accesses ---------------------------------
 
-template <int MODE>
+template <int MODE, bool MULTI>
 __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_constant__ Entry single,
                                                              const Entry* __restrict__ table, int index,
                                                              uint32_t step_lo, uint32_t step_hi) {
   constexpr int T = kGeneralThreads, WARPS = T / 32;
   __shared__ float red[WARPS];
   __shared__ float bcast;
-  const Entry e = (table == nullptr) ? single : table[index];
+  Entry e;
+  if (MULTI) e = table[index]; else e = single;
   const uint16_t* in = reinterpret_cast<const uint16_t*>(e.in);
   uint16_t* out = reinterpret_cast<uint16_t*>(e.out);
   const int64_t gr = e.group_rows, gc = e.group_cols;
@@ -385,7 +451,7 @@ __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_consta
       float m = 0.0f;
       for (int64_t k = threadIdx.x; k < count; k += T) {
         const int64_t i = r0 + k / wd, j = c0 + k % wd;
-        m = fmaxf(m, fabsf(__uint_as_float(static_cast<uint32_t>(in[i * e.ld + j]) << 16)));
+        m = fmaxf(m, fabsf(__uint_as_float(static_cast<uint32_t>(ld_u16(in, i * e.ld + j)) << 16)));
       }
 #pragma unroll
       for (uint32_t o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
@@ -395,10 +461,10 @@ __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_consta
         float a = red[0];
         for (int w = 1; w < WARPS; ++w) a = fmaxf(a, red[w]);
         if (MODE == kAbsmax) {
-          e.gout[g] = a;
+          st_f32(e.gout, g, a);
         } else {
-          const float s = __fmul_rn(a, pow2_one_minus(e.gin[g]));
-          if (e.gout != nullptr) e.gout[g] = s;
+          const float s = __fmul_rn(a, pow2_one_minus(ld_f32(e.gin, g)));
+          if (e.gout != nullptr) st_f32(e.gout, g, s);
           bcast = s;
         }
       }
@@ -412,15 +478,15 @@ __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_consta
         const uint64_t el = e.elem_offset + static_cast<uint64_t>(i * e.cols + j);
         const Words4 words = philox_for_vector(el >> 3, step_lo, step_hi, e.seed_lo, e.seed_hi);
         const int r = decode_field(field_of(words, static_cast<unsigned>(el & 7u)));
-        const uint16_t bits = in[i * e.ld + j];
+        const uint16_t bits = ld_u16(in, i * e.ld + j);
         const float val = __uint_as_float(static_cast<uint32_t>(bits) << 16);
         if (MODE == kFwd) {
           const float q = __fmul_rn(static_cast<float>(r), scale);
           const float y = __fadd_rn(val, q);
-          out[i * e.ld + j] = static_cast<uint16_t>(pack_bf16_rne(y, 0.0f) & 0xFFFFu);
+          st_u16(out, i * e.ld + j, static_cast<uint16_t>(pack_bf16_rne(y, 0.0f) & 0xFFFFu));
         } else {
           acc = __fmaf_rn(val, static_cast<float>(r), acc);
-          if (out != nullptr) out[i * e.ld + j] = bits;
+          if (out != nullptr) st_u16(out, i * e.ld + j, bits);
         }
       }
       if (MODE == kBwd) {
@@ -431,7 +497,7 @@ __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_consta
         if (threadIdx.x == 0) {
           float total = 0.0f;
           for (int w = 0; w < WARPS; ++w) total += red[w];
-          e.gout[g] = __fmul_rn(__fmul_rn(-kLn2, e.gin[g]), total);
+          st_f32(e.gout, g, __fmul_rn(__fmul_rn(-kLn2, ld_f32(e.gin, g)), total));
         }
       }
     }
