@@ -189,6 +189,38 @@ int gws_multi_locate_probe(const gws_multi_plan* plan, int backward, int kernel_
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
 int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
 
+/* ---- forward over many tensors for callers that cannot allocate device memory --------------------
+ * (No counterpart in the paper: this entry point exists for the way the library gets embedded.)
+ *
+ * Some callers have nowhere to get the table workspace from: code that runs inside a framework's
+ * allocator hooks or out-of-memory handlers, plug-ins that are handed tensors but no allocator, and
+ * processes that have given all device memory to a pool at start-up and must not call cudaMalloc
+ * afterwards (it would fail, or synchronise the device in the middle of a step).  For them the tensor
+ * table lives in an array compiled into the library: sizeof = GWS_STATIC_MAX_TENSORS * 224 + 2048
+ * bytes (about 59 KB) of device memory on every GPU that loads the library, held until the process
+ * exits.  The call does what gws_multi_prepare followed by gws_sample_fwd_multi does, for the
+ * forward pass only, and allocates no device memory, frees none and calls no allocating library
+ * routine.
+ *   n, descs, ptrs   as for gws_multi_prepare; only w, bt, w_hat and scale of `ptrs` are used
+ *                    (scale, and each of its entries, may be NULL).  n > GWS_STATIC_MAX_TENSORS
+ *                    returns GWS_ERR_LIMIT and enqueues nothing.
+ *   step             gradient-update counter, as for gws_sample_fwd_multi
+ * Results are bit-identical to gws_sample_fwd_multi.  Things to know:
+ *   - The first call on each device looks up the array's device address (with that device current).
+ *     Make that first call outside any stream capture.
+ *   - Every call on a device rewrites the same array before launching, in stream order.  Two calls
+ *     whose work can overlap on the GPU (different streams without an ordering between them, or
+ *     different host threads doing so) race on it: keep all calls on one stream, or order them
+ *     with events.  Nothing in the array has to be cleared between calls: each call overwrites all
+ *     of what its own kernels read.
+ *   - The table is uploaded from pageable host memory on `stream`, so the call may wait for earlier
+ *     work on that stream; gws_multi_prepare + gws_sample_fwd_multi avoid that per-step cost and
+ *     remain the better choice for callers that can allocate.
+ */
+#define GWS_STATIC_MAX_TENSORS 256
+int gws_sample_fwd_multi_static(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, uint64_t step,
+                                void* stream);
+
 /* ---- host-buffer step (end-to-end path) --------------------------------------------------------
  * One forward + backward of one tensor whose data lives in HOST memory (pinned memory makes the
  * copies asynchronous).  Copies w, bt, grad_w_hat to the device staging buffers, runs

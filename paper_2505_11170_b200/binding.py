@@ -70,6 +70,7 @@ _SIGNATURES = {
     "gws_multi_locate_probe": (c_int, [POINTER(_MultiPlan), c_int, c_int, c_void_p, c_int, c_void_p, c_void_p]),
     "gws_sample_fwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_sample_bwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
+    "gws_sample_fwd_multi_static": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_uint64, c_void_p]),
     "gws_sample_step_host": (c_int, [POINTER(Desc)] + [c_void_p] * 13),
     "gws_philox_words": (c_int, [c_uint64, c_uint64, c_uint64, c_int64, c_void_p, c_void_p]),
     "gws_noise_alu_probe": (c_int, [POINTER(Desc), c_void_p, c_void_p]),
@@ -257,6 +258,25 @@ class MultiPlan:
 
     def sample_bwd_multi(self, step: int, stream=None) -> None:
         _check(load_library().gws_sample_bwd_multi(ctypes.byref(self.plan), step, _stream(stream)))
+
+
+STATIC_MAX_TENSORS = 256   # GWS_STATIC_MAX_TENSORS of include/gws.h
+
+
+def sample_fwd_multi_static(descs: Sequence[Desc], w, bt, w_hat, scale=None, step: int = 0, stream=None) -> None:
+    """Forward pass over many tensors with the tensor table kept in the library's built-in device array.
+
+    For callers that must not allocate device memory (allocator hooks, out-of-memory handlers, processes
+    whose memory all belongs to a pool): this wrapper and the entry point behind it allocate nothing on
+    the device; the caller passes every input and output tensor.  At most ``STATIC_MAX_TENSORS`` tensors;
+    calls share one array per GPU, so keep them on one stream (overlapping calls race).
+    """
+    n = len(descs)
+    _require_cuda(*w, *bt, *w_hat, *(scale or []))
+    arrays = [_ptr_array(g, n) for g in (w, bt, w_hat, scale, None, None, None)]
+    cast = lambda a: ctypes.cast(a, POINTER(c_void_p)) if a is not None else None
+    ptrs = _MultiPtrs(*[cast(a) for a in arrays])
+    _check(load_library().gws_sample_fwd_multi_static(n, (Desc * n)(*descs), ctypes.byref(ptrs), step, _stream(stream)))
 
 
 def sample_step_host(desc: Desc, h_w, h_bt, h_grad, h_w_hat, h_scale, h_grad_bt, d_w, d_w_hat, d_grad, d_bt, d_scale,

@@ -509,6 +509,65 @@ int gws_sample_step_host(const gws_desc* desc, const void* h_w, const float* h_b
   return GWS_OK;
 }
 
+// ---- forward over many tensors without any device allocation ----------------------------------------
+//
+// The multi-tensor kernels read a table of tensor records from global memory.  Everywhere else that
+// table sits in a workspace the caller allocated; here it sits in a fixed array that is part of the
+// library image, so a caller that has no way to obtain device memory can still use one launch per
+// kernel class.  The array exists once per GPU that loads the library and is shared by every call.
+
+constexpr int kStaticMaxTensors = GWS_STATIC_MAX_TENSORS;
+constexpr size_t kStaticTableBytes = static_cast<size_t>(kStaticMaxTensors) * 2u * sizeof(Entry) + 8u * 256u;
+static __device__ __align__(256) unsigned char g_static_tables[kStaticTableBytes];
+
+// In host code `g_static_tables` is only a handle for the runtime, not an address a kernel can use: the
+// device address is looked up once per device, with that device current, and cached here.
+constexpr int kMaxDevices = 64;
+static void* g_static_tables_addr[kMaxDevices];
+static std::atomic<int> g_static_tables_ready[kMaxDevices];
+
+static int static_tables_address(void** out) {
+  int dev = -1;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return cuda_fail(err, "current device");
+  if (dev < 0 || dev >= kMaxDevices) return GWS_ERR_LIMIT;
+  if (g_static_tables_ready[dev].load(std::memory_order_acquire) == 0) {
+    void* p = nullptr;
+    err = cudaGetSymbolAddress(&p, g_static_tables);
+    if (err != cudaSuccess) return cuda_fail(err, "address of the built-in table array");
+    if (p == nullptr || !aligned(p, 256)) return GWS_ERR_WORKSPACE;
+    g_static_tables_addr[dev] = p;  // every thread that gets here stores the same value
+    g_static_tables_ready[dev].store(1, std::memory_order_release);
+  }
+  *out = g_static_tables_addr[dev];
+  return GWS_OK;
+}
+
+int gws_sample_fwd_multi_static(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, uint64_t step, void* stream) {
+  if (n < 0) return GWS_ERR_SHAPE;
+  if (n > kStaticMaxTensors) return GWS_ERR_LIMIT;  // more tensors than the built-in table holds
+  if (descs == nullptr || ptrs == nullptr) return GWS_ERR_NULL;
+  if (ptrs->w == nullptr) return GWS_ERR_NULL;  // forward pointers are required
+  gws_multi_ptrs fwd_only = *ptrs;              // the backward arrays are ignored
+  fwd_only.grad_w_hat = nullptr;
+  fwd_only.grad_w = nullptr;
+  fwd_only.grad_bt = nullptr;
+  void* table = nullptr;
+  int st = static_tables_address(&table);
+  if (st != GWS_OK) return st;
+  std::vector<char> image;
+  gws_multi_plan plan;
+  st = build_tables(n, descs, &fwd_only, table, kStaticTableBytes, &plan, image);
+  if (st != GWS_OK) return st;
+  if (image.empty()) return GWS_OK;
+  // Overwrites whatever the previous call left in the array.  The source is pageable host memory: the
+  // runtime stages it before returning, so `image` may die with this call.
+  const cudaError_t err = cudaMemcpyAsync(table, image.data(), image.size(), cudaMemcpyHostToDevice,
+                                          static_cast<cudaStream_t>(stream));
+  if (err != cudaSuccess) return cuda_fail(err, "upload into the built-in table array");
+  return run_multi(&plan, step, stream, false);
+}
+
 // ---- diagnostics ----------------------------------------------------------------------------------
 
 void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed) {
