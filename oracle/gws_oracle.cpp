@@ -21,8 +21,14 @@
 //     Element (i, j) has the logical index e = elem_offset + i*cols + j.  The
 //     Philox counter is (lo32(e>>3), hi32(e>>3), lo32(step), hi32(step)), the
 //     key is (lo32(seed), hi32(seed)).  One call serves 8 consecutive
-//     elements; element e uses the 16-bit field number (e & 7) of the 128
-//     output bits, fields counted from the least significant bits of word 0.
+//     elements.  Section 3.4 treats every bit of the random integers as one
+//     "bitwise random variable" and combines whole integers with AND / OR, so
+//     the 16 random bits of an element are 16 bit positions spread over the
+//     four output words, not 16 neighbouring bits of one word: element
+//     t = e & 7 (j = t >> 1, h = t & 1) owns the four bit columns c+1, c, c-7
+//     and c-8 with c = 16h + 14 - 2j, in each of the four words.  Bit x_k of
+//     its field is bit (c + kFieldColumn[k]) of word kFieldWord[k] (tables
+//     below); the eight fields of a vector use each of the 128 bits once.
 //   * Noise decode (Eq. 9 / Eq. 10), field bits x0 (LSB) .. x15:
 //       m2 = x0 & x1 & ... & x7 & (x8 | x9)          Pr = 2^-8 * 3/4
 //       m1 = (x10 | x11) & (x12 | x13) & x14         Pr = (3/4)^2 * 1/2
@@ -127,13 +133,27 @@ int decode_field(uint32_t field) {
   return x[15] ? -magnitude : magnitude;
 }
 
+// Where the 16 field bits of an element come from: x_k is bit (c + column[k])
+// of output word word[k], with c = 16*(t & 1) + 14 - 2*(t >> 1) for element t
+// of the vector.  x0..x7 (the eight-input AND of |R| = 2) sit in the two low
+// columns c-7, c-8 and in word 0 of the top column; x8, x9 (its OR) and the
+// sign x15 are the rest of the top column c+1; x10..x13 (the two ORs of
+// |R| = 1) are column c, x14 the remaining bit of column c-8.
+constexpr int kFieldWord[16] = {0, 1, 2, 3, 1, 2, 3, 0, 1, 2, 0, 1, 2, 3, 0, 3};
+constexpr int kFieldColumn[16] = {-7, -7, -7, -7, -8, -8, -8, +1, +1, +1, 0, 0, 0, 0, -8, +1};
+
+uint32_t field_of_element(const uint32_t o[4], unsigned t) {
+  const int c = 16 * static_cast<int>(t & 1u) + 14 - 2 * static_cast<int>(t >> 1);
+  uint32_t field = 0;
+  for (int k = 0; k < 16; ++k) field |= ((o[kFieldWord[k]] >> (c + kFieldColumn[k])) & 1u) << k;
+  return field;
+}
+
 // Noise of the element with logical index e.
 int noise_of_element(uint64_t seed, uint64_t step, uint64_t e) {
   uint32_t o[4];
   philox_for_vector(seed, step, e >> 3, o);
-  const unsigned t = static_cast<unsigned>(e & 7u);
-  const uint32_t field = (o[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu;
-  return decode_field(field);
+  return decode_field(field_of_element(o, static_cast<unsigned>(e & 7u)));
 }
 
 // ---- group geometry ----------------------------------------------------------
@@ -180,6 +200,9 @@ void gwso_philox_words(uint64_t seed, uint64_t step, uint64_t first_vec, int64_t
 }
 
 int gwso_decode_field(uint32_t field16) { return decode_field(field16 & 0xFFFFu); }
+
+// The 16-bit field of element t (0..7) of a vector whose four output words are words4.
+uint32_t gwso_field_of_element(const uint32_t* words4, uint32_t t) { return field_of_element(words4, t & 7u); }
 
 int64_t gwso_n_groups(int64_t rows, int64_t cols, int64_t group_rows, int64_t group_cols) {
   return make_geometry(rows, cols, cols, group_rows, group_cols).n_groups;
@@ -257,8 +280,7 @@ void gwso_sample_fwd(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows,
         cached_vec = e >> 3;
         philox_for_vector(seed, step, cached_vec, o);
       }
-      const unsigned t = static_cast<unsigned>(e & 7u);
-      const int r = decode_field((o[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu);
+      const int r = decode_field(field_of_element(o, static_cast<unsigned>(e & 7u)));
       const int64_t g = group_of(geo, i, j);
       const float s = scale_of(absmax_scratch[g], bt[g]);
       const float pqn = static_cast<float>(r) * s;
@@ -303,8 +325,7 @@ void gwso_sample_bwd(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows,
         cached_vec = e >> 3;
         philox_for_vector(seed, step, cached_vec, o);
       }
-      const unsigned t = static_cast<unsigned>(e & 7u);
-      const int r = decode_field((o[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu);
+      const int r = decode_field(field_of_element(o, static_cast<unsigned>(e & 7u)));
       const uint16_t gbits = grad_w_hat[i * ld + j];
       if (grad_w) grad_w[i * ld + j] = gbits;
       acc_scratch[group_of(geo, i, j)] += static_cast<double>(bf16_to_f32(gbits)) * static_cast<double>(r);

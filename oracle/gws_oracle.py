@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
         L.gwso_philox_words.restype = None
         L.gwso_decode_field.argtypes = [c_uint32]
         L.gwso_decode_field.restype = c_int
+        L.gwso_field_of_element.argtypes = [POINTER(c_uint32), c_uint32]
+        L.gwso_field_of_element.restype = c_uint32
         L.gwso_n_groups.argtypes = [c_int64] * 4
         L.gwso_n_groups.restype = c_int64
         L.gwso_noise_r.argtypes = [c_uint64, c_uint64, c_uint64, c_int64, i8p]
@@ -116,6 +118,13 @@ def philox_words(seed: int, step: int, first_vec: int, n_vec: int) -> np.ndarray
 
 def decode_field(field16: int) -> int:
     return int(lib().gwso_decode_field(field16))
+
+
+def field_of_element(words4, t: int) -> int:
+    """The 16 field bits x0..x15 of element ``t`` (0..7) gathered from the four Philox output words of its vector."""
+    w = _c(words4, np.uint32)
+    assert w.size == 4
+    return int(lib().gwso_field_of_element(_p(w, c_uint32), t))
 
 
 def n_groups(rows: int, cols: int, group_rows: int, group_cols: int) -> int:

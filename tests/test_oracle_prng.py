@@ -50,14 +50,67 @@ def test_counter_key_mapping():
     assert [int(x) for x in got] == want
 
 
-def test_field_order_inside_a_vector():
-    # element t of a vector uses bits [16*(t&1), +16) of output word t>>1
+def _columns_of(t):
+    """Bit columns owned by element t of a vector (j = t >> 1, h = t & 1): c+1, c, c-7, c-8 with c = 16h + 14 - 2j."""
+    c = 16 * (t & 1) + 14 - 2 * (t >> 1)
+    return c, {c + 1, c, c - 7, c - 8}
+
+
+def test_fields_partition_the_128_bits_of_a_vector():
+    # Flip each of the 128 output bits in turn: exactly one element's field changes, in exactly one bit, and that
+    # element is the one that owns the bit's column.  So the eight fields use every random bit exactly once
+    # (independent elements, Eq. 9's premise) and the column layout is the stated one.
+    rng = np.random.default_rng(3)
+    base = rng.integers(0, 1 << 32, 4, dtype=np.uint64).astype(np.uint32)
+    f0 = [orc.field_of_element(base, t) for t in range(8)]
+    seen = {t: set() for t in range(8)}
+    for word in range(4):
+        for col in range(32):
+            w = base.copy()
+            w[word] ^= np.uint32(1 << col)
+            changed = [(t, orc.field_of_element(w, t) ^ f0[t]) for t in range(8)]
+            changed = [(t, d) for t, d in changed if d]
+            assert len(changed) == 1, (word, col, changed)
+            t, d = changed[0]
+            assert bin(d).count("1") == 1
+            assert col in _columns_of(t)[1], (word, col, t)
+            seen[t].add(d.bit_length() - 1)
+    assert all(seen[t] == set(range(16)) for t in range(8))
+
+
+def test_field_bits_feed_the_stated_terms():
+    # Which word / column feeds which AND / OR term, stated as sets (order inside a term cannot matter):
+    #   eight-input AND of |R| = 2: columns c-7 (all four words), c-8 (words 1..3), c+1 (word 0)
+    #   its OR: column c+1 of words 1, 2;  sign: column c+1 of word 3
+    #   |R| = 1: (word 0 | word 1) & (word 2 | word 3) at column c, and word 0 at column c-8
+    for t in range(8):
+        c, _ = _columns_of(t)
+        def field_with(bits):
+            w = np.zeros(4, np.uint32)
+            for word, col in bits:
+                w[word] |= np.uint32(1 << col)
+            return orc.field_of_element(w, t)
+        and8 = [(k, c - 7) for k in range(4)] + [(k, c - 8) for k in (1, 2, 3)] + [(0, c + 1)]
+        assert field_with(and8) == 0x00FF
+        assert {field_with([(1, c + 1)]), field_with([(2, c + 1)])} == {1 << 8, 1 << 9}
+        assert field_with([(3, c + 1)]) == 1 << 15
+        assert {field_with([(0, c)]), field_with([(1, c)])} == {1 << 10, 1 << 11}
+        assert {field_with([(2, c)]), field_with([(3, c)])} == {1 << 12, 1 << 13}
+        assert field_with([(0, c - 8)]) == 1 << 14
+        # and through the decode: a full |R| = 2 pattern, a |R| = 1 pattern, their negatives
+        assert orc.decode_field(field_with(and8 + [(2, c + 1)])) == 2
+        assert orc.decode_field(field_with(and8 + [(1, c + 1), (3, c + 1)])) == -2
+        assert orc.decode_field(field_with([(1, c), (2, c), (0, c - 8)])) == 1
+        assert orc.decode_field(field_with([(0, c), (3, c), (0, c - 8), (3, c + 1)])) == -1
+        assert orc.decode_field(field_with([(0, c), (3, c)])) == 0
+
+
+def test_noise_is_decode_of_the_gathered_field():
     seed, step, vec = 99, 5, 1234
     o = orc.philox_words(seed, step, vec, 1)[0]
     r = orc.noise_r(seed, step, vec * 8, 8)
     for t in range(8):
-        field = (int(o[t >> 1]) >> (16 * (t & 1))) & 0xFFFF
-        assert int(r[t]) == orc.decode_field(field)
+        assert int(r[t]) == orc.decode_field(orc.field_of_element(o, t))
 
 
 def test_bits_are_balanced_and_streams_differ():
