@@ -574,9 +574,8 @@ void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed) {
   gws::Words4 w;
   for (int k = 0; k < 4; ++k) w.o[k] = words4[k];
   uint32_t p[4];
-  gws::decode4(w.o[0], w.o[1], p[0], p[1]);
-  gws::decode4(w.o[2], w.o[3], p[2], p[3]);
-  for (unsigned t = 0; t < 8; ++t) r8[t] = static_cast<int8_t>(gws::r_from_pair(p[t >> 1], t & 1u));
+  gws::decode8(w, p);
+  for (unsigned t = 0; t < 8; ++t) r8[t] = static_cast<int8_t>(gws::r_from_pairs(p, t));
   if (packed) *packed = gws::pack_nibbles(w);
 }
 

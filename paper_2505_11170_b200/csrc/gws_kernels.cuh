@@ -1,18 +1,25 @@
 // Device code of the sampling pass for sm_100a.
 //
-// The pass is elementwise plus a small per-group reduction, so it is bound by HBM
-// bandwidth first and by the integer pipe (Philox + decode) second.  Every kernel
-// therefore moves 16-byte vectors of 8 BF16 elements (one Philox call serves exactly
-// one such vector), issues all loads of a thread before the first use, and reduces
-// inside a warp with shuffles.  Three tilings cover the fast cases:
+// The pass is elementwise plus a small per-group reduction.  Its algorithmic cost is 4 bytes per
+// element forward and 2 backward, but every element also needs 16 random bits, so the instruction
+// issue rate (Philox4x32-10: 20 wide multiplies + 20 three-input XORs per 8 elements; the AND / OR
+// decode; the FP32 add) is the ceiling that binds before HBM does for backward and close to it for
+// forward.  The kernels are therefore written for instruction count first:
 //
-//   flat      group = 8 << k contiguous elements (k = 0..5) of a dense tensor: the tensor is
-//             a flat run of vectors, a group is 1 << k adjacent lanes of a warp.
-//   row-warp  group = one row of up to 4096 elements: one warp per row, up to 16 vectors
-//             per lane kept in registers between the max and the add (single pass over W).
+//   * one Philox call and one whole-word decode serve the 8 elements of a 16-byte vector;
+//   * the noise reaches the FP32 pipe as a BF16 bit pattern (2R), low halves widened by a shift,
+//     high halves consumed directly by the mixed-precision add / fma of sm_100;
+//   * a thread owns 64 contiguous bytes (4 vectors) of a flat group, loaded with two 32-byte loads,
+//     so a group of 128 elements is 4 lanes and needs two shuffle steps;
+//   * |w| maxima are taken on packed BF16 pairs (max.xorsign.abs), never widened.
+//
+// Four tilings:
+//   flat      group = 8 << k contiguous elements (k = 0..5) of a dense tensor: the tensor is a flat
+//             run of 64-byte chunks, one per thread; groups up to a chunk live inside the thread.
+//   row-warp  group = one row of up to 4096 elements: one warp per row, up to 16 vectors per lane
+//             kept in registers between the max and the add (single pass over W).
 //   row-cta   group = one row of up to 65536 elements: one 512-thread block per row.
-//
-// and a general kernel (one block per group, scalar accesses) handles every other shape.
+//   general   every other shape: one block per group, scalar accesses.
 // All kernels read their tensor from a table so that one launch serves many tensors.
 #pragma once
 #include <cuda_bf16.h>
@@ -93,6 +100,32 @@ __device__ __forceinline__ void st_vec(void* base, uint64_t v, const uint4& x) {
   GWS_CHECK(p, 16, 2, );
   *p = x;
 }
+// 32-byte (sm_100) accesses; `byte_off` from a 32-byte aligned base.
+struct __align__(32) Vec32 {
+  uint32_t v[8];
+};
+__device__ __forceinline__ Vec32 ld_vec32(const void* base, uint64_t byte_off) {
+  const char* p = reinterpret_cast<const char*>(base) + byte_off;
+  Vec32 r;
+#ifdef GWS_SELF_CHECK
+  if (!check_access(p, 32, 1)) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r.v[i] = 0;
+    return r;
+  }
+#endif
+  asm volatile("ld.global.nc.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]), "=r"(r.v[4]), "=r"(r.v[5]), "=r"(r.v[6]), "=r"(r.v[7])
+               : "l"(p));
+  return r;
+}
+__device__ __forceinline__ void st_vec32(void* base, uint64_t byte_off, const uint32_t* x) {
+  char* p = reinterpret_cast<char*>(base) + byte_off;
+  GWS_CHECK(p, 32, 2, );
+  asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]), "r"(x[4]),
+               "r"(x[5]), "r"(x[6]), "r"(x[7])
+               : "memory");
+}
 __device__ __forceinline__ float ld_f32(const float* base, uint64_t i) {
   GWS_CHECK(base + i, 4, 3, 0.0f);
   return __ldg(base + i);
@@ -110,30 +143,28 @@ __device__ __forceinline__ void st_u16(uint16_t* base, int64_t i, uint16_t x) {
   base[i] = x;
 }
 
-__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
-  // max of two packed pairs of non-negative BF16 values
-  __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
-  return *reinterpret_cast<uint32_t*>(&r);
+// Packed pair holding max(|a|, |b|) per BF16 half in its magnitude bits (the sign bits are the XOR
+// of the operands' signs and are dropped by absmax_finish).
+__device__ __forceinline__ uint32_t maxabs2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
 }
-
-// Packed pair whose both halves hold ... partial maxima of |x| over the vector; the caller
-// finishes with absmax_finish() after any cross-lane reduction.
-__device__ __forceinline__ uint32_t absmax_vec(const uint4& x) {
-  const uint32_t m = 0x7FFF7FFFu;
-  return bmax2(bmax2(x.x & m, x.y & m), bmax2(x.z & m, x.w & m));
-}
+__device__ __forceinline__ uint32_t absmax_vec(const uint4& x) { return maxabs2(maxabs2(x.x, x.y), maxabs2(x.z, x.w)); }
+// max over both halves, as the FP32 value of that BF16 magnitude
 __device__ __forceinline__ float absmax_finish(uint32_t pair) {
-  const uint32_t both = bmax2(pair, __byte_perm(pair, pair, 0x1032));  // max(lo, hi) in both halves
-  return __uint_as_float(both << 16);
+  const uint32_t both = maxabs2(pair, __byte_perm(pair, pair, 0x1032));
+  return __uint_as_float((both << 16) & 0x7FFF0000u);
 }
 
 // 2^(1 - b): exact for integer-valued b, double exp2 rounded to float otherwise.
+__device__ __noinline__ float pow2_one_minus_slow(float b) { return static_cast<float>(exp2(1.0 - static_cast<double>(b))); }
 __device__ __forceinline__ float pow2_one_minus(float b) {
-  if (b == truncf(b) && b >= -126.0f && b <= 127.0f) {
-    const int e = 1 - static_cast<int>(b);
-    return __int_as_float((127 + e) << 23);
+  if (b >= -126.0f && b <= 127.0f) {
+    const int bi = __float2int_rz(b);
+    if (static_cast<float>(bi) == b) return __int_as_float((128 - bi) << 23);
   }
-  return static_cast<float>(exp2(1.0 - static_cast<double>(b)));
+  return pow2_one_minus_slow(b);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16_rne(float lo, float hi) {
@@ -141,46 +172,66 @@ __device__ __forceinline__ uint32_t pack_bf16_rne(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&r);
 }
 
-// Eq. 3 + cast for one vector: 8 x ( bf16_rne( fl32(w + R*s) ) ).
-// The decode gives float(R) * 2^-126 as a bit pattern; two exact multiplies rebuild R*s.
-// w + 0.0f turns a -0.0 weight into +0.0 first, so that a signed zero noise term adds
-// nothing (R == 0 must contribute +0.0).
-__device__ __forceinline__ uint4 sample_vec(const uint4& w, const Words4& r, float s) {
-  uint32_t p[4];
-  decode4(r.o[0], r.o[1], p[0], p[1]);
-  decode4(r.o[2], r.o[3], p[2], p[3]);
-  const uint32_t wi[4] = {w.x, w.y, w.z, w.w};
-  uint32_t o[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float wl = __uint_as_float(wi[j] << 16);
-    const float wh = __uint_as_float(wi[j] & 0xFFFF0000u);
-    const float fl = __fmul_rn(__uint_as_float(p[j] << 16), 0x1p126f);
-    const float fh = __fmul_rn(__uint_as_float(p[j] & 0xFFFF0000u), 0x1p126f);
-    const float yl = __fadd_rn(__fadd_rn(wl, 0.0f), __fmul_rn(fl, s));
-    const float yh = __fadd_rn(__fadd_rn(wh, 0.0f), __fmul_rn(fh, s));
-    o[j] = pack_bf16_rne(yl, yh);
-  }
-  return make_uint4(o[0], o[1], o[2], o[3]);
+// Mixed-precision operations of sm_100: BF16 operands widened exactly, one FP32 rounding.
+__device__ __forceinline__ float fma_bf16(uint16_t a, uint16_t b, float c) {
+  float d;
+  asm("fma.rn.f32.bf16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float add_bf16(uint16_t a, float c) {
+  float d;
+  asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(a), "f"(c));
+  return d;
+}
+__device__ __forceinline__ uint16_t hi16(uint32_t x) { return static_cast<uint16_t>(x >> 16); }
+
+// The per-group factor in the forms the forward pass needs.  The decode delivers 2R, so the
+// multiplier is s/2; halving is exact unless s is below 2^-125, where the product is formed as
+// (2R * 0.5) * s instead (both roundings then match R * s).
+struct Scale {
+  float s, half;
+  bool tiny;
+};
+__device__ __forceinline__ Scale make_scale(float s) {
+  Scale k;
+  k.s = s;
+  k.half = __fmul_rn(s, 0.5f);
+  k.tiny = s < 0x1p-120f;
+  return k;
+}
+__device__ __forceinline__ float noise_term(float two_r, const Scale& k) {
+  return k.tiny ? __fmul_rn(__fmul_rn(two_r, 0.5f), k.s) : __fmul_rn(two_r, k.half);
 }
 
-// sum over the vector of float(g) * R, accumulated in element order.
-__device__ __forceinline__ float dot_vec(const uint4& g, const Words4& r) {
+// Eq. 3 + cast for one pair word: 2 x ( bf16_rne( fl32(w + R*s) ) ).  R*s is exact, the add rounds
+// once in FP32 (a separate instruction: never contracted), the pack rounds to nearest even.
+__device__ __forceinline__ uint32_t sample_pair(uint32_t w, uint32_t pair, const Scale& k) {
+  const float ql = noise_term(__uint_as_float(pair << 16), k);
+  const float qh = noise_term(__uint_as_float(pair & 0xFFFF0000u), k);
+  return pack_bf16_rne(__fadd_rn(__uint_as_float(w << 16), ql), add_bf16(hi16(w), qh));
+}
+__device__ __forceinline__ uint4 sample_vec(const uint4& w, const Words4& r, const Scale& k) {
   uint32_t p[4];
-  decode4(r.o[0], r.o[1], p[0], p[1]);
-  decode4(r.o[2], r.o[3], p[2], p[3]);
-  const uint32_t gi[4] = {g.x, g.y, g.z, g.w};
-  float acc = 0.0f;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float gl = __uint_as_float(gi[j] << 16);
-    const float gh = __uint_as_float(gi[j] & 0xFFFF0000u);
-    const float fl = __fmul_rn(__uint_as_float(p[j] << 16), 0x1p126f);
-    const float fh = __fmul_rn(__uint_as_float(p[j] & 0xFFFF0000u), 0x1p126f);
-    acc = __fmaf_rn(gl, fl, acc);
-    acc = __fmaf_rn(gh, fh, acc);
-  }
-  return acc;
+  decode8(r, p);
+  return make_uint4(sample_pair(w.x, p[0], k), sample_pair(w.y, p[1], k), sample_pair(w.z, p[2], k), sample_pair(w.w, p[3], k));
+}
+
+// acc + sum over the vector of float(g) * 2R, accumulated in element-pair order (low, high).
+__device__ __forceinline__ float dot_pair(uint32_t g, uint32_t pair, float acc) {
+  acc = __fmaf_rn(__uint_as_float(g << 16), __uint_as_float(pair << 16), acc);
+  return fma_bf16(hi16(g), hi16(pair), acc);
+}
+__device__ __forceinline__ float dot_vec(const uint4& g, const Words4& r, float acc) {
+  uint32_t p[4];
+  decode8(r, p);
+  acc = dot_pair(g.x, p[0], acc);
+  acc = dot_pair(g.y, p[1], acc);
+  acc = dot_pair(g.z, p[2], acc);
+  return dot_pair(g.w, p[3], acc);
+}
+// dL/db_t of a group from its scale and the sum of g * 2R.
+__device__ __forceinline__ float grad_bt_of(float scale, float sum_g_2r) {
+  return __fmul_rn(__fmul_rn(-kLn2, scale), __fmul_rn(sum_g_2r, 0.5f));
 }
 
 __device__ __forceinline__ Words4 philox_vec(const Entry& e, uint64_t vec_in_tensor, uint32_t step_lo, uint32_t step_hi) {
@@ -227,56 +278,153 @@ __global__ void k_locate_probe(const Entry* __restrict__ table, int n, const int
 }
 
 // ---- flat groups ------------------------------------------------------------------------------
+//
+// Tile = 256 threads x one 64-byte chunk (4 vectors, 32 elements) = 1024 vectors.  Groups of
+// 32..256 elements are 1..8 neighbouring lanes (shuffle reduction); groups of 8 or 16 elements are
+// handled inside the thread.  Only those small groups can leave a last chunk partly filled.
+
+struct Chunk {
+  uint32_t x[16];
+};
+
+// USE32: both tensor pointers are 32-byte aligned, so a chunk moves as two 32-byte accesses.
+template <bool USE32>
+__device__ __forceinline__ Chunk load_chunk(const void* base, uint64_t chunk, uint32_t n_valid) {
+  Chunk c;
+  if (USE32) {
+    const Vec32 a = ld_vec32(base, chunk * 64u), b = ld_vec32(base, chunk * 64u + 32u);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { c.x[i] = a.v[i]; c.x[8 + i] = b.v[i]; }
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint4 t = (static_cast<uint32_t>(k) < n_valid) ? ld_vec(base, chunk * 4u + k) : make_uint4(0, 0, 0, 0);
+      c.x[4 * k] = t.x; c.x[4 * k + 1] = t.y; c.x[4 * k + 2] = t.z; c.x[4 * k + 3] = t.w;
+    }
+  }
+  return c;
+}
+template <bool USE32>
+__device__ __forceinline__ void store_chunk(void* base, uint64_t chunk, uint32_t n_valid, const Chunk& c) {
+  if (USE32) {
+    st_vec32(base, chunk * 64u, c.x);
+    st_vec32(base, chunk * 64u + 32u, c.x + 8);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (static_cast<uint32_t>(k) < n_valid)
+        st_vec(base, chunk * 4u + k, make_uint4(c.x[4 * k], c.x[4 * k + 1], c.x[4 * k + 2], c.x[4 * k + 3]));
+  }
+}
+__device__ __forceinline__ uint32_t absmax_words4(const uint32_t* x) { return maxabs2(maxabs2(x[0], x[1]), maxabs2(x[2], x[3])); }
+
+// Groups of at least one chunk: `lanes` = chunks per group (1, 2, 4 or 8 neighbouring lanes).
+template <int MODE, bool USE32>
+__device__ __forceinline__ void flat_wide(const Entry& e, uint64_t chunk0, uint32_t lanes, uint32_t lanes_log2, uint32_t step_lo,
+                                          uint32_t step_hi) {
+  const uint64_t n_chunks = e.n_vec >> 2;
+  const bool ok = chunk0 < n_chunks;
+  const uint64_t chunk = ok ? chunk0 : n_chunks - 1;   // keeps the warp whole for the shuffles
+  const Chunk c = load_chunk<USE32>(e.in, chunk, 4);
+  const uint64_t g = chunk >> lanes_log2;
+  const float gv = (MODE != kAbsmax) ? ld_f32(e.gin, g) : 0.0f;
+  const bool writer = ok && (threadIdx.x & (lanes - 1u)) == 0u;
+  const uint64_t v0 = (e.elem_offset >> 3) + chunk * 4u;
+
+  if (MODE == kBwd) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const Words4 r = philox_for_vector(v0 + k, step_lo, step_hi, e.seed_lo, e.seed_hi);
+      acc = dot_vec(make_uint4(c.x[4 * k], c.x[4 * k + 1], c.x[4 * k + 2], c.x[4 * k + 3]), r, acc);
+    }
+    for (uint32_t o = 1; o < lanes; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if (writer) st_f32(e.gout, g, grad_bt_of(gv, acc));
+    if (ok && e.out != nullptr) store_chunk<USE32>(e.out, chunk, 4, c);
+    return;
+  }
+  uint32_t m = maxabs2(maxabs2(absmax_words4(c.x), absmax_words4(c.x + 4)), maxabs2(absmax_words4(c.x + 8), absmax_words4(c.x + 12)));
+  for (uint32_t o = 1; o < lanes; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  const float a = absmax_finish(m);
+  if (MODE == kAbsmax) {
+    if (writer) st_f32(e.gout, g, a);
+    return;
+  }
+  const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv)));
+  Chunk y;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const Words4 r = philox_for_vector(v0 + k, step_lo, step_hi, e.seed_lo, e.seed_hi);
+    uint32_t p[4];
+    decode8(r, p);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) y.x[4 * k + j] = sample_pair(c.x[4 * k + j], p[j], sc);
+  }
+  if (ok) {
+    store_chunk<USE32>(e.out, chunk, 4, y);
+    if (writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
+  }
+}
+
+// Groups of one or two vectors (8 or 16 elements): 4 or 2 groups inside the thread's chunk.
+template <int MODE>
+__device__ __forceinline__ void flat_narrow(const Entry& e, uint64_t chunk, uint32_t ll, uint32_t step_lo, uint32_t step_hi) {
+  const uint64_t first = chunk * 4u;
+  if (first >= e.n_vec) return;
+  const uint32_t n_valid = static_cast<uint32_t>(min(static_cast<uint64_t>(4), e.n_vec - first));
+  const Chunk c = load_chunk<false>(e.in, chunk, n_valid);
+  const uint64_t v0 = (e.elem_offset >> 3) + first;
+  Chunk y;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    if (static_cast<uint32_t>(k) >= n_valid) break;
+    const uint64_t g = (first + k) >> ll;
+    const bool writer = ll == 0u || (k & 1) == 0;
+    const uint4 xv = make_uint4(c.x[4 * k], c.x[4 * k + 1], c.x[4 * k + 2], c.x[4 * k + 3]);
+    const int mate = k ^ 1;   // the other vector of a two-vector group (always inside the chunk)
+    const Words4 r = philox_for_vector(v0 + k, step_lo, step_hi, e.seed_lo, e.seed_hi);
+    if (MODE == kBwd) {
+      if (writer) {
+        float acc = dot_vec(xv, r, 0.0f);
+        if (ll == 1u) {
+          const Words4 r2 = philox_for_vector(v0 + mate, step_lo, step_hi, e.seed_lo, e.seed_hi);
+          acc = dot_vec(make_uint4(c.x[4 * mate], c.x[4 * mate + 1], c.x[4 * mate + 2], c.x[4 * mate + 3]), r2, acc);
+        }
+        st_f32(e.gout, g, grad_bt_of(ld_f32(e.gin, g), acc));
+      }
+      continue;
+    }
+    uint32_t m = absmax_vec(xv);
+    if (ll == 1u) m = maxabs2(m, absmax_words4(c.x + 4 * mate));
+    const float a = absmax_finish(m);
+    if (MODE == kAbsmax) {
+      if (writer) st_f32(e.gout, g, a);
+      continue;
+    }
+    const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(ld_f32(e.gin, g))));
+    const uint4 yv = sample_vec(xv, r, sc);
+    y.x[4 * k] = yv.x; y.x[4 * k + 1] = yv.y; y.x[4 * k + 2] = yv.z; y.x[4 * k + 3] = yv.w;
+    if (writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
+  }
+  if (MODE == kFwd) store_chunk<false>(e.out, chunk, n_valid, y);
+  if (MODE == kBwd && e.out != nullptr) store_chunk<false>(e.out, chunk, n_valid, c);
+}
 
 template <int MODE, bool MULTI>
 __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ Entry single,
                                                        const Entry* __restrict__ table, int n, uint32_t step_lo,
                                                        uint32_t step_hi) {
-  constexpr int T = kFlatThreads, V = kFlatVecs;
   GWS_RESOLVE_ENTRY(e, tile)
-  const uint32_t ll = e.lanes_log2;
-  const uint32_t L = 1u << ll;
-  const uint32_t lane_in_group = threadIdx.x & (L - 1u);
-  const uint64_t base = static_cast<uint64_t>(tile) * (T * V) + threadIdx.x;
-
-  uint4 x[V];
-  float gv[V];
-  bool ok[V];
-#pragma unroll
-  for (int k = 0; k < V; ++k) {
-    const uint64_t v = base + static_cast<uint64_t>(k) * T;
-    ok[k] = v < e.n_vec;
-    x[k] = ok[k] ? ld_vec(e.in, v) : make_uint4(0, 0, 0, 0);
-    gv[k] = 0.0f;
-    if (MODE != kAbsmax && ok[k]) gv[k] = ld_f32(e.gin, v >> ll);
+  const uint32_t ll = e.lanes_log2;   // log2(vectors per group)
+  const uint64_t chunk = static_cast<uint64_t>(tile) * kFlatThreads + threadIdx.x;
+  if (ll < 2u) {
+    flat_narrow<MODE>(e, chunk, ll, step_lo, step_hi);
+    return;
   }
-#pragma unroll
-  for (int k = 0; k < V; ++k) {
-    const uint64_t v = base + static_cast<uint64_t>(k) * T;
-    const uint64_t g = v >> ll;
-    if (MODE == kBwd) {
-      float acc = dot_vec(x[k], philox_vec(e, v, step_lo, step_hi));
-      for (uint32_t o = 1; o < L; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-      if (ok[k]) {
-        if (lane_in_group == 0) st_f32(e.gout, g, __fmul_rn(__fmul_rn(-kLn2, gv[k]), acc));
-        if (e.out != nullptr) st_vec(e.out, v, x[k]);
-      }
-    } else {
-      uint32_t m = absmax_vec(x[k]);
-      for (uint32_t o = 1; o < L; o <<= 1) m = bmax2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-      const float a = absmax_finish(m);
-      if (MODE == kAbsmax) {
-        if (ok[k] && lane_in_group == 0) st_f32(e.gout, g, a);
-      } else {
-        const float s = __fmul_rn(a, pow2_one_minus(gv[k]));
-        const uint4 y = sample_vec(x[k], philox_vec(e, v, step_lo, step_hi), s);
-        if (ok[k]) {
-          st_vec(e.out, v, y);
-          if (e.gout != nullptr && lane_in_group == 0) st_f32(e.gout, g, s);
-        }
-      }
-    }
-  }
+  const uint32_t lanes_log2 = ll - 2u, lanes = 1u << lanes_log2;
+  const bool use32 = ((reinterpret_cast<uintptr_t>(e.in) | reinterpret_cast<uintptr_t>(e.out)) & 31u) == 0u;
+  if (use32) flat_wide<MODE, true>(e, chunk, lanes, lanes_log2, step_lo, step_hi);
+  else flat_wide<MODE, false>(e, chunk, lanes, lanes_log2, step_lo, step_hi);
 }
 
 // ---- one warp per row ---------------------------------------------------------------------------
@@ -311,28 +459,26 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
       if (k * 32u < vpr) {
         const uint32_t j = k * 32u + lane;
         const bool ok = okr && j < vpr;
-        const float part = dot_vec(x[k], philox_vec(e, vbase + j, step_lo, step_hi));
-        if (ok) {
-          acc += part;
-          if (e.out != nullptr) st_vec(e.out, vbase + j, x[k]);
-        }
+        // vectors past the end of the row are all zero and add nothing
+        acc = dot_vec(x[k], philox_vec(e, vbase + j, step_lo, step_hi), acc);
+        if (ok && e.out != nullptr) st_vec(e.out, vbase + j, x[k]);
       }
     }
 #pragma unroll
     for (uint32_t o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-    if (okr && lane == 0) st_f32(e.gout, row, __fmul_rn(__fmul_rn(-kLn2, gvr), acc));
+    if (okr && lane == 0) st_f32(e.gout, row, grad_bt_of(gvr, acc));
   } else {
     uint32_t m = 0;
 #pragma unroll
     for (int k = 0; k < V; ++k)
-      if (k * 32u < vpr) m = bmax2(m, absmax_vec(x[k]));
+      if (k * 32u < vpr) m = maxabs2(m, absmax_vec(x[k]));
 #pragma unroll
-    for (uint32_t o = 16; o > 0; o >>= 1) m = bmax2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    for (uint32_t o = 16; o > 0; o >>= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     const float a = absmax_finish(m);
     if (MODE == kAbsmax) {
       if (okr && lane == 0) st_f32(e.gout, row, a);
     } else {
-      const float s = __fmul_rn(a, pow2_one_minus(gvr));
+      const Scale s = make_scale(__fmul_rn(a, pow2_one_minus(gvr)));
 #pragma unroll
       for (int k = 0; k < V; ++k) {
         if (k * 32u < vpr) {
@@ -341,7 +487,7 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
           if (okr && j < vpr) st_vec(e.out, vbase + j, y);
         }
       }
-      if (okr && lane == 0 && e.gout != nullptr) st_f32(e.gout, row, s);
+      if (okr && lane == 0 && e.gout != nullptr) st_f32(e.gout, row, s.s);
     }
   }
 }
@@ -378,11 +524,8 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
     for (int k = 0; k < V; ++k) {
       if (static_cast<uint32_t>(k) * T < vpr) {
         const uint32_t j = k * T + threadIdx.x;
-        const float part = dot_vec(x[k], philox_vec(e, vbase + j, step_lo, step_hi));
-        if (j < vpr) {
-          acc += part;
-          if (e.out != nullptr) st_vec(e.out, vbase + j, x[k]);
-        }
+        acc = dot_vec(x[k], philox_vec(e, vbase + j, step_lo, step_hi), acc);   // zero vectors past the row add nothing
+        if (j < vpr && e.out != nullptr) st_vec(e.out, vbase + j, x[k]);
       }
     }
 #pragma unroll
@@ -392,25 +535,25 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
     if (threadIdx.x == 0) {
       float total = 0.0f;
       for (int w = 0; w < WARPS; ++w) total += red_f[w];  // fixed order
-      st_f32(e.gout, row, __fmul_rn(__fmul_rn(-kLn2, gvr), total));
+      st_f32(e.gout, row, grad_bt_of(gvr, total));
     }
   } else {
     uint32_t m = 0;
 #pragma unroll
     for (int k = 0; k < V; ++k)
-      if (static_cast<uint32_t>(k) * T < vpr) m = bmax2(m, absmax_vec(x[k]));
+      if (static_cast<uint32_t>(k) * T < vpr) m = maxabs2(m, absmax_vec(x[k]));
 #pragma unroll
-    for (uint32_t o = 16; o > 0; o >>= 1) m = bmax2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    for (uint32_t o = 16; o > 0; o >>= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     if (lane == 0) red_u[warp] = m;
     __syncthreads();
     uint32_t mm = red_u[0];
 #pragma unroll
-    for (int w = 1; w < WARPS; ++w) mm = bmax2(mm, red_u[w]);
+    for (int w = 1; w < WARPS; ++w) mm = maxabs2(mm, red_u[w]);
     const float a = absmax_finish(mm);
     if (MODE == kAbsmax) {
       if (threadIdx.x == 0) st_f32(e.gout, row, a);
     } else {
-      const float s = __fmul_rn(a, pow2_one_minus(gvr));
+      const Scale s = make_scale(__fmul_rn(a, pow2_one_minus(gvr)));
 #pragma unroll
       for (int k = 0; k < V; ++k) {
         if (static_cast<uint32_t>(k) * T < vpr) {
@@ -419,7 +562,7 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
           if (j < vpr) st_vec(e.out, vbase + j, y);
         }
       }
-      if (threadIdx.x == 0 && e.gout != nullptr) st_f32(e.gout, row, s);
+      if (threadIdx.x == 0 && e.gout != nullptr) st_f32(e.gout, row, s.s);
     }
   }
 }
@@ -477,7 +620,9 @@ __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_consta
         const int64_t i = r0 + k / wd, j = c0 + k % wd;
         const uint64_t el = e.elem_offset + static_cast<uint64_t>(i * e.cols + j);
         const Words4 words = philox_for_vector(el >> 3, step_lo, step_hi, e.seed_lo, e.seed_hi);
-        const int r = decode_field(field_of(words, static_cast<unsigned>(el & 7u)));
+        uint32_t pairs[4];
+        decode8(words, pairs);
+        const int r = r_from_pairs(pairs, static_cast<unsigned>(el & 7u));
         const uint16_t bits = ld_u16(in, i * e.ld + j);
         const float val = __uint_as_float(static_cast<uint32_t>(bits) << 16);
         if (MODE == kFwd) {

@@ -1,6 +1,6 @@
-// Inline arithmetic of the sampling pass: Philox4x32-10, the AND/OR noise decode of
-// Eq. 9 / Eq. 10 and the nibble packing of Section 3.4.  Integer-only, so the same
-// code runs in kernels and (for host-side tests of the bit tricks) on the CPU.
+// Inline integer arithmetic of the sampling pass: Philox4x32-10, the AND/OR noise decode of
+// Eq. 9 / Eq. 10 on whole random words, and the nibble packing of Section 3.4.  Integer-only,
+// so the same code runs in kernels and (for host-side tests of the bit tricks) on the CPU.
 #pragma once
 #include <stdint.h>
 
@@ -47,75 +47,58 @@ GWS_HD Words4 philox_for_vector(uint64_t vec, uint32_t step_lo, uint32_t step_hi
   return philox4x32_10(static_cast<uint32_t>(vec), static_cast<uint32_t>(vec >> 32), step_lo, step_hi, seed_lo, seed_hi);
 }
 
-// Byte permute with the semantics of the PTX prmt instruction in its default mode,
-// selector nibbles restricted to 0..7 (no sign replication).
-GWS_HD uint32_t byte_perm(uint32_t a, uint32_t b, uint32_t sel) {
-#if defined(__CUDA_ARCH__)
-  return __byte_perm(a, b, sel);
-#else
-  const uint64_t both = (static_cast<uint64_t>(b) << 32) | a;
-  uint32_t out = 0;
-  for (int k = 0; k < 4; ++k) {
-    const uint32_t idx = (sel >> (4 * k)) & 7u;
-    out |= static_cast<uint32_t>((both >> (8 * idx)) & 0xFFu) << (8 * k);
-  }
-  return out;
-#endif
-}
-
-// Decode four 16-bit fields (two Philox words) at once, one byte lane per field.
+// ---- noise decode on whole words ------------------------------------------------------------------
 //
-// Field bits x0..x15; hi byte y = x8..x15, lo byte l = x0..x7.
-//   m2 = (l == 0xFF) & (x8|x9)          |R| = 2
-//   m1 = (x10|x11) & (x12|x13) & x14    |R| = 1 unless m2
-// Output: two words, each holding two elements as the upper halves of FP32 bit patterns,
-// element (2k) in bits 0..15 and element (2k+1) in bits 16..31 of p[k]:
-//   bit 15: x15 (raw sign), bit 8: m2, bit 7: m1 & ~m2, all other bits 0.
-// Shifted into the top of a 32-bit word this is sign | exponent field 2 or 1, i.e.
-// +-2^-125 or +-2^-126 (or +-0): multiply by 2^126 to get float(R) (with R = 0 possibly -0.0).
-GWS_HD void decode4(uint32_t wa, uint32_t wb, uint32_t& p01, uint32_t& p23) {
-  const uint32_t H = byte_perm(wa, wb, 0x7531u);  // hi bytes of fields 0..3
-  const uint32_t L = byte_perm(wa, wb, 0x6420u);  // lo bytes of fields 0..3
-  const uint32_t a = H | (H >> 1);                // per byte: bit0 = x8|x9, bit2 = x10|x11, bit4 = x12|x13
-  const uint32_t M1 = (a << 4) & (a << 2) & H;    // per byte bit 6 = m1
-  const uint32_t c = (L & 0x7F7F7F7Fu) + 0x01010101u;  // per byte bit 7 = (x0..x6 all ones)
-  const uint32_t M2 = c & L & (a << 7);           // per byte bit 7 = m2
-  const uint32_t C = (H & 0x80808080u) | ((M2 >> 7) & 0x01010101u);  // sign at bit 7, m2 at bit 0
-  const uint32_t A = ((M1 << 1) & ~M2) & 0x80808080u;                // m1 & ~m2 at bit 7
-  p01 = byte_perm(C, A, 0x1504u);
-  p23 = byte_perm(C, A, 0x3726u);
+// Element t of a vector (j = t >> 1, h = t & 1) owns four bit columns of the four output words
+// o0..o3:  A = 16h + 14 - 2j,  S = A + 1,  M = A - 7,  F = A - 8.  With o_k[c] = bit c of word k:
+//
+//   |R| = 2  iff  o0[M] & o1[M] & o2[M] & o3[M] & o1[F] & o2[F] & o3[F] & o0[S] & (o1[S] | o2[S])   Pr = 2^-8 * 3/4
+//   |R| = 1  iff  not that, and (o0[A] | o1[A]) & (o2[A] | o3[A]) & o0[F]                           Pr = (3/4)^2 / 2
+//   R < 0    iff  o3[S] and |R| != 0
+//
+// Every AND / OR below therefore evaluates one term of Eq. 10 for all eight elements at once; shifts
+// only line up columns (M + 7 = A, F + 8 = A, S - 8 = M, F + 1 = M).  The columns are laid out so
+// that `Z << 2j` brings the three flags of elements 2j (low half) and 2j+1 (high half) to bits
+// 15 (sign), 14 (non-zero) and 7 (|R| = 2) of each 16-bit half: with all other bits cleared that
+// half is the BF16 number 2R (0x4000 = 2.0, 0x4080 = 4.0, sign on top), and zero is always +0.
+constexpr uint32_t kColsM = 0x00AA00AAu;   // bit columns M of the eight elements
+constexpr uint32_t kColsS = 0xAA00AA00u;   // bit columns S
+constexpr uint32_t kPairMask = 0xC080C080u;
+
+GWS_HD void decode8(const Words4& r, uint32_t (&pair)[4]) {
+  const uint32_t o0 = r.o[0], o1 = r.o[1], o2 = r.o[2], o3 = r.o[3];
+  const uint32_t t1 = o1 & o2 & o3;
+  const uint32_t and7 = t1 & o0 & (t1 << 1);        // at M: o0..o3[M] & o1..o3[F]
+  const uint32_t top = o0 & (o1 | o2);              // at S: o0[S] & (o1[S] | o2[S])
+  const uint32_t m2 = and7 & (top >> 8);            // at M
+  const uint32_t m1 = (o0 | o1) & (o0 << 8) & (o2 | o3);   // at A
+  const uint32_t any = m1 | (m2 << 7);              // at A
+  const uint32_t z1 = (any & ~kColsM) | (m2 & kColsM);
+  const uint32_t sgn = o3 & (any << 1);             // at S; zero noise keeps a positive sign
+  const uint32_t z = (sgn & kColsS) | (z1 & ~kColsS);
+  pair[0] = z & kPairMask;
+  pair[1] = (z << 2) & kPairMask;
+  pair[2] = (z << 4) & kPairMask;
+  pair[3] = (z << 6) & kPairMask;
 }
 
-// Plain per-field decode, straight from the definition (used by the general kernel,
-// the noise packer and as the cross-check of decode4).
-GWS_HD int decode_field(uint32_t x) {
-  const bool m2 = ((x & 0xFFu) == 0xFFu) && ((x & 0x300u) != 0u);
-  const bool m1 = ((x & 0xC00u) != 0u) && ((x & 0x3000u) != 0u) && ((x & 0x4000u) != 0u);
-  const int mag = m2 ? 2 : (m1 ? 1 : 0);
-  return (x & 0x8000u) ? -mag : mag;
-}
-
-GWS_HD uint32_t field_of(const Words4& w, unsigned t) { return (w.o[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu; }
-
-// R of field t (0..7) recovered from the decode4 outputs.
-GWS_HD int r_from_pair(uint32_t pair, unsigned odd) {
-  const uint32_t h = (pair >> (16u * odd)) & 0xFFFFu;
-  const int mag = static_cast<int>((h >> 7) & 3u);  // 1 or 2 (never 3)
+// R of element t (0..7) from the pair words of its vector.
+GWS_HD int r_from_pairs(const uint32_t (&pair)[4], unsigned t) {
+  const uint32_t h = (pair[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu;
+  const int mag = static_cast<int>(((h >> 14) & 1u) + ((h >> 7) & 1u));
   return (h & 0x8000u) ? -mag : mag;
 }
 
-// Packed sign-magnitude nibbles of 8 elements; zero is never negative.
+// Packed sign-magnitude nibbles of 8 elements (nibble t = sign << 3 | |R|); zero is never negative.
 GWS_HD uint32_t pack_nibbles(const Words4& w) {
-  uint32_t p[4];
-  decode4(w.o[0], w.o[1], p[0], p[1]);
-  decode4(w.o[2], w.o[3], p[2], p[3]);
+  uint32_t pair[4];
+  decode8(w, pair);
   uint32_t out = 0;
 #pragma unroll
   for (unsigned t = 0; t < 8; ++t) {
-    const uint32_t h = (p[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu;
-    const uint32_t mag = (h >> 7) & 3u;
-    const uint32_t neg = (mag != 0u) ? (h >> 15) : 0u;
-    out |= ((neg << 3) | mag) << (4u * t);
+    const uint32_t h = (pair[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu;
+    const uint32_t mag = ((h >> 14) & 1u) + ((h >> 7) & 1u);
+    out |= (((h >> 15) << 3) | mag) << (4u * t);
   }
   return out;
 }

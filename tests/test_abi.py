@@ -115,23 +115,35 @@ def test_inline_philox_matches_oracle(lib):
 
 
 def test_inline_decode_matches_oracle_on_every_field_value(lib):
-    # each of the 65536 field values, placed in each of the 8 field positions, random bits elsewhere
+    # each of the 65536 field values, scattered into the bit columns of each of the 8 elements, random bits elsewhere
     rng = np.random.default_rng(1)
     want = np.array([orc.decode_field(x) for x in range(1 << 16)], np.int64)
     noise_words = rng.integers(0, 1 << 32, size=(1 << 16, 4), dtype=np.uint64)
+    # where the oracle reads bit k of element t's field: found by probing it with single-bit words
+    where = {}
+    for word in range(4):
+        for col in range(32):
+            w = [0, 0, 0, 0]
+            w[word] = 1 << col
+            for t in range(8):
+                f = orc.field_of_element(w, t)
+                if f:
+                    where[(t, f.bit_length() - 1)] = (word, col)
+    assert len(where) == 128
     for t in range(8):
         for x in range(0, 1 << 16, 1):
             if (x * 8 + t) % 5:            # a fifth of all (value, position) pairs, every value covered in some position
                 continue
             words = [int(v) for v in noise_words[x]]
-            k, sh = t >> 1, 16 * (t & 1)
-            words[k] = (words[k] & ~(0xFFFF << sh)) | (x << sh)
+            for k in range(16):
+                word, col = where[(t, k)]
+                words[word] = (words[word] & ~(1 << col)) | (((x >> k) & 1) << col)
             r, packed = binding.host_decode8(words)
             assert r[t] == want[x], (hex(x), t, r[t], want[x])
             nib = (packed >> (4 * t)) & 0xF
             mag = abs(int(want[x]))
             assert nib == ((8 if want[x] < 0 else 0) | mag)
-            # neighbours are decoded from their own bits
-            for u in range(8):
-                fu = (words[u >> 1] >> (16 * (u & 1))) & 0xFFFF
-                assert r[u] == want[fu]
+            if x % 64 == 0:
+                # neighbours are decoded from their own bits
+                for u in range(8):
+                    assert r[u] == want[orc.field_of_element(words, u)]
