@@ -148,6 +148,7 @@ typedef struct gws_multi_ptrs {
 /* Caller-owned, filled by gws_multi_prepare, read by the *_multi calls.  Plain data. */
 typedef struct gws_multi_plan {
   void* workspace;
+  const void* host_tables; /* the host copy of the tables (host_workspace of gws_multi_prepare)          */
   int32_t n_tensors;
   int32_t has_fwd, has_bwd;
   int32_t count[4];     /* tensors per kernel class: flat groups, warp-per-row, CTA-per-row, general */
@@ -156,17 +157,22 @@ typedef struct gws_multi_plan {
   int64_t total_elements;
 } gws_multi_plan;
 
-/* Bytes of device workspace gws_multi_prepare needs for n tensors (256-byte aligned base). */
+/* Bytes gws_multi_prepare needs for n tensors, both of device workspace (256-byte aligned base) and
+ * of host workspace. */
 size_t gws_workspace_bytes(int n_tensors);
 
 /*
- * Validate n descriptors and pointer sets, build the tile tables and copy them into
- * `workspace` on `stream` (from pageable host memory: the call may wait for earlier work
- * on the stream, so call it outside the training loop).  desc[i].step is ignored.
- * The workspace must stay untouched for as long as the plan is used.
+ * Validate n descriptors and pointer sets, build the tile tables, keep one copy in `host_workspace`
+ * (HOST memory, caller-owned, at least gws_workspace_bytes(n)) and copy them into `workspace`
+ * (DEVICE memory) on `stream`; the call waits for that copy, so call it outside the training loop.
+ * desc[i].step is ignored.  Both workspaces must stay untouched for as long as the plan is used:
+ * row and general kernels read their tensor records from the device copy; flat-group launches
+ * (groups of 8..256 contiguous elements) take theirs from the host copy and pass up to 240 of them
+ * by value in the kernel parameters, so that a thread block finds its tensor without a memory access.
  */
 int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace,
-                      size_t workspace_bytes, gws_multi_plan* plan_out, void* stream);
+                      size_t workspace_bytes, void* host_workspace, size_t host_workspace_bytes,
+                      gws_multi_plan* plan_out, void* stream);
 
 /* The bytes gws_multi_prepare would upload, written to HOST memory instead (nothing touches the
  * GPU): lets a caller or a test inspect the tables.  Returns the image size in bytes (pass
@@ -178,12 +184,17 @@ int64_t gws_multi_table_image(int n, const gws_desc* descs, const gws_multi_ptrs
                               size_t workspace_bytes, gws_multi_plan* plan_out, void* host_image,
                               size_t host_image_bytes);
 
-/* Diagnostic: resolves n_tiles thread-block indices of one launch (kernel_class 0..2, forward or
+/* Diagnostic: resolves n_tiles thread-block indices of one launch (kernel_class 1..2, forward or
  * backward table) to their tensors on the device.  tiles: device, int64 [n_tiles], each inside
  * [0, plan->tiles[kernel_class]).  out: device, u64 [6*n_tiles] = {in, out, gin, gout pointers,
  * tile index inside the tensor, rows of the tensor} per tile.  Reads the tables only. */
 int gws_multi_locate_probe(const gws_multi_plan* plan, int backward, int kernel_class, const int64_t* tiles,
                            int n_tiles, uint64_t* out, void* stream);
+
+/* Kernel launches one forward (backward != 0: backward) pass of the plan enqueues: one per kernel
+ * class in use, one more if groups of 8 / 16 elements occur beside wider flat groups, one per 240
+ * flat-group tensors beyond the first 240, one per general-class tensor. */
+int gws_multi_launch_count(const gws_multi_plan* plan, int backward);
 
 /* Forward / backward of every tensor of the plan for gradient-update counter `step`. */
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);

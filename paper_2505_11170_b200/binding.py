@@ -50,7 +50,7 @@ class _MultiPtrs(Structure):
 
 
 class _MultiPlan(Structure):
-    _fields_ = [("workspace", c_void_p), ("n_tensors", c_int32), ("has_fwd", c_int32), ("has_bwd", c_int32),
+    _fields_ = [("workspace", c_void_p), ("host_tables", c_void_p), ("n_tensors", c_int32), ("has_fwd", c_int32), ("has_bwd", c_int32),
                 ("count", c_int32 * 4), ("tiles", c_int64 * 4), ("fwd_offset", c_int64 * 4), ("bwd_offset", c_int64 * 4),
                 ("total_elements", c_int64)]
 
@@ -65,9 +65,11 @@ _SIGNATURES = {
     "gws_sample_fwd": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gws_sample_bwd": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gws_workspace_bytes": (c_size_t, [c_int]),
-    "gws_multi_prepare": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, POINTER(_MultiPlan), c_void_p]),
+    "gws_multi_prepare": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, c_void_p, c_size_t,
+                                  POINTER(_MultiPlan), c_void_p]),
     "gws_multi_table_image": (c_int64, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, POINTER(_MultiPlan), c_void_p, c_size_t]),
     "gws_multi_locate_probe": (c_int, [POINTER(_MultiPlan), c_int, c_int, c_void_p, c_int, c_void_p, c_void_p]),
+    "gws_multi_launch_count": (c_int, [POINTER(_MultiPlan), c_int]),
     "gws_sample_fwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_sample_bwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_sample_fwd_multi_static": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_uint64, c_void_p]),
@@ -232,8 +234,9 @@ class MultiPlan:
         nbytes = int(lib.gws_workspace_bytes(n))
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=anyt.device)
         self.plan = _MultiPlan()
+        self._host_workspace = (ctypes.c_char * max(nbytes, 1))()     # the plan reads it at every launch
         _check(lib.gws_multi_prepare(n, self._descs, ctypes.byref(self._ptrs), _ptr(self.workspace), nbytes,
-                                     ctypes.byref(self.plan), _stream(stream)))
+                                     ctypes.cast(self._host_workspace, c_void_p), nbytes, ctypes.byref(self.plan), _stream(stream)))
 
     @property
     def total_elements(self) -> int:
@@ -241,8 +244,10 @@ class MultiPlan:
 
     @property
     def launches_per_pass(self) -> int:
-        c = list(self.plan.count)
-        return sum(1 for k in range(3) if c[k]) + c[3]
+        n = load_library().gws_multi_launch_count(ctypes.byref(self.plan), 0 if self.plan.has_fwd else 1)
+        if n < 0:
+            raise GwsError(int(n))
+        return int(n)
 
     def locate_probe(self, backward: bool, kernel_class: int, tiles: torch.Tensor, stream=None) -> torch.Tensor:
         """Diagnostic: (n_tiles, 6) int64 rows {in, out, gin, gout, tile inside tensor, rows} resolved on the device."""

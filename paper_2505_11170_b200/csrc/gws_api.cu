@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in gws.h: argument validation, choice of kernel class,
 // launch geometry, the multi-tensor table.  No device memory is allocated here.
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstring>
@@ -119,13 +120,85 @@ Entry make_entry(const gws_desc* d, int cls, const void* in, void* out, const fl
   return e;
 }
 
+// ---- flat-group launches: tensor records by value in the kernel parameters ---------------------------
+
+gws::FlatRec to_flat_rec(const Entry& e) {
+  gws::FlatRec r;
+  std::memset(&r, 0, sizeof r);
+  r.in = e.in;
+  r.out = e.out;
+  r.gin = e.gin;
+  r.gout = e.gout;
+  r.vec0 = e.elem_offset >> 3;
+  r.n_vec = e.n_vec;
+  r.seed_lo = e.seed_lo;
+  r.seed_hi = e.seed_hi;
+  r.lanes_log2 = e.lanes_log2;
+  return r;
+}
+
+int64_t flat_tiles_of(const gws::FlatRec& r) {
+  const int64_t per = static_cast<int64_t>(gws::kFlatThreads) * gws::kFlatVecs;
+  return (static_cast<int64_t>(r.n_vec) + per - 1) / per;
+}
+
+template <int MODE, int VARIANT, int CAP>
+int launch_flat_batch(gws::FlatRec* recs, int count, uint32_t lo, uint32_t hi, cudaStream_t stream) {
+  gws::FlatBatch<CAP> b;
+  std::memset(&b, 0, sizeof b);
+  int64_t tiles = 0;
+  for (int k = 0; k < count; ++k) {
+    b.e[k] = recs[k];
+    b.e[k].tile_begin = static_cast<int32_t>(tiles);
+    tiles += flat_tiles_of(recs[k]);
+    if (tiles > kMaxGrid) return GWS_ERR_LIMIT;
+  }
+  b.n = count;
+  while (((tiles - 1) >> b.hint_shift) >= gws::kFlatHint) ++b.hint_shift;
+  int owner = 0;
+  for (int h = 0; h < gws::kFlatHint; ++h) {
+    const int64_t t = static_cast<int64_t>(h) << b.hint_shift;
+    while (owner + 1 < count && b.e[owner + 1].tile_begin <= t) ++owner;
+    b.hint[h] = static_cast<uint16_t>(owner);
+  }
+  gws::k_flat<MODE, VARIANT, CAP><<<static_cast<unsigned>(tiles), gws::kFlatThreads, 0, stream>>>(b, lo, hi);
+  return check_launch("flat-group kernel");
+}
+
+template <int MODE, int VARIANT>
+int launch_flat_variant(std::vector<gws::FlatRec>& recs, uint32_t lo, uint32_t hi, cudaStream_t stream) {
+  for (size_t first = 0; first < recs.size(); first += gws::kFlatCapLarge) {
+    const int count = static_cast<int>(std::min(recs.size() - first, static_cast<size_t>(gws::kFlatCapLarge)));
+    const int st = count <= gws::kFlatCapSmall
+                       ? launch_flat_batch<MODE, VARIANT, gws::kFlatCapSmall>(recs.data() + first, count, lo, hi, stream)
+                       : launch_flat_batch<MODE, VARIANT, gws::kFlatCapLarge>(recs.data() + first, count, lo, hi, stream);
+    if (st != GWS_OK) return st;
+  }
+  return GWS_OK;
+}
+
+// Launches needed for `count` flat-class entries: groups of 8 / 16 elements run apart from the wider ones.
+template <int MODE>
+int launch_flat(const Entry* entries, int count, uint64_t step, cudaStream_t stream) {
+  std::vector<gws::FlatRec> wide, narrow;
+  bool all32 = true;
+  for (int k = 0; k < count; ++k) {
+    const gws::FlatRec r = to_flat_rec(entries[k]);
+    if (r.lanes_log2 < 2u) { narrow.push_back(r); continue; }
+    wide.push_back(r);
+    all32 = all32 && aligned(r.in, 32) && aligned(r.out, 32);
+  }
+  const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
+  int st = all32 ? launch_flat_variant<MODE, gws::kWide32>(wide, lo, hi, stream)
+                 : launch_flat_variant<MODE, gws::kWide16>(wide, lo, hi, stream);
+  if (st != GWS_OK) return st;
+  return launch_flat_variant<MODE, gws::kNarrow>(narrow, lo, hi, stream);
+}
+
 template <int MODE, bool MULTI>
 int launch_as(int cls, const Entry& single, const Entry* table, int n_or_index, unsigned grid, uint32_t lo, uint32_t hi,
               cudaStream_t stream) {
   switch (cls) {
-    case gws::kFlat:
-      gws::k_flat<MODE, MULTI><<<grid, gws::kFlatThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
-      return check_launch("flat-group kernel");
     case gws::kRowWarp:
       gws::k_row_warp<MODE, MULTI><<<grid, gws::kRowWarpThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
       return check_launch("warp-per-row kernel");
@@ -145,6 +218,7 @@ int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int
            cudaStream_t stream) {
   if (tiles <= 0) return GWS_OK;
   if (tiles > kMaxGrid) return GWS_ERR_LIMIT;
+  if (cls == gws::kFlat) return launch_flat<MODE>(&single, 1, step, stream);   // single-tensor calls only
   const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
   const unsigned grid = static_cast<unsigned>(tiles);
   return table == nullptr ? launch_as<MODE, false>(cls, single, table, n_or_index, grid, lo, hi, stream)
@@ -364,19 +438,23 @@ static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs
 }
 
 int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace, size_t workspace_bytes,
-                      gws_multi_plan* plan_out, void* stream) {
+                      void* host_workspace, size_t host_workspace_bytes, gws_multi_plan* plan_out, void* stream) {
+  if (host_workspace == nullptr || host_workspace_bytes < gws_workspace_bytes(n)) return GWS_ERR_WORKSPACE;
   std::vector<char> image;
   gws_multi_plan plan;
   const int st = build_tables(n, descs, ptrs, workspace, workspace_bytes, &plan, image);
   if (st != GWS_OK) return st;
   if (!image.empty()) {
-    cudaError_t err = cudaMemcpyAsync(workspace, image.data(), image.size(), cudaMemcpyHostToDevice,
+    // The host copy stays with the plan: flat-group launches pass their records by value from it.
+    std::memcpy(host_workspace, image.data(), image.size());
+    cudaError_t err = cudaMemcpyAsync(workspace, host_workspace, image.size(), cudaMemcpyHostToDevice,
                                       static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return cuda_fail(err, "table upload");
-    // The upload reads pageable host memory that dies with this call: wait for it.
+    // The caller may reuse the stream at once and the host copy may be pageable: wait for the upload.
     err = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return cuda_fail(err, "table upload");
   }
+  plan.host_tables = host_workspace;
   *plan_out = plan;
   return GWS_OK;
 }
@@ -395,7 +473,7 @@ int64_t gws_multi_table_image(int n, const gws_desc* descs, const gws_multi_ptrs
 
 static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream, bool backward) {
   if (plan == nullptr) return GWS_ERR_NULL;
-  if (plan->workspace == nullptr) return GWS_ERR_WORKSPACE;
+  if (plan->workspace == nullptr || plan->host_tables == nullptr) return GWS_ERR_WORKSPACE;
   if (backward ? !plan->has_bwd : !plan->has_fwd) return GWS_ERR_NULL;
   const Entry none{};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -404,7 +482,12 @@ static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream, bo
     if (count == 0) continue;
     const Entry* table = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->workspace) +
                                                         (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
-    if (cls != gws::kGeneral) {
+    if (cls == gws::kFlat) {
+      const Entry* host = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
+                                                         (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
+      const int st = backward ? launch_flat<gws::kBwd>(host, count, step, s) : launch_flat<gws::kFwd>(host, count, step, s);
+      if (st != GWS_OK) return st;
+    } else if (cls != gws::kGeneral) {
       const int st = backward ? launch<gws::kBwd>(cls, none, table, count, plan->tiles[cls], step, s)
                               : launch<gws::kFwd>(cls, none, table, count, plan->tiles[cls], step, s);
       if (st != GWS_OK) return st;
@@ -419,6 +502,18 @@ static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream, bo
   return GWS_OK;
 }
 
+int gws_multi_launch_count(const gws_multi_plan* plan, int backward) {
+  if (plan == nullptr) return GWS_ERR_NULL;
+  if (plan->host_tables == nullptr) return GWS_ERR_WORKSPACE;
+  if (backward ? !plan->has_bwd : !plan->has_fwd) return 0;
+  const Entry* flat = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
+                                                     (backward ? plan->bwd_offset[0] : plan->fwd_offset[0]));
+  int wide = 0, narrow = 0;
+  for (int k = 0; k < plan->count[0]; ++k) (flat[k].lanes_log2 < 2u ? narrow : wide) += 1;
+  const int cap = gws::kFlatCapLarge;
+  return (wide + cap - 1) / cap + (narrow + cap - 1) / cap + (plan->count[1] ? 1 : 0) + (plan->count[2] ? 1 : 0) + plan->count[3];
+}
+
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
   return run_multi(plan, step, stream, false);
 }
@@ -430,7 +525,7 @@ int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream
 int gws_multi_locate_probe(const gws_multi_plan* plan, int backward, int kernel_class, const int64_t* tiles, int n_tiles,
                            uint64_t* out, void* stream) {
   if (plan == nullptr || tiles == nullptr || out == nullptr) return GWS_ERR_NULL;
-  if (kernel_class < 0 || kernel_class > 2 || n_tiles < 0) return GWS_ERR_SHAPE;
+  if (kernel_class < 1 || kernel_class > 2 || n_tiles < 0) return GWS_ERR_SHAPE;   // flat groups carry no device table
   if (plan->workspace == nullptr) return GWS_ERR_WORKSPACE;
   if (n_tiles == 0 || plan->count[kernel_class] == 0) return GWS_OK;
   const Entry* table = reinterpret_cast<const Entry*>(
@@ -565,6 +660,7 @@ int gws_sample_fwd_multi_static(int n, const gws_desc* descs, const gws_multi_pt
   const cudaError_t err = cudaMemcpyAsync(table, image.data(), image.size(), cudaMemcpyHostToDevice,
                                           static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return cuda_fail(err, "upload into the built-in table array");
+  plan.host_tables = image.data();   // lives until the launches below have copied their parameters
   return run_multi(&plan, step, stream, false);
 }
 

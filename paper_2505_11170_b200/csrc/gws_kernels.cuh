@@ -283,6 +283,35 @@ __global__ void k_locate_probe(const Entry* __restrict__ table, int n, const int
 // 32..256 elements are 1..8 neighbouring lanes (shuffle reduction); groups of 8 or 16 elements are
 // handled inside the thread.  Only those small groups can leave a last chunk partly filled.
 
+// One tensor of a flat-group launch.  The records travel BY VALUE in the kernel parameters (constant
+// bank): a thread block finds its tensor without touching global memory, which matters because a
+// block lives for only a few microseconds.  Pointer meanings as in Entry.
+struct FlatRec {
+  const void* in;
+  void* out;
+  const float* gin;
+  float* gout;
+  uint64_t vec0;        // elem_offset / 8: Philox counter of the tensor's first vector
+  uint64_t n_vec;
+  uint32_t seed_lo, seed_hi;
+  uint32_t lanes_log2;  // log2(vectors per group)
+  int32_t tile_begin;   // first tile of this tensor inside its launch
+};
+static_assert(sizeof(FlatRec) == 64, "FlatRec layout");
+constexpr int kFlatHint = 128;
+// hint[t >> hint_shift] is the record that owns tile (t >> hint_shift) << hint_shift; the owner of t
+// is that record or one a few places further on.
+template <int CAP>
+struct FlatBatch {
+  int32_t n;
+  uint32_t hint_shift;
+  uint32_t pad[2];
+  uint16_t hint[kFlatHint];
+  FlatRec e[CAP];
+};
+constexpr int kFlatCapSmall = 4, kFlatCapLarge = 240;   // 0.5 KiB and 15.3 KiB of parameters
+enum FlatVariant { kWide32 = 0, kWide16 = 1, kNarrow = 2 };
+
 struct Chunk {
   uint32_t x[16];
 };
@@ -320,7 +349,7 @@ __device__ __forceinline__ uint32_t absmax_words4(const uint32_t* x) { return ma
 
 // Groups of at least one chunk: `lanes` = chunks per group (1, 2, 4 or 8 neighbouring lanes).
 template <int MODE, bool USE32>
-__device__ __forceinline__ void flat_wide(const Entry& e, uint64_t chunk0, uint32_t lanes, uint32_t lanes_log2, uint32_t step_lo,
+__device__ __forceinline__ void flat_wide(const FlatRec& e, uint64_t chunk0, uint32_t lanes, uint32_t lanes_log2, uint32_t step_lo,
                                           uint32_t step_hi) {
   const uint64_t n_chunks = e.n_vec >> 2;
   const bool ok = chunk0 < n_chunks;
@@ -329,7 +358,7 @@ __device__ __forceinline__ void flat_wide(const Entry& e, uint64_t chunk0, uint3
   const uint64_t g = chunk >> lanes_log2;
   const float gv = (MODE != kAbsmax) ? ld_f32(e.gin, g) : 0.0f;
   const bool writer = ok && (threadIdx.x & (lanes - 1u)) == 0u;
-  const uint64_t v0 = (e.elem_offset >> 3) + chunk * 4u;
+  const uint64_t v0 = e.vec0 + chunk * 4u;
 
   if (MODE == kBwd) {
     float acc = 0.0f;
@@ -368,12 +397,12 @@ __device__ __forceinline__ void flat_wide(const Entry& e, uint64_t chunk0, uint3
 
 // Groups of one or two vectors (8 or 16 elements): 4 or 2 groups inside the thread's chunk.
 template <int MODE>
-__device__ __forceinline__ void flat_narrow(const Entry& e, uint64_t chunk, uint32_t ll, uint32_t step_lo, uint32_t step_hi) {
+__device__ __forceinline__ void flat_narrow(const FlatRec& e, uint64_t chunk, uint32_t ll, uint32_t step_lo, uint32_t step_hi) {
   const uint64_t first = chunk * 4u;
   if (first >= e.n_vec) return;
   const uint32_t n_valid = static_cast<uint32_t>(min(static_cast<uint64_t>(4), e.n_vec - first));
   const Chunk c = load_chunk<false>(e.in, chunk, n_valid);
-  const uint64_t v0 = (e.elem_offset >> 3) + first;
+  const uint64_t v0 = e.vec0 + first;
   Chunk y;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
@@ -410,21 +439,21 @@ __device__ __forceinline__ void flat_narrow(const Entry& e, uint64_t chunk, uint
   if (MODE == kBwd && e.out != nullptr) store_chunk<false>(e.out, chunk, n_valid, c);
 }
 
-template <int MODE, bool MULTI>
-__global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ Entry single,
-                                                       const Entry* __restrict__ table, int n, uint32_t step_lo,
-                                                       uint32_t step_hi) {
-  GWS_RESOLVE_ENTRY(e, tile)
-  const uint32_t ll = e.lanes_log2;   // log2(vectors per group)
-  const uint64_t chunk = static_cast<uint64_t>(tile) * kFlatThreads + threadIdx.x;
-  if (ll < 2u) {
-    flat_narrow<MODE>(e, chunk, ll, step_lo, step_hi);
-    return;
+// VARIANT: kWide32 / kWide16 = groups of 32..256 elements with 32-byte / 16-byte accesses (the
+// former needs every tensor pointer of the launch 32-byte aligned); kNarrow = groups of 8 or 16.
+template <int MODE, int VARIANT, int CAP>
+__global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ FlatBatch<CAP> b, uint32_t step_lo, uint32_t step_hi) {
+  const int32_t tile = static_cast<int32_t>(blockIdx.x);
+  int idx = b.hint[tile >> b.hint_shift];
+  while (idx + 1 < b.n && b.e[idx + 1].tile_begin <= tile) ++idx;
+  const FlatRec& e = b.e[idx];
+  const uint64_t chunk = static_cast<uint64_t>(tile - e.tile_begin) * kFlatThreads + threadIdx.x;
+  if (VARIANT == kNarrow) {
+    flat_narrow<MODE>(e, chunk, e.lanes_log2, step_lo, step_hi);
+  } else {
+    const uint32_t lanes_log2 = e.lanes_log2 - 2u;
+    flat_wide<MODE, VARIANT == kWide32>(e, chunk, 1u << lanes_log2, lanes_log2, step_lo, step_hi);
   }
-  const uint32_t lanes_log2 = ll - 2u, lanes = 1u << lanes_log2;
-  const bool use32 = ((reinterpret_cast<uintptr_t>(e.in) | reinterpret_cast<uintptr_t>(e.out)) & 31u) == 0u;
-  if (use32) flat_wide<MODE, true>(e, chunk, lanes, lanes_log2, step_lo, step_hi);
-  else flat_wide<MODE, false>(e, chunk, lanes, lanes_log2, step_lo, step_hi);
 }
 
 // ---- one warp per row ---------------------------------------------------------------------------

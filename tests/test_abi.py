@@ -74,14 +74,17 @@ def test_validation_happens_before_any_launch(lib):
     plan = binding._MultiPlan()
     ptrs = binding._MultiPtrs()
     d = (Desc * 1)(good)
-    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), fake, 1 << 20, ctypes.byref(plan), null) == binding.ERR_NULL
+    hostws = ctypes.create_string_buffer(1 << 20)
+    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), fake, 1 << 20, hostws, 1 << 20, ctypes.byref(plan), null) == binding.ERR_NULL
     arr = (ctypes.c_void_p * 1)(0x2000)
     out = (ctypes.c_void_p * 1)(0x9000)
     pp = ctypes.POINTER(ctypes.c_void_p)
     ptrs = binding._MultiPtrs(ctypes.cast(arr, pp), ctypes.cast(arr, pp), ctypes.cast(out, pp), None, None, None, None)
-    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), null, 1 << 20, ctypes.byref(plan), null) == binding.ERR_WORKSPACE
-    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), ctypes.c_void_p(0x10010), 1 << 20, ctypes.byref(plan), null) == binding.ERR_WORKSPACE
-    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), ctypes.c_void_p(0x10000), 8, ctypes.byref(plan), null) == binding.ERR_WORKSPACE
+    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), null, 1 << 20, hostws, 1 << 20, ctypes.byref(plan), null) == binding.ERR_WORKSPACE
+    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), ctypes.c_void_p(0x10010), 1 << 20, hostws, 1 << 20, ctypes.byref(plan), null) == binding.ERR_WORKSPACE
+    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), ctypes.c_void_p(0x10000), 8, hostws, 1 << 20, ctypes.byref(plan), null) == binding.ERR_WORKSPACE
+    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), ctypes.c_void_p(0x10000), 1 << 20, null, 1 << 20, ctypes.byref(plan), null) == binding.ERR_WORKSPACE
+    assert L.gws_multi_prepare(1, d, ctypes.byref(ptrs), ctypes.c_void_p(0x10000), 1 << 20, hostws, 8, ctypes.byref(plan), null) == binding.ERR_WORKSPACE
     assert L.gws_workspace_bytes(154) >= 154 * 2 * 112
     assert L.gws_sample_fwd_multi(None, 0, null) == binding.ERR_NULL
 
