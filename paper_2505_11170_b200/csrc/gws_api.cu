@@ -67,7 +67,10 @@ int classify(const gws_desc* d, bool vec_ok) {
   const int64_t gc = resolved_group_cols(d);
   const bool dense = vec_ok && d->ld == d->cols && d->cols % 8 == 0 && d->group_rows == 1;
   if (!dense) return gws::kGeneral;
-  if (gc <= 256 && gc >= 8 && (gc & (gc - 1)) == 0 && d->cols % gc == 0) return gws::kFlat;
+  // flat kernels keep the high word of the Philox counter uniform: the tensor's vectors must not straddle 2^32
+  const uint64_t first_vec = d->elem_offset >> 3, last_vec = first_vec + static_cast<uint64_t>(d->rows * d->cols / 8) - 1;
+  const bool uniform_hi = (first_vec >> 32) == (last_vec >> 32) && (last_vec - first_vec) < 0xFFFFFFFFull;
+  if (gc <= 256 && gc >= 8 && (gc & (gc - 1)) == 0 && d->cols % gc == 0 && uniform_hi) return gws::kFlat;
   if (gc == d->cols) {
     const int64_t vpr = d->cols / 8;
     if (vpr <= 32 * gws::kRowWarpVecs) return gws::kRowWarp;
@@ -129,10 +132,11 @@ gws::FlatRec to_flat_rec(const Entry& e) {
   r.out = e.out;
   r.gin = e.gin;
   r.gout = e.gout;
-  r.vec0 = e.elem_offset >> 3;
-  r.n_vec = e.n_vec;
-  r.seed_lo = e.seed_lo;
-  r.seed_hi = e.seed_hi;
+  r.vec_lo = static_cast<uint32_t>(e.elem_offset >> 3);
+  r.vec_hi = static_cast<uint32_t>(e.elem_offset >> 35);
+  r.n_vec = static_cast<uint32_t>(e.n_vec);   // classify() keeps tensors of 2^32 vectors or more out of this class
+  r.k0 = e.seed_lo;
+  r.k1 = e.seed_hi;
   r.lanes_log2 = e.lanes_log2;
   return r;
 }
@@ -150,6 +154,7 @@ int launch_flat_batch(gws::FlatRec* recs, int count, uint32_t lo, uint32_t hi, c
   for (int k = 0; k < count; ++k) {
     b.e[k] = recs[k];
     b.e[k].tile_begin = static_cast<int32_t>(tiles);
+    b.e[k].pre = gws::philox_pre(recs[k].vec_hi, lo, hi, recs[k].k0, recs[k].k1);
     tiles += flat_tiles_of(recs[k]);
     if (tiles > kMaxGrid) return GWS_ERR_LIMIT;
   }

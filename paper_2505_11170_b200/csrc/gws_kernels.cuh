@@ -291,13 +291,15 @@ struct FlatRec {
   void* out;
   const float* gin;
   float* gout;
-  uint64_t vec0;        // elem_offset / 8: Philox counter of the tensor's first vector
-  uint64_t n_vec;
-  uint32_t seed_lo, seed_hi;
-  uint32_t lanes_log2;  // log2(vectors per group)
-  int32_t tile_begin;   // first tile of this tensor inside its launch
+  uint32_t vec_lo, vec_hi;  // elem_offset / 8: Philox counter of the first vector; vec_hi is the same for every vector
+  uint32_t n_vec;
+  uint32_t lanes_log2;      // log2(vectors per group)
+  int32_t tile_begin;       // first tile of this tensor inside its launch
+  uint32_t k0, k1;          // seed
+  PhiloxPre pre;            // the step- and seed-dependent constants of the first two Philox rounds
+  uint32_t pad;
 };
-static_assert(sizeof(FlatRec) == 64, "FlatRec layout");
+static_assert(sizeof(FlatRec) == 80, "FlatRec layout");
 constexpr int kFlatHint = 128;
 // hint[t >> hint_shift] is the record that owns tile (t >> hint_shift) << hint_shift; the owner of t
 // is that record or one a few places further on.
@@ -309,7 +311,7 @@ struct FlatBatch {
   uint16_t hint[kFlatHint];
   FlatRec e[CAP];
 };
-constexpr int kFlatCapSmall = 4, kFlatCapLarge = 240;   // 0.5 KiB and 15.3 KiB of parameters
+constexpr int kFlatCapSmall = 4, kFlatCapLarge = 192;   // 0.6 KiB and 15.3 KiB of parameters
 enum FlatVariant { kWide32 = 0, kWide16 = 1, kNarrow = 2 };
 
 struct Chunk {
@@ -349,22 +351,22 @@ __device__ __forceinline__ uint32_t absmax_words4(const uint32_t* x) { return ma
 
 // Groups of at least one chunk: `lanes` = chunks per group (1, 2, 4 or 8 neighbouring lanes).
 template <int MODE, bool USE32>
-__device__ __forceinline__ void flat_wide(const FlatRec& e, uint64_t chunk0, uint32_t lanes, uint32_t lanes_log2, uint32_t step_lo,
+__device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t chunk0, uint32_t lanes, uint32_t lanes_log2, uint32_t step_lo,
                                           uint32_t step_hi) {
-  const uint64_t n_chunks = e.n_vec >> 2;
+  const uint32_t n_chunks = e.n_vec >> 2;
   const bool ok = chunk0 < n_chunks;
-  const uint64_t chunk = ok ? chunk0 : n_chunks - 1;   // keeps the warp whole for the shuffles
+  const uint32_t chunk = ok ? chunk0 : n_chunks - 1u;  // keeps the warp whole for the shuffles
   const Chunk c = load_chunk<USE32>(e.in, chunk, 4);
-  const uint64_t g = chunk >> lanes_log2;
+  const uint32_t g = chunk >> lanes_log2;
   const float gv = (MODE != kAbsmax) ? ld_f32(e.gin, g) : 0.0f;
   const bool writer = ok && (threadIdx.x & (lanes - 1u)) == 0u;
-  const uint64_t v0 = e.vec0 + chunk * 4u;
+  const uint32_t v0 = e.vec_lo + chunk * 4u;
 
   if (MODE == kBwd) {
     float acc = 0.0f;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const Words4 r = philox_for_vector(v0 + k, step_lo, step_hi, e.seed_lo, e.seed_hi);
+      const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
       acc = dot_vec(make_uint4(c.x[4 * k], c.x[4 * k + 1], c.x[4 * k + 2], c.x[4 * k + 3]), r, acc);
     }
     for (uint32_t o = 1; o < lanes; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
@@ -383,7 +385,7 @@ __device__ __forceinline__ void flat_wide(const FlatRec& e, uint64_t chunk0, uin
   Chunk y;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    const Words4 r = philox_for_vector(v0 + k, step_lo, step_hi, e.seed_lo, e.seed_hi);
+    const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
     uint32_t p[4];
     decode8(r, p);
 #pragma unroll
@@ -397,26 +399,26 @@ __device__ __forceinline__ void flat_wide(const FlatRec& e, uint64_t chunk0, uin
 
 // Groups of one or two vectors (8 or 16 elements): 4 or 2 groups inside the thread's chunk.
 template <int MODE>
-__device__ __forceinline__ void flat_narrow(const FlatRec& e, uint64_t chunk, uint32_t ll, uint32_t step_lo, uint32_t step_hi) {
-  const uint64_t first = chunk * 4u;
-  if (first >= e.n_vec) return;
-  const uint32_t n_valid = static_cast<uint32_t>(min(static_cast<uint64_t>(4), e.n_vec - first));
+__device__ __forceinline__ void flat_narrow(const FlatRec& e, uint32_t chunk, uint32_t ll, uint32_t step_lo, uint32_t step_hi) {
+  if (chunk > (e.n_vec - 1u) >> 2) return;
+  const uint32_t first = chunk * 4u;
+  const uint32_t n_valid = min(4u, e.n_vec - first);
   const Chunk c = load_chunk<false>(e.in, chunk, n_valid);
-  const uint64_t v0 = e.vec0 + first;
+  const uint32_t v0 = e.vec_lo + first;
   Chunk y;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     if (static_cast<uint32_t>(k) >= n_valid) break;
-    const uint64_t g = (first + k) >> ll;
+    const uint32_t g = (first + k) >> ll;
     const bool writer = ll == 0u || (k & 1) == 0;
     const uint4 xv = make_uint4(c.x[4 * k], c.x[4 * k + 1], c.x[4 * k + 2], c.x[4 * k + 3]);
     const int mate = k ^ 1;   // the other vector of a two-vector group (always inside the chunk)
-    const Words4 r = philox_for_vector(v0 + k, step_lo, step_hi, e.seed_lo, e.seed_hi);
+    const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
     if (MODE == kBwd) {
       if (writer) {
         float acc = dot_vec(xv, r, 0.0f);
         if (ll == 1u) {
-          const Words4 r2 = philox_for_vector(v0 + mate, step_lo, step_hi, e.seed_lo, e.seed_hi);
+          const Words4 r2 = philox4x32_10_pre(v0 + mate, e.k0, e.k1, e.pre);
           acc = dot_vec(make_uint4(c.x[4 * mate], c.x[4 * mate + 1], c.x[4 * mate + 2], c.x[4 * mate + 3]), r2, acc);
         }
         st_f32(e.gout, g, grad_bt_of(ld_f32(e.gin, g), acc));
@@ -447,7 +449,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ F
   int idx = b.hint[tile >> b.hint_shift];
   while (idx + 1 < b.n && b.e[idx + 1].tile_begin <= tile) ++idx;
   const FlatRec& e = b.e[idx];
-  const uint64_t chunk = static_cast<uint64_t>(tile - e.tile_begin) * kFlatThreads + threadIdx.x;
+  const uint32_t chunk = static_cast<uint32_t>(tile - e.tile_begin) * kFlatThreads + threadIdx.x;
   if (VARIANT == kNarrow) {
     flat_narrow<MODE>(e, chunk, e.lanes_log2, step_lo, step_hi);
   } else {

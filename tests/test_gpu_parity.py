@@ -208,6 +208,31 @@ def test_elem_offset_reproduces_the_unsharded_tensor():
     assert (part == full[half:]).all()
 
 
+@pytest.mark.parametrize("offset,group_cols,want_class", [
+    ((1 << 35) + 8 * 40, 128, 0),          # high counter word 1 for every vector: flat kernel
+    ((5 << 35) + 8 * 12, 16, 0),           # narrow groups, high word 5
+    ((1 << 35) - 8 * 1000, 128, 3),        # the vectors straddle 2^32: not a flat-kernel tensor
+    ((1 << 35) - 8 * 1000, 0, 1),          # whole-row groups keep their 64-bit counters
+    (((1 << 64) - (1 << 40)) & ~7, 32, 0),  # the top of the index range
+])
+def test_large_element_offsets(offset, group_cols, want_class, step=(1 << 40) + 3, seed=0xF00DFACE12345678):
+    rows, cols = 48, 512
+    d = Desc.make(rows, cols, 1, group_cols, seed=seed, step=step, elem_offset=offset)
+    assert gws.kernel_class(d) == want_class
+    w, g = _make(rows, cols, None, 21), _make(rows, cols, None, 22, sigma=1e-4)
+    bt = _bt(gws.n_groups(d), seed=5)
+    w_hat, scale = gws.sample_fwd(d, w.to(DEV), bt.to(DEV))
+    _, gbt = gws.sample_bwd(d, g.to(DEV), scale)
+    want_hat, want_sc = orc.sample_fwd(bits_of(w), bt.numpy(), rows, cols, 1, group_cols, seed=seed, step=step, elem_offset=offset)
+    _, want_gbt = orc.sample_bwd(bits_of(g), want_sc, rows, cols, 1, group_cols, seed=seed, step=step, elem_offset=offset)
+    assert (bits_of(w_hat).ravel() == want_hat).all()
+    assert (scale.cpu().numpy().view(np.uint32) == want_sc.view(np.uint32)).all()
+    err = np.abs(gbt.cpu().numpy().astype(np.float64) - want_gbt)
+    assert err.max() <= 1e-5 * np.abs(want_gbt).max()
+    packed = gws.noise(d).cpu().numpy().view(np.uint32)
+    assert (packed == orc.noise_packed(seed, step, offset, rows * cols)).all()
+
+
 def test_steps_and_seeds_give_different_noise_and_same_step_repeats():
     rows, cols = 32, 1024
     w = _make(rows, cols, None, 9).to(DEV)
