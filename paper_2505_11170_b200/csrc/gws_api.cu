@@ -8,6 +8,12 @@
 #include <vector>
 
 #include "gws.h"
+#ifndef GWS_FLAT_CPT_FWD
+#define GWS_FLAT_CPT_FWD 2
+#endif
+#ifndef GWS_FLAT_CPT_BWD
+#define GWS_FLAT_CPT_BWD 2
+#endif
 #include "gws_kernels.cuh"
 
 namespace {
@@ -141,32 +147,21 @@ gws::FlatRec to_flat_rec(const Entry& e) {
   return r;
 }
 
-int64_t flat_tiles_of(const gws::FlatRec& r) {
-  const int64_t per = static_cast<int64_t>(gws::kFlatThreads) * gws::kFlatVecs;
-  return (static_cast<int64_t>(r.n_vec) + per - 1) / per;
+// Chunks (64 bytes) a thread handles in each mode.
+template <int MODE, int VARIANT>
+constexpr int flat_cpt() {
+  return VARIANT == gws::kNarrow ? 1 : (MODE == gws::kFwd ? GWS_FLAT_CPT_FWD : GWS_FLAT_CPT_BWD);
 }
 
 template <int MODE, int VARIANT, int CAP>
 int launch_flat_batch(gws::FlatRec* recs, int count, uint32_t lo, uint32_t hi, cudaStream_t stream) {
+  constexpr int CPT = flat_cpt<MODE, VARIANT>();
   gws::FlatBatch<CAP> b;
   std::memset(&b, 0, sizeof b);
-  int64_t tiles = 0;
-  for (int k = 0; k < count; ++k) {
-    b.e[k] = recs[k];
-    b.e[k].tile_begin = static_cast<int32_t>(tiles);
-    b.e[k].pre = gws::philox_pre(recs[k].vec_hi, lo, hi, recs[k].k0, recs[k].k1);
-    tiles += flat_tiles_of(recs[k]);
-    if (tiles > kMaxGrid) return GWS_ERR_LIMIT;
-  }
-  b.n = count;
-  while (((tiles - 1) >> b.hint_shift) >= gws::kFlatHint) ++b.hint_shift;
-  int owner = 0;
-  for (int h = 0; h < gws::kFlatHint; ++h) {
-    const int64_t t = static_cast<int64_t>(h) << b.hint_shift;
-    while (owner + 1 < count && b.e[owner + 1].tile_begin <= t) ++owner;
-    b.hint[h] = static_cast<uint16_t>(owner);
-  }
-  gws::k_flat<MODE, VARIANT, CAP><<<static_cast<unsigned>(tiles), gws::kFlatThreads, 0, stream>>>(b, lo, hi);
+  const int64_t tiles = gws::fill_flat_batch<CAP>(b, recs, count, CPT, lo, hi);
+  if (tiles < 0) return GWS_ERR_LIMIT;
+  if (tiles == 0) return GWS_OK;
+  gws::k_flat<MODE, VARIANT, CAP, CPT><<<static_cast<unsigned>(tiles), gws::kFlatThreads, 0, stream>>>(b);
   return check_launch("flat-group kernel");
 }
 

@@ -350,56 +350,68 @@ __device__ __forceinline__ void store_chunk(void* base, uint64_t chunk, uint32_t
 __device__ __forceinline__ uint32_t absmax_words4(const uint32_t* x) { return maxabs2(maxabs2(x[0], x[1]), maxabs2(x[2], x[3])); }
 
 // Groups of at least one chunk: `lanes` = chunks per group (1, 2, 4 or 8 neighbouring lanes).
-template <int MODE, bool USE32>
-__device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t chunk0, uint32_t lanes, uint32_t lanes_log2, uint32_t step_lo,
-                                          uint32_t step_hi) {
+// A thread handles CPT chunks, 256 chunks apart, all loaded before the first is used.
+template <int MODE, bool USE32, int CPT>
+__device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t first_chunk, uint32_t lanes, uint32_t lanes_log2) {
   const uint32_t n_chunks = e.n_vec >> 2;
-  const bool ok = chunk0 < n_chunks;
-  const uint32_t chunk = ok ? chunk0 : n_chunks - 1u;  // keeps the warp whole for the shuffles
-  const Chunk c = load_chunk<USE32>(e.in, chunk, 4);
-  const uint32_t g = chunk >> lanes_log2;
-  const float gv = (MODE != kAbsmax) ? ld_f32(e.gin, g) : 0.0f;
-  const bool writer = ok && (threadIdx.x & (lanes - 1u)) == 0u;
-  const uint32_t v0 = e.vec_lo + chunk * 4u;
-
-  if (MODE == kBwd) {
-    float acc = 0.0f;
+  const bool writer_lane = (threadIdx.x & (lanes - 1u)) == 0u;
+  uint32_t chunk[CPT];
+  bool ok[CPT];
+  Chunk c[CPT];
+  float gv[CPT];
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    const uint32_t chunk0 = first_chunk + static_cast<uint32_t>(i) * kFlatThreads;
+    ok[i] = chunk0 < n_chunks;
+    chunk[i] = ok[i] ? chunk0 : n_chunks - 1u;   // keeps the warp whole for the shuffles
+    c[i] = load_chunk<USE32>(e.in, chunk[i], 4);
+    gv[i] = (MODE != kAbsmax) ? ld_f32(e.gin, chunk[i] >> lanes_log2) : 0.0f;
+  }
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    const uint32_t g = chunk[i] >> lanes_log2;
+    const bool writer = ok[i] && writer_lane;
+    const uint32_t v0 = e.vec_lo + chunk[i] * 4u;
+    if (MODE == kBwd) {
+      float acc = 0.0f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
+        acc = dot_vec(make_uint4(c[i].x[4 * k], c[i].x[4 * k + 1], c[i].x[4 * k + 2], c[i].x[4 * k + 3]), r, acc);
+      }
+      for (uint32_t o = 1; o < lanes; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+      if (writer) st_f32(e.gout, g, grad_bt_of(gv[i], acc));
+      if (ok[i] && e.out != nullptr) store_chunk<USE32>(e.out, chunk[i], 4, c[i]);
+      continue;
+    }
+    uint32_t m = maxabs2(maxabs2(absmax_words4(c[i].x), absmax_words4(c[i].x + 4)),
+                         maxabs2(absmax_words4(c[i].x + 8), absmax_words4(c[i].x + 12)));
+    for (uint32_t o = 1; o < lanes; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    const float a = absmax_finish(m);
+    if (MODE == kAbsmax) {
+      if (writer) st_f32(e.gout, g, a);
+      continue;
+    }
+    const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv[i])));
+    Chunk y;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
-      acc = dot_vec(make_uint4(c.x[4 * k], c.x[4 * k + 1], c.x[4 * k + 2], c.x[4 * k + 3]), r, acc);
+      uint32_t p[4];
+      decode8(r, p);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) y.x[4 * k + j] = sample_pair(c[i].x[4 * k + j], p[j], sc);
     }
-    for (uint32_t o = 1; o < lanes; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-    if (writer) st_f32(e.gout, g, grad_bt_of(gv, acc));
-    if (ok && e.out != nullptr) store_chunk<USE32>(e.out, chunk, 4, c);
-    return;
-  }
-  uint32_t m = maxabs2(maxabs2(absmax_words4(c.x), absmax_words4(c.x + 4)), maxabs2(absmax_words4(c.x + 8), absmax_words4(c.x + 12)));
-  for (uint32_t o = 1; o < lanes; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-  const float a = absmax_finish(m);
-  if (MODE == kAbsmax) {
-    if (writer) st_f32(e.gout, g, a);
-    return;
-  }
-  const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv)));
-  Chunk y;
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
-    uint32_t p[4];
-    decode8(r, p);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) y.x[4 * k + j] = sample_pair(c.x[4 * k + j], p[j], sc);
-  }
-  if (ok) {
-    store_chunk<USE32>(e.out, chunk, 4, y);
-    if (writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
+    if (ok[i]) {
+      store_chunk<USE32>(e.out, chunk[i], 4, y);
+      if (writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
+    }
   }
 }
 
 // Groups of one or two vectors (8 or 16 elements): 4 or 2 groups inside the thread's chunk.
 template <int MODE>
-__device__ __forceinline__ void flat_narrow(const FlatRec& e, uint32_t chunk, uint32_t ll, uint32_t step_lo, uint32_t step_hi) {
+__device__ __forceinline__ void flat_narrow(const FlatRec& e, uint32_t chunk, uint32_t ll) {
   if (chunk > (e.n_vec - 1u) >> 2) return;
   const uint32_t first = chunk * 4u;
   const uint32_t n_valid = min(4u, e.n_vec - first);
@@ -443,19 +455,46 @@ __device__ __forceinline__ void flat_narrow(const FlatRec& e, uint32_t chunk, ui
 
 // VARIANT: kWide32 / kWide16 = groups of 32..256 elements with 32-byte / 16-byte accesses (the
 // former needs every tensor pointer of the launch 32-byte aligned); kNarrow = groups of 8 or 16.
-template <int MODE, int VARIANT, int CAP>
-__global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ FlatBatch<CAP> b, uint32_t step_lo, uint32_t step_hi) {
+// A tile is 256 threads x CPT chunks (CPT = 1 for narrow groups).
+template <int MODE, int VARIANT, int CAP, int CPT>
+__global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ FlatBatch<CAP> b) {
   const int32_t tile = static_cast<int32_t>(blockIdx.x);
   int idx = b.hint[tile >> b.hint_shift];
   while (idx + 1 < b.n && b.e[idx + 1].tile_begin <= tile) ++idx;
   const FlatRec& e = b.e[idx];
-  const uint32_t chunk = static_cast<uint32_t>(tile - e.tile_begin) * kFlatThreads + threadIdx.x;
+  const uint32_t chunk = static_cast<uint32_t>(tile - e.tile_begin) * (kFlatThreads * CPT) + threadIdx.x;
   if (VARIANT == kNarrow) {
-    flat_narrow<MODE>(e, chunk, e.lanes_log2, step_lo, step_hi);
+    flat_narrow<MODE>(e, chunk, e.lanes_log2);
   } else {
     const uint32_t lanes_log2 = e.lanes_log2 - 2u;
-    flat_wide<MODE, VARIANT == kWide32>(e, chunk, 1u << lanes_log2, lanes_log2, step_lo, step_hi);
+    flat_wide<MODE, VARIANT == kWide32, CPT>(e, chunk, 1u << lanes_log2, lanes_log2);
   }
+}
+
+// Host side: copies `count` records into a parameter block for the pass of gradient-update counter
+// (step_lo, step_hi), numbers their tiles and builds the tile hint.  Returns the number of tiles.
+template <int CAP>
+inline int64_t fill_flat_batch(FlatBatch<CAP>& b, const FlatRec* recs, int count, int chunks_per_thread, uint32_t step_lo,
+                               uint32_t step_hi) {
+  b.n = count;
+  b.hint_shift = 0;
+  const int64_t per_tile = static_cast<int64_t>(kFlatThreads) * 4 * chunks_per_thread;   // vectors
+  int64_t tiles = 0;
+  for (int k = 0; k < count; ++k) {
+    b.e[k] = recs[k];
+    b.e[k].tile_begin = static_cast<int32_t>(tiles);
+    b.e[k].pre = philox_pre(recs[k].vec_hi, step_lo, step_hi, recs[k].k0, recs[k].k1);
+    tiles += (static_cast<int64_t>(recs[k].n_vec) + per_tile - 1) / per_tile;
+    if (tiles > 2147483647LL) return -1;
+  }
+  while (tiles > 0 && ((tiles - 1) >> b.hint_shift) >= kFlatHint) ++b.hint_shift;
+  int owner = 0;
+  for (int h = 0; h < kFlatHint; ++h) {
+    const int64_t t = static_cast<int64_t>(h) << b.hint_shift;
+    while (owner + 1 < count && b.e[owner + 1].tile_begin <= t) ++owner;
+    b.hint[h] = static_cast<uint16_t>(owner);
+  }
+  return tiles;
 }
 
 // ---- one warp per row ---------------------------------------------------------------------------
