@@ -42,12 +42,32 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+PROFILE = os.path.join(ROOT, "profiles", "k_flat_llama2_1b_g128.md")
+KERNEL_SOURCES = [os.path.join(ROOT, "paper_2505_11170_b200", "csrc", f) for f in ("gws_api.cu", "gws_kernels.cuh", "gws_math.cuh")]
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for path in KERNEL_SOURCES:
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
 def ncu_traffic():
-    """Per-launch DRAM bytes of the forward kernel from the committed ncu summary, if there is one."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(path):
-        with open(path) as f:
-            return json.load(f)
+    """Per-launch DRAM bytes from the committed ncu summary: its line
+    ``bench: fwd_bytes_per_launch=<n> bwd_bytes_per_launch=<n> sources=<hash>``.
+    Empty (traffic null) if there is no summary or the kernel sources changed since the counters were taken."""
+    if not os.path.exists(PROFILE):
+        return {}
+    with open(PROFILE) as f:
+        for line in f:
+            if line.startswith("bench:"):
+                kv = dict(item.split("=", 1) for item in line.split()[1:])
+                if kv.get("sources") != kernel_source_hash():
+                    return {}
+                return {k: int(v) for k, v in kv.items() if k.endswith("_bytes_per_launch")}
     return {}
 
 
@@ -61,7 +81,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -164,15 +184,24 @@ def cpu_baseline(specs):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 400; 3 for --impl reference)")
+    ap.add_argument("--warmup", type=int, default=None, help="untimed steps (default 5, at least 3; 1 for --impl reference)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--blocks", type=int, default=22, help="Llama blocks in the set (22 = the full workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--source-hash", action="store_true", help="print the hash an ncu summary records with its counters")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "ours":
+        args.steps = 400 if args.steps is None else args.steps            # ~0.55 s of device time at N = 1
+        args.warmup = 5 if args.warmup is None else max(args.warmup, 3)
+    else:
+        args.steps = 3 if args.steps is None else args.steps              # ~2.4 s of CPU time per step
+        args.warmup = 1 if args.warmup is None else args.warmup
 
+    if args.source_hash:
+        print(kernel_source_hash())
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
