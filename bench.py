@@ -184,7 +184,7 @@ def cpu_baseline(specs):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 400; 3 for --impl reference)")
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 100; 3 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=None, help="untimed steps (default 5, at least 3; 1 for --impl reference)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--blocks", type=int, default=22, help="Llama blocks in the set (22 = the full workload)")
@@ -193,7 +193,7 @@ def main():
     ap.add_argument("--source-hash", action="store_true", help="print the hash an ncu summary records with its counters")
     args = ap.parse_args()
     if args.impl == "ours":
-        args.steps = 400 if args.steps is None else args.steps            # ~0.55 s of device time at N = 1
+        args.steps = 100 if args.steps is None else args.steps            # ~0.15 s of device time at N = 1
         args.warmup = 5 if args.warmup is None else max(args.warmup, 3)
     else:
         args.steps = 3 if args.steps is None else args.steps              # ~2.4 s of CPU time per step
