@@ -71,6 +71,20 @@ def ncu_traffic():
     return {}
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of per-rank numbers over all ranks (the values themselves if not distributed)."""
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def whole_job_throughput(units_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Units per second of the whole job: every rank processes ``units_per_rank`` per step (replicas, weak scaling)
+    and a step takes as long as the slowest rank."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -268,14 +282,11 @@ def main():
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     fwd_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
     bwd_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
-    t = torch.tensor([total_ms, fwd_ms, bwd_ms], device=dev, dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, fwd_ms, bwd_ms = (float(x) for x in t.tolist())
+    total_ms, fwd_ms, bwd_ms = max_over_ranks([total_ms, fwd_ms, bwd_ms], dist, dev)
     ms_per_step = total_ms / args.steps
     bytes_per_step = n_elem * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM)
-    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
-    gelem = world * n_elem / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_throughput(bytes_per_step, world, ms_per_step) / 1e9
+    gelem = whole_job_throughput(n_elem, world, ms_per_step) / 1e9
 
     # ---- end to end through the host-buffer entry point: pinned host tensors in, results out ----
     e2e = None
@@ -302,11 +313,9 @@ def main():
             host_step(1 + k)
         e1.record(stream)
         barrier()
-        e2e_ms = torch.tensor([e0.elapsed_time(e1) / e2e_steps], device=dev, dtype=torch.float64)
-        if dist is not None:
-            dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+        e2e_ms = max_over_ranks([e0.elapsed_time(e1) / e2e_steps], dist, dev)[0]
         n_groups = sum(s.n_groups for s in specs)
-        e2e = {"value": world * bytes_per_step / (float(e2e_ms) * 1e-3) / 1e9, "unit": "GB/s",
+        e2e = {"value": whole_job_throughput(bytes_per_step, world, e2e_ms) / 1e9, "unit": "GB/s",
                "h2d_bytes_per_step": int(n_elem * 4 + n_groups * 4), "d2h_bytes_per_step": int(n_elem * 2 + n_groups * 8),
                "ms_per_step": float(e2e_ms), "steps": e2e_steps,
                "note": "gws_sample_step_host per tensor; pinned host buffers of one transformer block reused for all 22"}
