@@ -191,9 +191,11 @@ int64_t gws_multi_table_image(int n, const gws_desc* descs, const gws_multi_ptrs
 int gws_multi_locate_probe(const gws_multi_plan* plan, int backward, int kernel_class, const int64_t* tiles,
                            int n_tiles, uint64_t* out, void* stream);
 
-/* Kernel launches one forward (backward != 0: backward) pass of the plan enqueues: one per kernel
- * class in use, one more if groups of 8 / 16 elements occur beside wider flat groups, one per 240
- * flat-group tensors beyond the first 240, one per general-class tensor. */
+/* Kernel launches one forward (backward != 0: backward) pass of the plan enqueues.  Tensors that share
+ * a kernel share a launch (up to 192 flat-group or 168 whole-row tensors each): flat groups of 32..256
+ * elements; flat groups of 8 / 16; rows up to 4096 elements; rows up to 32768 elements.  Whole-row
+ * tensors whose rows are not a multiple of 32 elements, are longer, or are not 32-byte aligned, and
+ * general-class tensors, take one launch each. */
 int gws_multi_launch_count(const gws_multi_plan* plan, int backward);
 
 /* Forward / backward of every tensor of the plan for gradient-update counter `step`. */

@@ -195,6 +195,95 @@ int launch_flat(const Entry* entries, int count, uint64_t step, cudaStream_t str
   return launch_flat_variant<MODE, gws::kNarrow>(narrow, lo, hi, stream);
 }
 
+// ---- whole-row launches on chunks -------------------------------------------------------------------
+
+// The chunk kernel takes rows of a multiple of 32 elements up to 32768, 32-byte aligned, whose Philox
+// counters share one high word; everything else of the row classes runs on the vector kernels.
+bool row_chunk_eligible(const Entry& e) {
+  if (e.cols % 32 != 0 || e.cols > 32768 || e.ld != e.cols || e.group_rows != 1 || e.group_cols != e.cols) return false;
+  if (!aligned(e.in, 32) || !aligned(e.out, 32)) return false;
+  const uint64_t first = e.elem_offset >> 3, last = first + e.n_vec - 1;
+  return (first >> 32) == (last >> 32) && (last - first) < 0xFFFFFFFFull;
+}
+
+gws::RowRec to_row_rec(const Entry& e) {
+  gws::RowRec r;
+  std::memset(&r, 0, sizeof r);
+  r.in = e.in;
+  r.out = e.out;
+  r.gin = e.gin;
+  r.gout = e.gout;
+  r.vec_lo = static_cast<uint32_t>(e.elem_offset >> 3);
+  r.vec_hi = static_cast<uint32_t>(e.elem_offset >> 35);
+  r.rows = static_cast<uint32_t>(e.rows);
+  r.cpr = static_cast<uint32_t>(e.cols / 32);
+  r.k0 = e.seed_lo;
+  r.k1 = e.seed_hi;
+  if (r.cpr > 128u) {   // one block per row
+    r.tpr_log2 = 8;
+    r.cpt = (r.cpr + gws::kRowThreads - 1) / gws::kRowThreads;
+  } else {              // 1..32 threads per row: the (threads, chunks per thread) pair with the fewest idle slots
+    uint32_t best_slots = ~0u;
+    for (uint32_t cpt = 1; cpt <= static_cast<uint32_t>(gws::kRowMaxCpt); ++cpt) {
+      uint32_t need = (r.cpr + cpt - 1) / cpt, log2 = 0;
+      while ((1u << log2) < need) ++log2;
+      if (log2 > 5u) continue;
+      const uint32_t slots = (1u << log2) * cpt;
+      if (slots < best_slots) { best_slots = slots; r.tpr_log2 = log2; r.cpt = cpt; }
+    }
+  }
+  return r;
+}
+
+template <int MODE, bool BLOCK, int CAP>
+int launch_row_batch(const gws::RowRec* recs, int count, uint32_t lo, uint32_t hi, cudaStream_t stream) {
+  gws::RowBatch<CAP> b;
+  std::memset(&b, 0, sizeof b);
+  const int64_t tiles = gws::fill_row_batch<CAP>(b, recs, count, BLOCK, lo, hi);
+  if (tiles < 0) return GWS_ERR_LIMIT;
+  if (tiles == 0) return GWS_OK;
+  gws::k_row<MODE, BLOCK, CAP><<<static_cast<unsigned>(tiles), gws::kRowThreads, 0, stream>>>(b);
+  return check_launch("row kernel");
+}
+
+template <int MODE, bool BLOCK>
+int launch_row_chunks(const std::vector<gws::RowRec>& recs, uint32_t lo, uint32_t hi, cudaStream_t stream) {
+  for (size_t first = 0; first < recs.size(); first += gws::kRowCapLarge) {
+    const int count = static_cast<int>(std::min(recs.size() - first, static_cast<size_t>(gws::kRowCapLarge)));
+    const int st = count <= gws::kRowCapSmall
+                       ? launch_row_batch<MODE, BLOCK, gws::kRowCapSmall>(recs.data() + first, count, lo, hi, stream)
+                       : launch_row_batch<MODE, BLOCK, gws::kRowCapLarge>(recs.data() + first, count, lo, hi, stream);
+    if (st != GWS_OK) return st;
+  }
+  return GWS_OK;
+}
+
+template <int MODE>
+int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int64_t tiles, uint64_t step,
+           cudaStream_t stream);
+
+// All entries of a row class (kRowWarp or kRowCta): chunk kernel where it applies, else one launch each.
+template <int MODE>
+int launch_rows(int cls, const Entry* entries, int count, uint64_t step, cudaStream_t stream) {
+  std::vector<gws::RowRec> shared_rows, block_rows;
+  const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
+  for (int k = 0; k < count; ++k) {
+    if (row_chunk_eligible(entries[k])) {
+      const gws::RowRec r = to_row_rec(entries[k]);
+      (r.tpr_log2 == 8u ? block_rows : shared_rows).push_back(r);
+    } else {
+      Entry e = entries[k];
+      e.tile_begin = 0;
+      const int64_t tiles = cls == gws::kRowWarp ? (e.rows + (gws::kRowWarpThreads / 32) - 1) / (gws::kRowWarpThreads / 32) : e.rows;
+      const int st = launch<MODE>(cls, e, nullptr, -1, tiles, step, stream);
+      if (st != GWS_OK) return st;
+    }
+  }
+  const int st = launch_row_chunks<MODE, false>(shared_rows, lo, hi, stream);
+  if (st != GWS_OK) return st;
+  return launch_row_chunks<MODE, true>(block_rows, lo, hi, stream);
+}
+
 template <int MODE, bool MULTI>
 int launch_as(int cls, const Entry& single, const Entry* table, int n_or_index, unsigned grid, uint32_t lo, uint32_t hi,
               cudaStream_t stream) {
@@ -219,6 +308,8 @@ int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int
   if (tiles <= 0) return GWS_OK;
   if (tiles > kMaxGrid) return GWS_ERR_LIMIT;
   if (cls == gws::kFlat) return launch_flat<MODE>(&single, 1, step, stream);   // single-tensor calls only
+  if ((cls == gws::kRowWarp || cls == gws::kRowCta) && table == nullptr && n_or_index != -1)
+    return launch_rows<MODE>(cls, &single, 1, step, stream);
   const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
   const unsigned grid = static_cast<unsigned>(tiles);
   return table == nullptr ? launch_as<MODE, false>(cls, single, table, n_or_index, grid, lo, hi, stream)
@@ -488,8 +579,9 @@ static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream, bo
       const int st = backward ? launch_flat<gws::kBwd>(host, count, step, s) : launch_flat<gws::kFwd>(host, count, step, s);
       if (st != GWS_OK) return st;
     } else if (cls != gws::kGeneral) {
-      const int st = backward ? launch<gws::kBwd>(cls, none, table, count, plan->tiles[cls], step, s)
-                              : launch<gws::kFwd>(cls, none, table, count, plan->tiles[cls], step, s);
+      const Entry* host = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
+                                                         (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
+      const int st = backward ? launch_rows<gws::kBwd>(cls, host, count, step, s) : launch_rows<gws::kFwd>(cls, host, count, step, s);
       if (st != GWS_OK) return st;
     } else {
       for (int i = 0; i < count; ++i) {
@@ -506,12 +598,20 @@ int gws_multi_launch_count(const gws_multi_plan* plan, int backward) {
   if (plan == nullptr) return GWS_ERR_NULL;
   if (plan->host_tables == nullptr) return GWS_ERR_WORKSPACE;
   if (backward ? !plan->has_bwd : !plan->has_fwd) return 0;
-  const Entry* flat = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
-                                                     (backward ? plan->bwd_offset[0] : plan->fwd_offset[0]));
-  int wide = 0, narrow = 0;
-  for (int k = 0; k < plan->count[0]; ++k) (flat[k].lanes_log2 < 2u ? narrow : wide) += 1;
-  const int cap = gws::kFlatCapLarge;
-  return (wide + cap - 1) / cap + (narrow + cap - 1) / cap + (plan->count[1] ? 1 : 0) + (plan->count[2] ? 1 : 0) + plan->count[3];
+  auto host = [&](int cls) {
+    return reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
+                                          (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
+  };
+  auto batches = [](int count, int cap) { return (count + cap - 1) / cap; };
+  int wide = 0, narrow = 0, shared_rows = 0, block_rows = 0, single = 0;
+  for (int k = 0; k < plan->count[0]; ++k) (host(0)[k].lanes_log2 < 2u ? narrow : wide) += 1;
+  for (int cls = 1; cls <= 2; ++cls)
+    for (int k = 0; k < plan->count[cls]; ++k) {
+      if (!row_chunk_eligible(host(cls)[k])) ++single;
+      else (host(cls)[k].cols > 4096 ? block_rows : shared_rows) += 1;
+    }
+  return batches(wide, gws::kFlatCapLarge) + batches(narrow, gws::kFlatCapLarge) + batches(shared_rows, gws::kRowCapLarge) +
+         batches(block_rows, gws::kRowCapLarge) + single + plan->count[3];
 }
 
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {

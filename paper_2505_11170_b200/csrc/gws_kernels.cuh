@@ -497,6 +497,159 @@ inline int64_t fill_flat_batch(FlatBatch<CAP>& b, const FlatRec* recs, int count
   return tiles;
 }
 
+// ---- whole-row groups on 64-byte chunks --------------------------------------------------------------
+//
+// Rows of a multiple of 32 elements, 32-byte aligned tensors.  T threads share a row (T = 1..32, a power
+// of two: several rows per warp, shuffle reductions only; or T = 256: one row per block, one
+// shared-memory step), each holding up to 4 chunks, T chunks apart, in registers between the max
+// and the add, so W is read once.  Records by value in the kernel parameters, as for flat groups.
+struct RowRec {
+  const void* in;
+  void* out;
+  const float* gin;
+  float* gout;
+  uint32_t vec_lo, vec_hi;
+  uint32_t rows, cpr;        // chunks per row = cols / 32
+  uint32_t tpr_log2, cpt;    // threads per row (log2; 8 for the block kernel), chunks per thread (1..4)
+  int32_t tile_begin;
+  uint32_t k0, k1;
+  PhiloxPre pre;
+  uint32_t pad;
+};
+static_assert(sizeof(RowRec) == 88, "RowRec layout");
+template <int CAP>
+struct RowBatch {
+  int32_t n;
+  uint32_t hint_shift;
+  uint32_t pad[2];
+  uint16_t hint[kFlatHint];
+  RowRec e[CAP];
+};
+constexpr int kRowCapSmall = 4, kRowCapLarge = 168;
+constexpr int kRowThreads = 256, kRowMaxCpt = 4;
+
+template <int MODE, bool BLOCK, int CAP>
+__global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ RowBatch<CAP> b) {
+  __shared__ uint32_t red_u[kRowThreads / 32];
+  __shared__ float red_f[kRowThreads / 32];
+  const int32_t tile = static_cast<int32_t>(blockIdx.x);
+  int idx = b.hint[tile >> b.hint_shift];
+  while (idx + 1 < b.n && b.e[idx + 1].tile_begin <= tile) ++idx;
+  const RowRec& e = b.e[idx];
+  const uint32_t tpr_log2 = BLOCK ? 8u : e.tpr_log2, tpr = 1u << tpr_log2;
+  const uint32_t local = static_cast<uint32_t>(tile - e.tile_begin);
+  const uint32_t row0 = BLOCK ? local : local * (kRowThreads >> tpr_log2) + (threadIdx.x >> tpr_log2);
+  const uint32_t t = threadIdx.x & (tpr - 1u);
+  const bool okr = row0 < e.rows;
+  const uint32_t row = okr ? row0 : e.rows - 1u;   // keeps warps whole for the shuffles; nothing is stored for it
+  const uint32_t cpr = e.cpr, cpt = e.cpt;
+  const uint32_t row_chunk0 = row * cpr;
+
+  Chunk c[kRowMaxCpt];
+  bool ok[kRowMaxCpt];
+#pragma unroll
+  for (int k = 0; k < kRowMaxCpt; ++k) {
+    const uint32_t q = static_cast<uint32_t>(k) * tpr + t;
+    ok[k] = static_cast<uint32_t>(k) < cpt && q < cpr;
+    if (ok[k]) {
+      c[k] = load_chunk<true>(e.in, row_chunk0 + q, 4);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) c[k].x[i] = 0u;
+    }
+  }
+  const float gv = (MODE != kAbsmax) ? ld_f32(e.gin, row) : 0.0f;
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const uint32_t span = BLOCK ? 32u : tpr;   // lanes of this warp that share the row
+
+  if (MODE == kBwd) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int k = 0; k < kRowMaxCpt; ++k) {
+      if (!ok[k]) continue;
+      const uint32_t chunk = row_chunk0 + static_cast<uint32_t>(k) * tpr + t;
+      const uint32_t v0 = e.vec_lo + chunk * 4u;
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        const Words4 r = philox4x32_10_pre(v0 + v, e.k0, e.k1, e.pre);
+        acc = dot_vec(make_uint4(c[k].x[4 * v], c[k].x[4 * v + 1], c[k].x[4 * v + 2], c[k].x[4 * v + 3]), r, acc);
+      }
+      if (okr && e.out != nullptr) store_chunk<true>(e.out, chunk, 4, c[k]);
+    }
+    for (uint32_t o = 1; o < span; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if (BLOCK) {
+      if (lane == 0) red_f[warp] = acc;
+      __syncthreads();
+      acc = 0.0f;
+#pragma unroll
+      for (int w = 0; w < kRowThreads / 32; ++w) acc += red_f[w];   // fixed order
+    }
+    if (okr && t == 0u) st_f32(e.gout, row, grad_bt_of(gv, acc));
+    return;
+  }
+
+  uint32_t m = 0u;
+#pragma unroll
+  for (int k = 0; k < kRowMaxCpt; ++k)
+    m = maxabs2(m, maxabs2(maxabs2(absmax_words4(c[k].x), absmax_words4(c[k].x + 4)),
+                           maxabs2(absmax_words4(c[k].x + 8), absmax_words4(c[k].x + 12))));
+  for (uint32_t o = 1; o < span; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if (BLOCK) {
+    if (lane == 0) red_u[warp] = m;
+    __syncthreads();
+    m = red_u[0];
+#pragma unroll
+    for (int w = 1; w < kRowThreads / 32; ++w) m = maxabs2(m, red_u[w]);
+  }
+  const float a = absmax_finish(m);
+  if (MODE == kAbsmax) {
+    if (okr && t == 0u) st_f32(e.gout, row, a);
+    return;
+  }
+  const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv)));
+#pragma unroll
+  for (int k = 0; k < kRowMaxCpt; ++k) {
+    if (!ok[k]) continue;
+    const uint32_t chunk = row_chunk0 + static_cast<uint32_t>(k) * tpr + t;
+    const uint32_t v0 = e.vec_lo + chunk * 4u;
+    Chunk y;
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const Words4 r = philox4x32_10_pre(v0 + v, e.k0, e.k1, e.pre);
+      uint32_t p[4];
+      decode8(r, p);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) y.x[4 * v + j] = sample_pair(c[k].x[4 * v + j], p[j], sc);
+    }
+    if (okr) store_chunk<true>(e.out, chunk, 4, y);
+  }
+  if (okr && t == 0u && e.gout != nullptr) st_f32(e.gout, row, sc.s);
+}
+
+// Host side: as fill_flat_batch.  Tiles: rows per block for shared rows (256 / threads per row), one row per block else.
+template <int CAP>
+inline int64_t fill_row_batch(RowBatch<CAP>& b, const RowRec* recs, int count, bool block, uint32_t step_lo, uint32_t step_hi) {
+  b.n = count;
+  b.hint_shift = 0;
+  int64_t tiles = 0;
+  for (int k = 0; k < count; ++k) {
+    b.e[k] = recs[k];
+    b.e[k].tile_begin = static_cast<int32_t>(tiles);
+    b.e[k].pre = philox_pre(recs[k].vec_hi, step_lo, step_hi, recs[k].k0, recs[k].k1);
+    const int64_t rows_per_tile = block ? 1 : (kRowThreads >> recs[k].tpr_log2);
+    tiles += (static_cast<int64_t>(recs[k].rows) + rows_per_tile - 1) / rows_per_tile;
+    if (tiles > 2147483647LL) return -1;
+  }
+  while (tiles > 0 && ((tiles - 1) >> b.hint_shift) >= kFlatHint) ++b.hint_shift;
+  int owner = 0;
+  for (int h = 0; h < kFlatHint; ++h) {
+    const int64_t t = static_cast<int64_t>(h) << b.hint_shift;
+    while (owner + 1 < count && b.e[owner + 1].tile_begin <= t) ++owner;
+    b.hint[h] = static_cast<uint16_t>(owner);
+  }
+  return tiles;
+}
+
 // ---- one warp per row ---------------------------------------------------------------------------
 
 template <int MODE, bool MULTI>
