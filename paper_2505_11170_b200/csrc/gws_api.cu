@@ -235,27 +235,42 @@ gws::RowRec to_row_rec(const Entry& e) {
   return r;
 }
 
-template <int MODE, bool BLOCK, int CAP>
+template <int MODE, bool BLOCK, int CAP, int MAXCPT>
 int launch_row_batch(const gws::RowRec* recs, int count, uint32_t lo, uint32_t hi, cudaStream_t stream) {
   gws::RowBatch<CAP> b;
   std::memset(&b, 0, sizeof b);
   const int64_t tiles = gws::fill_row_batch<CAP>(b, recs, count, BLOCK, lo, hi);
   if (tiles < 0) return GWS_ERR_LIMIT;
   if (tiles == 0) return GWS_OK;
-  gws::k_row<MODE, BLOCK, CAP><<<static_cast<unsigned>(tiles), gws::kRowThreads, 0, stream>>>(b);
+  gws::k_row<MODE, BLOCK, CAP, MAXCPT><<<static_cast<unsigned>(tiles), gws::kRowThreads, 0, stream>>>(b);
   return check_launch("row kernel");
+}
+
+// Register-array size class of a record: its chunks per thread (1..4).
+int row_cpt_class(const gws::RowRec& r) { return static_cast<int>(r.cpt < 1u ? 1u : r.cpt); }
+
+template <int MODE, bool BLOCK, int MAXCPT>
+int launch_row_chunks_of(const std::vector<gws::RowRec>& all, uint32_t lo, uint32_t hi, cudaStream_t stream) {
+  std::vector<gws::RowRec> recs;
+  for (const gws::RowRec& r : all)
+    if (row_cpt_class(r) == MAXCPT) recs.push_back(r);
+  for (size_t first = 0; first < recs.size(); first += gws::kRowCapLarge) {
+    const int count = static_cast<int>(std::min(recs.size() - first, static_cast<size_t>(gws::kRowCapLarge)));
+    const int st = count <= gws::kRowCapSmall
+                       ? launch_row_batch<MODE, BLOCK, gws::kRowCapSmall, MAXCPT>(recs.data() + first, count, lo, hi, stream)
+                       : launch_row_batch<MODE, BLOCK, gws::kRowCapLarge, MAXCPT>(recs.data() + first, count, lo, hi, stream);
+    if (st != GWS_OK) return st;
+  }
+  return GWS_OK;
 }
 
 template <int MODE, bool BLOCK>
 int launch_row_chunks(const std::vector<gws::RowRec>& recs, uint32_t lo, uint32_t hi, cudaStream_t stream) {
-  for (size_t first = 0; first < recs.size(); first += gws::kRowCapLarge) {
-    const int count = static_cast<int>(std::min(recs.size() - first, static_cast<size_t>(gws::kRowCapLarge)));
-    const int st = count <= gws::kRowCapSmall
-                       ? launch_row_batch<MODE, BLOCK, gws::kRowCapSmall>(recs.data() + first, count, lo, hi, stream)
-                       : launch_row_batch<MODE, BLOCK, gws::kRowCapLarge>(recs.data() + first, count, lo, hi, stream);
-    if (st != GWS_OK) return st;
-  }
-  return GWS_OK;
+  int st = launch_row_chunks_of<MODE, BLOCK, 1>(recs, lo, hi, stream);
+  if (st == GWS_OK) st = launch_row_chunks_of<MODE, BLOCK, 2>(recs, lo, hi, stream);
+  if (st == GWS_OK) st = launch_row_chunks_of<MODE, BLOCK, 3>(recs, lo, hi, stream);
+  if (st == GWS_OK) st = launch_row_chunks_of<MODE, BLOCK, 4>(recs, lo, hi, stream);
+  return st;
 }
 
 template <int MODE>
@@ -603,15 +618,18 @@ int gws_multi_launch_count(const gws_multi_plan* plan, int backward) {
                                           (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
   };
   auto batches = [](int count, int cap) { return (count + cap - 1) / cap; };
-  int wide = 0, narrow = 0, shared_rows = 0, block_rows = 0, single = 0;
+  int wide = 0, narrow = 0, single = 0, rows[2][5] = {{0}};
   for (int k = 0; k < plan->count[0]; ++k) (host(0)[k].lanes_log2 < 2u ? narrow : wide) += 1;
   for (int cls = 1; cls <= 2; ++cls)
     for (int k = 0; k < plan->count[cls]; ++k) {
-      if (!row_chunk_eligible(host(cls)[k])) ++single;
-      else (host(cls)[k].cols > 4096 ? block_rows : shared_rows) += 1;
+      if (!row_chunk_eligible(host(cls)[k])) { ++single; continue; }
+      const gws::RowRec r = to_row_rec(host(cls)[k]);
+      rows[r.tpr_log2 == 8u ? 1 : 0][row_cpt_class(r)] += 1;
     }
-  return batches(wide, gws::kFlatCapLarge) + batches(narrow, gws::kFlatCapLarge) + batches(shared_rows, gws::kRowCapLarge) +
-         batches(block_rows, gws::kRowCapLarge) + single + plan->count[3];
+  int total = batches(wide, gws::kFlatCapLarge) + batches(narrow, gws::kFlatCapLarge) + single + plan->count[3];
+  for (int blk = 0; blk < 2; ++blk)
+    for (int c = 1; c <= 4; ++c) total += batches(rows[blk][c], gws::kRowCapLarge);
+  return total;
 }
 
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {

@@ -528,7 +528,8 @@ struct RowBatch {
 constexpr int kRowCapSmall = 4, kRowCapLarge = 168;
 constexpr int kRowThreads = 256, kRowMaxCpt = 4;
 
-template <int MODE, bool BLOCK, int CAP>
+// MAXCPT (1..4): the chunks a thread holds in this launch; sizes the register arrays.
+template <int MODE, bool BLOCK, int CAP, int MAXCPT>
 __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ RowBatch<CAP> b) {
   __shared__ uint32_t red_u[kRowThreads / 32];
   __shared__ float red_f[kRowThreads / 32];
@@ -545,10 +546,10 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
   const uint32_t cpr = e.cpr, cpt = e.cpt;
   const uint32_t row_chunk0 = row * cpr;
 
-  Chunk c[kRowMaxCpt];
-  bool ok[kRowMaxCpt];
+  Chunk c[MAXCPT];
+  bool ok[MAXCPT];
 #pragma unroll
-  for (int k = 0; k < kRowMaxCpt; ++k) {
+  for (int k = 0; k < MAXCPT; ++k) {
     const uint32_t q = static_cast<uint32_t>(k) * tpr + t;
     ok[k] = static_cast<uint32_t>(k) < cpt && q < cpr;
     if (ok[k]) {
@@ -565,7 +566,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
   if (MODE == kBwd) {
     float acc = 0.0f;
 #pragma unroll
-    for (int k = 0; k < kRowMaxCpt; ++k) {
+    for (int k = 0; k < MAXCPT; ++k) {
       if (!ok[k]) continue;
       const uint32_t chunk = row_chunk0 + static_cast<uint32_t>(k) * tpr + t;
       const uint32_t v0 = e.vec_lo + chunk * 4u;
@@ -590,7 +591,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
 
   uint32_t m = 0u;
 #pragma unroll
-  for (int k = 0; k < kRowMaxCpt; ++k)
+  for (int k = 0; k < MAXCPT; ++k)
     m = maxabs2(m, maxabs2(maxabs2(absmax_words4(c[k].x), absmax_words4(c[k].x + 4)),
                            maxabs2(absmax_words4(c[k].x + 8), absmax_words4(c[k].x + 12))));
   for (uint32_t o = 1; o < span; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
@@ -608,7 +609,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
   }
   const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv)));
 #pragma unroll
-  for (int k = 0; k < kRowMaxCpt; ++k) {
+  for (int k = 0; k < MAXCPT; ++k) {
     if (!ok[k]) continue;
     const uint32_t chunk = row_chunk0 + static_cast<uint32_t>(k) * tpr + t;
     const uint32_t v0 = e.vec_lo + chunk * 4u;

@@ -287,7 +287,9 @@ def test_multi_tensor_launch_mixed_classes():
              T("i", 2, 16384, 1, 0), T("j", 33, 2048, 1, 128)]
     plan = _run_multi_against_oracle(specs, steps=(0, 1, 9), with_copy=True)
     assert list(plan.plan.count) == [4, 2, 2, 2]
-    assert plan.launches_per_pass == 5
+    # flat groups (a, e, g, j): 1; short rows b, f (3 chunks per thread): 1; block rows c (1 chunk per thread) and
+    # i (2 chunks): 1 each; general d, h: 1 each
+    assert plan.launches_per_pass == 6
 
 
 def test_multi_tensor_empty_entries_and_forward_only():
