@@ -194,7 +194,7 @@ int gws_multi_locate_probe(const gws_multi_plan* plan, int backward, int kernel_
 /* Kernel launches one forward (backward != 0: backward) pass of the plan enqueues.  Tensors that share
  * a kernel share a launch (up to 192 flat-group or 168 whole-row tensors each): flat groups of 32..256
  * elements; flat groups of 8 / 16; rows up to 4096 elements and rows up to 32768 elements, each split
- * by how many 64-byte chunks a thread holds (1 to 4).  Whole-row
+ * by how many 64-byte chunks a thread holds (1 to 4); tensors of whole 32 x 32 blocks.  Whole-row
  * tensors whose rows are not a multiple of 32 elements, are longer, or are not 32-byte aligned, and
  * general-class tensors, take one launch each. */
 int gws_multi_launch_count(const gws_multi_plan* plan, int backward);

@@ -299,6 +299,57 @@ int launch_rows(int cls, const Entry* entries, int count, uint64_t step, cudaStr
   return launch_row_chunks<MODE, true>(block_rows, lo, hi, stream);
 }
 
+// ---- 32 x 32 square blocks --------------------------------------------------------------------------
+
+bool square_eligible(const Entry& e) {
+  if (e.group_rows != 32 || e.group_cols != 32 || e.rows % 32 != 0 || e.cols % 32 != 0 || e.ld != e.cols) return false;
+  if (!aligned(e.in, 32) || !aligned(e.out, 32)) return false;
+  const uint64_t n_vec = static_cast<uint64_t>(e.rows) * static_cast<uint64_t>(e.cols) / 8u;
+  const uint64_t first = e.elem_offset >> 3, last = first + n_vec - 1;
+  return (first >> 32) == (last >> 32) && (last - first) < 0xFFFFFFFFull;
+}
+
+template <int MODE, int CAP>
+int launch_square_batch(const Entry* const* entries, int count, uint32_t lo, uint32_t hi, cudaStream_t stream) {
+  gws::SquareBatch<CAP> b;
+  std::memset(&b, 0, sizeof b);
+  gws::SquareRec recs[CAP];
+  uint32_t bands[CAP];
+  for (int k = 0; k < count; ++k) {
+    const Entry& e = *entries[k];
+    gws::SquareRec& r = recs[k];
+    std::memset(&r, 0, sizeof r);
+    r.in = e.in;
+    r.out = e.out;
+    r.gin = e.gin;
+    r.gout = e.gout;
+    r.vec_lo = static_cast<uint32_t>(e.elem_offset >> 3);
+    r.vec_hi = static_cast<uint32_t>(e.elem_offset >> 35);
+    r.cpr = static_cast<uint32_t>(e.cols / 32);
+    r.k0 = e.seed_lo;
+    r.k1 = e.seed_hi;
+    bands[k] = static_cast<uint32_t>(e.rows / 32);
+  }
+  const int64_t tiles = gws::fill_square_batch<CAP>(b, recs, bands, count, lo, hi);
+  if (tiles < 0) return GWS_ERR_LIMIT;
+  if (tiles == 0) return GWS_OK;
+  gws::k_square<MODE, CAP><<<static_cast<unsigned>(tiles), gws::kFlatThreads, 0, stream>>>(b);
+  return check_launch("square-block kernel");
+}
+
+template <int MODE>
+int launch_squares(const std::vector<const Entry*>& entries, uint64_t step, cudaStream_t stream) {
+  const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
+  for (size_t first = 0; first < entries.size(); first += gws::kFlatCapLarge) {
+    const int count = static_cast<int>(std::min(entries.size() - first, static_cast<size_t>(gws::kFlatCapLarge)));
+    const int st = count <= gws::kFlatCapSmall
+                       ? launch_square_batch<MODE, gws::kFlatCapSmall>(entries.data() + first, count, lo, hi, stream)
+                       : launch_square_batch<MODE, gws::kFlatCapLarge>(entries.data() + first, count, lo, hi, stream);
+    if (st != GWS_OK) return st;
+  }
+  return GWS_OK;
+}
+
 template <int MODE, bool MULTI>
 int launch_as(int cls, const Entry& single, const Entry* table, int n_or_index, unsigned grid, uint32_t lo, uint32_t hi,
               cudaStream_t stream) {
@@ -325,6 +376,10 @@ int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int
   if (cls == gws::kFlat) return launch_flat<MODE>(&single, 1, step, stream);   // single-tensor calls only
   if ((cls == gws::kRowWarp || cls == gws::kRowCta) && table == nullptr && n_or_index != -1)
     return launch_rows<MODE>(cls, &single, 1, step, stream);
+  if (cls == gws::kGeneral && table == nullptr && square_eligible(single)) {
+    const std::vector<const Entry*> one{&single};
+    return launch_squares<MODE>(one, step, stream);
+  }
   const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
   const unsigned grid = static_cast<unsigned>(tiles);
   return table == nullptr ? launch_as<MODE, false>(cls, single, table, n_or_index, grid, lo, hi, stream)
@@ -599,11 +654,18 @@ static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream, bo
       const int st = backward ? launch_rows<gws::kBwd>(cls, host, count, step, s) : launch_rows<gws::kFwd>(cls, host, count, step, s);
       if (st != GWS_OK) return st;
     } else {
+      // whole 32 x 32 blocks share launches of the square-block kernel; every other shape: one launch per tensor
+      const Entry* host = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
+                                                         (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
+      std::vector<const Entry*> squares;
       for (int i = 0; i < count; ++i) {
+        if (square_eligible(host[i])) { squares.push_back(&host[i]); continue; }
         const int st = backward ? launch<gws::kBwd>(cls, none, table, i, kGeneralGrid, step, s)
                                 : launch<gws::kFwd>(cls, none, table, i, kGeneralGrid, step, s);
         if (st != GWS_OK) return st;
       }
+      const int st = backward ? launch_squares<gws::kBwd>(squares, step, s) : launch_squares<gws::kFwd>(squares, step, s);
+      if (st != GWS_OK) return st;
     }
   }
   return GWS_OK;
@@ -626,7 +688,10 @@ int gws_multi_launch_count(const gws_multi_plan* plan, int backward) {
       const gws::RowRec r = to_row_rec(host(cls)[k]);
       rows[r.tpr_log2 == 8u ? 1 : 0][row_cpt_class(r)] += 1;
     }
-  int total = batches(wide, gws::kFlatCapLarge) + batches(narrow, gws::kFlatCapLarge) + single + plan->count[3];
+  int squares = 0;
+  for (int k = 0; k < plan->count[3]; ++k) squares += square_eligible(host(3)[k]) ? 1 : 0;
+  int total = batches(wide, gws::kFlatCapLarge) + batches(narrow, gws::kFlatCapLarge) + single + (plan->count[3] - squares) +
+              batches(squares, gws::kFlatCapLarge);
   for (int blk = 0; blk < 2; ++blk)
     for (int c = 1; c <= 4; ++c) total += batches(rows[blk][c], gws::kRowCapLarge);
   return total;

@@ -497,6 +497,131 @@ inline int64_t fill_flat_batch(FlatBatch<CAP>& b, const FlatRec* recs, int count
   return tiles;
 }
 
+// ---- the paper's square blocks: 32 x 32 elements (Eq. 3, b_l = 32) -------------------------------------
+//
+// A 32 x 32 block is one 64-byte chunk in each of 32 consecutive rows: a warp takes one block, lane =
+// row, so the block maximum and the gradient sum are full-warp shuffle reductions and every lane still
+// moves 64 contiguous bytes.  The 8 warps of a thread block take 8 neighbouring blocks of the same 32
+// rows (512 contiguous bytes per row), CPT of them each.  Tensors with whole blocks only (rows and
+// cols multiples of 32), dense and 32-byte aligned; the general kernel covers the rest.
+struct SquareRec {
+  const void* in;
+  void* out;
+  const float* gin;
+  float* gout;
+  uint32_t vec_lo, vec_hi;
+  uint32_t cpr;             // chunks per row = blocks per row band = cols / 32
+  uint32_t tiles_per_band;  // ceil(cpr / (8 * CPT))
+  int32_t tile_begin;
+  uint32_t k0, k1;
+  PhiloxPre pre;
+  uint32_t pad;
+};
+static_assert(sizeof(SquareRec) == 80, "SquareRec layout");
+template <int CAP>
+struct SquareBatch {
+  int32_t n;
+  uint32_t hint_shift;
+  uint32_t pad[2];
+  uint16_t hint[kFlatHint];
+  SquareRec e[CAP];
+};
+constexpr int kSquareCpt = 2;
+
+template <int MODE, int CAP>
+__global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__ SquareBatch<CAP> b) {
+  constexpr int CPT = kSquareCpt;
+  const int32_t tile = static_cast<int32_t>(blockIdx.x);
+  int idx = b.hint[tile >> b.hint_shift];
+  while (idx + 1 < b.n && b.e[idx + 1].tile_begin <= tile) ++idx;
+  const SquareRec& e = b.e[idx];
+  const uint32_t local = static_cast<uint32_t>(tile - e.tile_begin);
+  const uint32_t band = local / e.tiles_per_band, in_band = local - band * e.tiles_per_band;
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const uint32_t cpr = e.cpr;
+  const uint32_t row_chunk0 = (band * 32u + lane) * cpr;
+
+  uint32_t q[CPT];
+  bool ok[CPT];       // uniform over the warp
+  Chunk c[CPT];
+  float gv[CPT];
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    q[i] = in_band * (8u * CPT) + static_cast<uint32_t>(i) * 8u + warp;
+    ok[i] = q[i] < cpr;
+    if (ok[i]) {
+      c[i] = load_chunk<true>(e.in, row_chunk0 + q[i], 4);
+      gv[i] = (MODE != kAbsmax) ? ld_f32(e.gin, band * cpr + q[i]) : 0.0f;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    if (!ok[i]) continue;
+    const uint32_t g = band * cpr + q[i];
+    const uint32_t chunk = row_chunk0 + q[i];
+    const uint32_t v0 = e.vec_lo + chunk * 4u;
+    if (MODE == kBwd) {
+      float acc = 0.0f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
+        acc = dot_vec(make_uint4(c[i].x[4 * k], c[i].x[4 * k + 1], c[i].x[4 * k + 2], c[i].x[4 * k + 3]), r, acc);
+      }
+#pragma unroll
+      for (uint32_t o = 1; o < 32u; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+      if (lane == 0u) st_f32(e.gout, g, grad_bt_of(gv[i], acc));
+      if (e.out != nullptr) store_chunk<true>(e.out, chunk, 4, c[i]);
+      continue;
+    }
+    uint32_t m = maxabs2(maxabs2(absmax_words4(c[i].x), absmax_words4(c[i].x + 4)),
+                         maxabs2(absmax_words4(c[i].x + 8), absmax_words4(c[i].x + 12)));
+#pragma unroll
+    for (uint32_t o = 1; o < 32u; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    const float a = absmax_finish(m);
+    if (MODE == kAbsmax) {
+      if (lane == 0u) st_f32(e.gout, g, a);
+      continue;
+    }
+    const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv[i])));
+    Chunk y;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
+      uint32_t p[4];
+      decode8(r, p);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) y.x[4 * k + j] = sample_pair(c[i].x[4 * k + j], p[j], sc);
+    }
+    store_chunk<true>(e.out, chunk, 4, y);
+    if (lane == 0u && e.gout != nullptr) st_f32(e.gout, g, sc.s);
+  }
+}
+
+// Host side: `bands[k]` = rows / 32 of record k.  Returns the number of tiles.
+template <int CAP>
+inline int64_t fill_square_batch(SquareBatch<CAP>& b, const SquareRec* recs, const uint32_t* bands, int count, uint32_t step_lo,
+                                 uint32_t step_hi) {
+  b.n = count;
+  b.hint_shift = 0;
+  int64_t tiles = 0;
+  for (int k = 0; k < count; ++k) {
+    b.e[k] = recs[k];
+    b.e[k].tile_begin = static_cast<int32_t>(tiles);
+    b.e[k].tiles_per_band = (recs[k].cpr + 8u * kSquareCpt - 1u) / (8u * kSquareCpt);
+    b.e[k].pre = philox_pre(recs[k].vec_hi, step_lo, step_hi, recs[k].k0, recs[k].k1);
+    tiles += static_cast<int64_t>(bands[k]) * b.e[k].tiles_per_band;
+    if (tiles > 2147483647LL) return -1;
+  }
+  while (tiles > 0 && ((tiles - 1) >> b.hint_shift) >= kFlatHint) ++b.hint_shift;
+  int owner = 0;
+  for (int h = 0; h < kFlatHint; ++h) {
+    const int64_t t = static_cast<int64_t>(h) << b.hint_shift;
+    while (owner + 1 < count && b.e[owner + 1].tile_begin <= t) ++owner;
+    b.hint[h] = static_cast<uint16_t>(owner);
+  }
+  return tiles;
+}
+
 // ---- whole-row groups on 64-byte chunks --------------------------------------------------------------
 //
 // Rows of a multiple of 32 elements, 32-byte aligned tensors.  T threads share a row (T = 1..32, a power

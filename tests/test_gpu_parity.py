@@ -26,9 +26,10 @@ FLAT = [(37, 384, 1, 128, None), (50, 160, 1, 32, None), (1030, 64, 1, 8, None),
 ROW_WARP = [(21, 768, 1, 0, None), (13, 3072, 1, 0, None), (9, 2304, 1, 0, None), (11, 4096, 1, 0, None),
             (70, 520, 1, 0, None), (1, 24, 1, 0, None), (12, 776, 1, 776, None)]
 ROW_CTA = [(5, 8192, 1, 0, None), (3, 28672, 1, 0, None), (2, 65536, 1, 0, None), (4, 4104, 1, 0, None)]
-GENERAL = [(64, 96, 32, 32, None), (33, 40, 32, 32, None), (5, 72, 1, 32, None), (6, 64, 1, 32, 80), (7, 13, 2, 5, None),
+SQUARE = [(64, 96, 32, 32, None), (96, 608, 32, 32, None), (32, 2048, 32, 32, None), (160, 32, 32, 32, None)]
+GENERAL = [(33, 40, 32, 32, None), (5, 72, 1, 32, None), (6, 64, 1, 32, 80), (7, 13, 2, 5, None),
            (4, 100, 1, 0, None), (3, 66000, 1, 0, None), (40, 48, 8, 48, 56), (300, 8, 1, 0, 8)]
-ALL = FLAT + ROW_WARP + ROW_CTA + GENERAL
+ALL = FLAT + ROW_WARP + ROW_CTA + SQUARE + GENERAL
 
 
 def _make(rows, cols, ld, seed, sigma=0.02):
@@ -231,6 +232,18 @@ def test_large_element_offsets(offset, group_cols, want_class, step=(1 << 40) + 
     assert err.max() <= 1e-5 * np.abs(want_gbt).max()
     packed = gws.noise(d).cpu().numpy().view(np.uint32)
     assert (packed == orc.noise_packed(seed, step, offset, rows * cols)).all()
+
+
+def test_square_blocks_commute_with_transposition():
+    # The paper's 32 x 32 blocks are chosen so that the block maxima of W^T are the transposed block maxima of W
+    # (Section 3.1: forward and backward GEMMs see the same scales).
+    rows, cols = 96, 160
+    w = _make(rows, cols, None, 31)
+    a = gws.group_absmax(Desc.make(rows, cols, 32, 32), w.to(DEV)).cpu().view(rows // 32, cols // 32)
+    at = gws.group_absmax(Desc.make(cols, rows, 32, 32), w.t().contiguous().to(DEV)).cpu().view(cols // 32, rows // 32)
+    assert torch.equal(a.t().contiguous(), at)
+    want = w.float().abs().view(rows // 32, 32, cols // 32, 32).amax(dim=(1, 3))
+    assert torch.equal(a, want)
 
 
 def test_steps_and_seeds_give_different_noise_and_same_step_repeats():
