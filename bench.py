@@ -204,6 +204,7 @@ def main():
     ap.add_argument("--blocks", type=int, default=22, help="Llama blocks in the set (22 = the full workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the side measurements (per-layer launches, copy mode, ALU ceiling)")
     ap.add_argument("--source-hash", action="store_true", help="print the hash an ncu summary records with its counters")
     args = ap.parse_args()
     if args.impl == "ours":
@@ -320,6 +321,44 @@ def main():
                "ms_per_step": float(e2e_ms), "steps": e2e_steps,
                "note": "gws_sample_step_host per tensor; pinned host buffers of one transformer block reused for all 22"}
 
+    # ---- side measurements (one GPU only; not part of `value`) ----
+    extras = None
+    if world == 1 and not args.no_extras:
+        def timed(fn, reps):
+            fn(0)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for k in range(reps):
+                fn(1 + k)
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        def per_layer(k):
+            for i in range(len(specs)):
+                d = descs[i].with_step(k)
+                gws.sample_fwd(d, W[i], BT[i], WH[i], SC[i], stream=stream)
+                gws.sample_bwd(d, G[i], SC[i], None, GBT[i], stream=stream)
+
+        per_layer_ms = timed(per_layer, 5)
+        GW = [torch.empty_like(t) for t in G]
+        copy_plan = gws.MultiPlan(descs, scale=SC, grad_w_hat=G, grad_w=GW, grad_bt=GBT)
+        bwd_copy_ms = timed(lambda k: copy_plan.sample_bwd_multi(k), 10)
+        del copy_plan, GW
+        probe_desc = Desc.make(n_elem // 2048, 2048, 1, 128, seed=1)
+        sink = gws.noise_alu_probe(probe_desc)
+        probe_ms = timed(lambda k: gws.noise_alu_probe(probe_desc.with_step(k), sink), 10)
+        extras = {
+            "per_layer_launches": {"ms_per_step": per_layer_ms, "launches_per_step": 2 * len(specs),
+                                   "GB/s": bytes_per_step / (per_layer_ms * 1e-3) / 1e9},
+            "bwd_with_grad_w_copy": {"ms_per_launch": bwd_copy_ms, "GB/s": n_elem * (4 + 8 / 128) / (bwd_copy_ms * 1e-3) / 1e9,
+                                     "bytes_per_element": 4 + 8 / 128},
+            "noise_arithmetic_ceiling": {"gelem_per_s": n_elem / (probe_ms * 1e-3) / 1e9, "ms": probe_ms,
+                                         "note": "Philox + decode with no memory traffic (gws_noise_alu_probe): "
+                                                 "what the backward pass (2.06 B/element) cannot exceed"},
+        }
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -348,6 +387,8 @@ def main():
                          "algorithmic_bytes_per_launch": bwd_bytes, "traffic": traffic.get("bwd_bytes_per_launch")},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
     }
+    if extras is not None:
+        line["extras"] = extras
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(syn.llama2_1b())
     print(json.dumps(line), flush=True)

@@ -256,9 +256,10 @@ int gws_sample_step_host(const gws_desc* desc, const void* h_w, const float* h_b
 int gws_philox_words(uint64_t seed, uint64_t step, uint64_t first_vec, int64_t n_vec, uint32_t* out4,
                      void* stream);
 
-/* Generates and decodes the noise of the descriptor exactly like gws_noise but stores only one
- * word per thread block (an XOR of the packed words it produced): the arithmetic ceiling of noise
- * generation without its memory traffic.  sink: device, u32 [gws_noise_alu_probe_words(desc)]. */
+/* Generates and decodes the noise of the descriptor with the arithmetic gws_sample_fwd / gws_sample_bwd
+ * spend on it (Philox4x32-10 and the AND / OR decode of Eq. 10) but stores only one word per thread
+ * block (an XOR of what it decoded): the rate of random-bit generation without memory traffic, which
+ * the backward pass (2 bytes per element) cannot exceed.  sink: device, u32 [gws_noise_alu_probe_words(desc)]. */
 int gws_noise_alu_probe(const gws_desc* desc, uint32_t* sink, void* stream);
 int64_t gws_noise_alu_probe_words(const gws_desc* desc);
 

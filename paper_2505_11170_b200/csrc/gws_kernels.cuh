@@ -1012,16 +1012,26 @@ __global__ void __launch_bounds__(256) k_noise(uint32_t* __restrict__ out, uint6
   out[v] = word;
 }
 
-// Same arithmetic as k_noise, 8 words per thread, one stored word per block.
+// The arithmetic the forward and backward kernels spend on noise (hoisted Philox rounds + whole-word decode)
+// with no memory traffic: 8 vectors per thread, one stored word per block.
 __global__ void __launch_bounds__(256) k_noise_probe(uint32_t* __restrict__ sink, uint64_t n_words, uint64_t vec0,
                                                      uint32_t seed_lo, uint32_t seed_hi, uint32_t step_lo,
                                                      uint32_t step_hi) {
   __shared__ uint32_t red[8];
   uint32_t acc = 0;
+  // one set of hoisted constants per block, as in the sampling kernels (its 2048 vectors share the high counter
+  // word unless the block straddles a multiple of 2^32, which only changes the value of this probe's sink)
+  const uint64_t block_vec0 = vec0 + static_cast<uint64_t>(blockIdx.x) * 2048u;
+  const PhiloxPre pre = philox_pre(static_cast<uint32_t>(block_vec0 >> 32), step_lo, step_hi, seed_lo, seed_hi);
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
     const uint64_t v = (static_cast<uint64_t>(blockIdx.x) * 8u + k) * 256u + threadIdx.x;
-    if (v < n_words) acc ^= pack_nibbles(philox_for_vector(vec0 + v, step_lo, step_hi, seed_lo, seed_hi));
+    if (v < n_words) {
+      const uint64_t vec = vec0 + v;
+      uint32_t p[4];
+      decode8(philox4x32_10_pre(static_cast<uint32_t>(vec), seed_lo, seed_hi, pre), p);
+      acc ^= p[0] ^ p[1] ^ p[2] ^ p[3];
+    }
   }
 #pragma unroll
   for (uint32_t o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xFFFFFFFFu, acc, o);

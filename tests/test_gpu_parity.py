@@ -246,6 +246,14 @@ def test_square_blocks_commute_with_transposition():
     assert torch.equal(a, want)
 
 
+def test_arithmetic_probe_runs_and_depends_on_the_stream():
+    d = Desc.make(512, 2048, 1, 128, seed=9, step=1)
+    a = gws.noise_alu_probe(d).cpu()
+    b = gws.noise_alu_probe(d).cpu()
+    c = gws.noise_alu_probe(d.with_step(2)).cpu()
+    assert a.numel() == 512 * 2048 // 8 // 2048 and torch.equal(a, b) and not torch.equal(a, c)
+
+
 def test_steps_and_seeds_give_different_noise_and_same_step_repeats():
     rows, cols = 32, 1024
     w = _make(rows, cols, None, 9).to(DEV)
