@@ -335,4 +335,48 @@ void gwso_sample_bwd(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows,
     grad_bt[g] = static_cast<float>(-ln2 * static_cast<double>(scale[g]) * acc_scratch[g]);
 }
 
+// ---- bit-width parametrisation and seeds (Section 3.6) ------------------------------------------------
+
+// Eq. 11: b_t = b_target + b_i * (b_init - b_target), in FP32 with one rounding per operation (the
+// result feeds 2^(1 - b_t), so its bits matter): delta = fl(b_init - b_target), then fl(b_i * delta),
+// then fl(b_target + that).
+void gwso_bitwidth(int64_t n, const float* bi, float b_init, float b_target, float* bt) {
+  const float delta = b_init - b_target;
+  for (int64_t k = 0; k < n; ++k) {
+    const float scaled = bi[k] * delta;
+    bt[k] = b_target + scaled;
+  }
+}
+
+// One layer's term of Eq. 12 without its lambda: the mean over the layer's m blocks of |b_t - b_target|.
+double gwso_bitwidth_loss(int64_t m, const float* bt, float b_target) {
+  double sum = 0.0;
+  for (int64_t k = 0; k < m; ++k) sum += std::fabs(static_cast<double>(bt[k]) - static_cast<double>(b_target));
+  return m > 0 ? sum / static_cast<double>(m) : 0.0;
+}
+
+// dL'/db_i for one layer: Eq. 12 adds lambda/m * sign(b_t - b_target) to dL/db_t (the derivative of |x|,
+// taken as 0 at x = 0), and Eq. 11 multiplies by db_t/db_i = b_init - b_target.
+void gwso_bitwidth_grad(int64_t m, const float* grad_bt, const float* bt, float b_init, float b_target, double lambda,
+                        double* grad_bi) {
+  const double delta = static_cast<double>(b_init) - static_cast<double>(b_target);
+  for (int64_t k = 0; k < m; ++k) {
+    const double x = static_cast<double>(bt[k]) - static_cast<double>(b_target);
+    const double sign = x > 0.0 ? 1.0 : (x < 0.0 ? -1.0 : 0.0);
+    grad_bi[k] = delta * (static_cast<double>(grad_bt[k]) + lambda / static_cast<double>(m) * sign);
+  }
+}
+
+// "Managing seed": the seed generator started from the user's seed gives every layer its own seed.
+// Reading: layer l gets the first 64 output bits of Philox4x32-10 with counter (lo32(l), hi32(l), 0, 0)
+// and key (lo32(user_seed), hi32(user_seed)); the per-update change of the layer's PRNG state is the
+// gradient-update counter `step` that goes into the sampling counter.
+uint64_t gwso_layer_seed(uint64_t user_seed, uint64_t layer) {
+  const uint32_t ctr[4] = {static_cast<uint32_t>(layer), static_cast<uint32_t>(layer >> 32), 0u, 0u};
+  const uint32_t key[2] = {static_cast<uint32_t>(user_seed), static_cast<uint32_t>(user_seed >> 32)};
+  uint32_t o[4];
+  philox4x32_10(ctr, key, o);
+  return static_cast<uint64_t>(o[0]) | (static_cast<uint64_t>(o[1]) << 32);
+}
+
 }  // extern "C"

@@ -51,6 +51,14 @@ def lib() -> ctypes.CDLL:
         L.gwso_philox_words.restype = None
         L.gwso_decode_field.argtypes = [c_uint32]
         L.gwso_decode_field.restype = c_int
+        L.gwso_bitwidth.argtypes = [c_int64, f32p, c_float, c_float, f32p]
+        L.gwso_bitwidth.restype = None
+        L.gwso_bitwidth_loss.argtypes = [c_int64, f32p, c_float]
+        L.gwso_bitwidth_loss.restype = c_double
+        L.gwso_bitwidth_grad.argtypes = [c_int64, f32p, f32p, c_float, c_float, c_double, f64p]
+        L.gwso_bitwidth_grad.restype = None
+        L.gwso_layer_seed.argtypes = [c_uint64, c_uint64]
+        L.gwso_layer_seed.restype = c_uint64
         L.gwso_field_of_element.argtypes = [POINTER(c_uint32), c_uint32]
         L.gwso_field_of_element.restype = c_uint32
         L.gwso_n_groups.argtypes = [c_int64] * 4
@@ -211,3 +219,32 @@ def sample_bwd(g, scale_, rows, cols, group_rows=1, group_cols=0, seed=0, step=0
         lib().gwso_sample_bwd_injected(rows, cols, ld, group_rows, group_cols, _p(g, c_uint16), _p(sc, c_float),
                                        _p(r, c_int8), _p(gw, c_uint16), _p(gbt, c_float), _p(acc, c_double))
     return gw, gbt
+
+
+# ---- bit-width parametrisation and seeds (Section 3.6) -------------------------------------------------
+
+def bitwidth(bi, b_init: float, b_target: float) -> np.ndarray:
+    """Eq. 11 in FP32: b_t = b_target + b_i * (b_init - b_target)."""
+    b = _c(bi, np.float32)
+    out = np.empty(b.size, np.float32)
+    lib().gwso_bitwidth(b.size, _p(b, c_float), b_init, b_target, _p(out, c_float))
+    return out
+
+
+def bitwidth_loss(bt, b_target: float) -> float:
+    """One layer's term of Eq. 12 without lambda: mean over its blocks of |b_t - b_target|."""
+    b = _c(bt, np.float32)
+    return float(lib().gwso_bitwidth_loss(b.size, _p(b, c_float), b_target))
+
+
+def bitwidth_grad(grad_bt, bt, b_init: float, b_target: float, lam: float) -> np.ndarray:
+    """dL'/db_i of one layer (float64): (b_init - b_target) * (dL/db_t + lam / m * sign(b_t - b_target))."""
+    g, b = _c(grad_bt, np.float32), _c(bt, np.float32)
+    assert g.size == b.size
+    out = np.empty(g.size, np.float64)
+    lib().gwso_bitwidth_grad(g.size, _p(g, c_float), _p(b, c_float), b_init, b_target, lam, _p(out, c_double))
+    return out
+
+
+def layer_seed(user_seed: int, layer: int) -> int:
+    return int(lib().gwso_layer_seed(user_seed & 0xFFFFFFFFFFFFFFFF, layer))
