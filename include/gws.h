@@ -203,6 +203,31 @@ int gws_multi_launch_count(const gws_multi_plan* plan, int backward);
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
 int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
 
+/* ---- bit-width parametrisation and seeds (Section 3.6, "Bitwidth" and "Managing seed") ---------------
+ *
+ * Eq. 11: b_t = b_target + b_i * (b_init - b_target), one trainable b_i per group (initialised to 1,
+ * pulled towards 0 by weight decay).  FP32, one rounding per operation (delta = fl(b_init - b_target),
+ * fl(b_i * delta), fl(b_target + that)): b_t feeds 2^(1 - b_t), so its bits matter.
+ *   bi, bt   device, FP32 [n_groups]; bt may be bi (in place)
+ */
+int gws_bitwidth(int64_t n_groups, const float* bi, float b_init, float b_target, float* bt, void* stream);
+
+/* One layer's term of Eq. 12 without lambda: loss_out[0] = mean over the layer's m groups of
+ * |b_t - b_target| (FP32, summed in a fixed order; 0 for m == 0).  bt, loss_out: device. */
+int gws_bitwidth_loss(int64_t m, const float* bt, float b_target, float* loss_out, void* stream);
+
+/* Chain rule back to b_i for one layer of m groups:
+ *   grad_bi = (b_init - b_target) * ( grad_bt + lambda / m * sign(b_t - b_target) ),  sign(0) = 0,
+ * i.e. Eq. 4's dL/db_t plus the derivative of the layer's Eq. 12 term, through Eq. 11.  lambda = 0
+ * gives the plain chain rule.  All arrays device, FP32 [m]; grad_bi may be grad_bt (in place). */
+int gws_bitwidth_grad(int64_t m, const float* grad_bt, const float* bt, float b_init, float b_target, double lambda,
+                      float* grad_bi, void* stream);
+
+/* Host only.  The seed of layer `layer` under the user's seed: the first 64 output bits of
+ * Philox4x32-10 with counter (lo32(layer), hi32(layer), 0, 0) and key (lo32(user_seed), hi32(user_seed)).
+ * The per-update change of a layer's PRNG state is the `step` of its descriptor. */
+uint64_t gws_layer_seed(uint64_t user_seed, uint64_t layer);
+
 /* ---- forward over many tensors for callers that cannot allocate device memory --------------------
  * (No counterpart in the paper: this entry point exists for the way the library gets embedded.)
  *

@@ -72,6 +72,10 @@ _SIGNATURES = {
     "gws_multi_launch_count": (c_int, [POINTER(_MultiPlan), c_int]),
     "gws_sample_fwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_sample_bwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
+    "gws_bitwidth": (c_int, [c_int64, c_void_p, c_float, c_float, c_void_p, c_void_p]),
+    "gws_bitwidth_loss": (c_int, [c_int64, c_void_p, c_float, c_void_p, c_void_p]),
+    "gws_bitwidth_grad": (c_int, [c_int64, c_void_p, c_void_p, c_float, c_float, ctypes.c_double, c_void_p, c_void_p]),
+    "gws_layer_seed": (c_uint64, [c_uint64, c_uint64]),
     "gws_sample_fwd_multi_static": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_uint64, c_void_p]),
     "gws_sample_step_host": (c_int, [POINTER(Desc)] + [c_void_p] * 13),
     "gws_philox_words": (c_int, [c_uint64, c_uint64, c_uint64, c_int64, c_void_p, c_void_p]),
@@ -263,6 +267,40 @@ class MultiPlan:
 
     def sample_bwd_multi(self, step: int, stream=None) -> None:
         _check(load_library().gws_sample_bwd_multi(ctypes.byref(self.plan), step, _stream(stream)))
+
+
+def bitwidth(bi: torch.Tensor, b_init: float, b_target: float, bt: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Eq. 11: b_t = b_target + b_i * (b_init - b_target)."""
+    _require_cuda(bi, bt)
+    if bt is None:
+        bt = torch.empty_like(bi)
+    _check(load_library().gws_bitwidth(bi.numel(), _ptr(bi), b_init, b_target, _ptr(bt), _stream(stream)))
+    return bt
+
+
+def bitwidth_loss(bt: torch.Tensor, b_target: float, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """One layer's term of Eq. 12 without lambda, as a one-element device tensor."""
+    _require_cuda(bt, out)
+    if out is None:
+        out = torch.empty(1, dtype=torch.float32, device=bt.device)
+    _check(load_library().gws_bitwidth_loss(bt.numel(), _ptr(bt), b_target, _ptr(out), _stream(stream)))
+    return out
+
+
+def bitwidth_grad(grad_bt: torch.Tensor, bt: torch.Tensor, b_init: float, b_target: float, lam: float = 0.0,
+                  grad_bi: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """dL'/db_i of one layer: (b_init - b_target) * (dL/db_t + lam / m * sign(b_t - b_target))."""
+    _require_cuda(grad_bt, bt, grad_bi)
+    if grad_bi is None:
+        grad_bi = torch.empty_like(grad_bt)
+    _check(load_library().gws_bitwidth_grad(bt.numel(), _ptr(grad_bt), _ptr(bt), b_init, b_target, lam, _ptr(grad_bi),
+                                            _stream(stream)))
+    return grad_bi
+
+
+def layer_seed(user_seed: int, layer: int) -> int:
+    """Seed of layer ``layer`` under ``user_seed`` (Section 3.6, "Managing seed"); host only."""
+    return int(load_library().gws_layer_seed(user_seed & 0xFFFFFFFFFFFFFFFF, layer))
 
 
 STATIC_MAX_TENSORS = 256   # GWS_STATIC_MAX_TENSORS of include/gws.h

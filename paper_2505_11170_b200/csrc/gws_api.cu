@@ -847,6 +847,53 @@ int gws_sample_fwd_multi_static(int n, const gws_desc* descs, const gws_multi_pt
   return run_multi(&plan, step, stream, false);
 }
 
+// ---- bit-width parametrisation and seeds (Section 3.6) ------------------------------------------------
+
+static unsigned elementwise_grid(int64_t n) {
+  const int64_t blocks = (n + 255) / 256;
+  return static_cast<unsigned>(std::min<int64_t>(blocks, 148 * 16));
+}
+
+int gws_bitwidth(int64_t n_groups, const float* bi, float b_init, float b_target, float* bt, void* stream) {
+  if (n_groups < 0) return GWS_ERR_SHAPE;
+  if (n_groups == 0) return GWS_OK;
+  if (bi == nullptr || bt == nullptr) return GWS_ERR_NULL;
+  if (!aligned(bi, 4) || !aligned(bt, 4)) return GWS_ERR_ALIGN;
+  gws::k_bitwidth<<<elementwise_grid(n_groups), 256, 0, static_cast<cudaStream_t>(stream)>>>(bi, b_init - b_target, b_target, bt,
+                                                                                           n_groups);
+  return check_launch("bit-width kernel");
+}
+
+int gws_bitwidth_loss(int64_t m, const float* bt, float b_target, float* loss_out, void* stream) {
+  if (m < 0) return GWS_ERR_SHAPE;
+  if (bt == nullptr && m > 0) return GWS_ERR_NULL;
+  if (loss_out == nullptr) return GWS_ERR_NULL;
+  if (!aligned(bt, 4) || !aligned(loss_out, 4)) return GWS_ERR_ALIGN;
+  if (m == 0) {
+    const cudaError_t err = cudaMemsetAsync(loss_out, 0, sizeof(float), static_cast<cudaStream_t>(stream));
+    return err == cudaSuccess ? GWS_OK : cuda_fail(err, "bit-width loss");
+  }
+  gws::k_bitwidth_loss<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(bt, b_target, loss_out, m);
+  return check_launch("bit-width loss kernel");
+}
+
+int gws_bitwidth_grad(int64_t m, const float* grad_bt, const float* bt, float b_init, float b_target, double lambda,
+                      float* grad_bi, void* stream) {
+  if (m < 0) return GWS_ERR_SHAPE;
+  if (m == 0) return GWS_OK;
+  if (grad_bt == nullptr || bt == nullptr || grad_bi == nullptr) return GWS_ERR_NULL;
+  if (!aligned(grad_bt, 4) || !aligned(bt, 4) || !aligned(grad_bi, 4)) return GWS_ERR_ALIGN;
+  gws::k_bitwidth_grad<<<elementwise_grid(m), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      grad_bt, bt, b_init - b_target, b_target, static_cast<float>(lambda / static_cast<double>(m)), grad_bi, m);
+  return check_launch("bit-width gradient kernel");
+}
+
+uint64_t gws_layer_seed(uint64_t user_seed, uint64_t layer) {
+  const gws::Words4 w = gws::philox4x32_10(static_cast<uint32_t>(layer), static_cast<uint32_t>(layer >> 32), 0u, 0u,
+                                           static_cast<uint32_t>(user_seed), static_cast<uint32_t>(user_seed >> 32));
+  return static_cast<uint64_t>(w.o[0]) | (static_cast<uint64_t>(w.o[1]) << 32);
+}
+
 // ---- diagnostics ----------------------------------------------------------------------------------
 
 void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed) {

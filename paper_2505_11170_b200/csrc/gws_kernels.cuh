@@ -1044,6 +1044,42 @@ __global__ void __launch_bounds__(256) k_noise_probe(uint32_t* __restrict__ sink
   }
 }
 
+// ---- bit-width parametrisation (Eq. 11), its loss term (Eq. 12) and the chain rule back to b_i ----------
+
+// b_t = fl(b_target + fl(b_i * delta)), delta = fl(b_init - b_target): one rounding per operation.
+__global__ void __launch_bounds__(256) k_bitwidth(const float* __restrict__ bi, float delta, float b_target, float* __restrict__ bt,
+                                                  int64_t n) {
+  for (int64_t k = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x; k < n; k += static_cast<int64_t>(gridDim.x) * 256)
+    st_f32(bt, k, __fadd_rn(b_target, __fmul_rn(ld_f32(bi, k), delta)));
+}
+
+// dL'/db_i = delta * (dL/db_t + lam_over_m * sign(b_t - b_target)); sign(0) = 0.
+__global__ void __launch_bounds__(256) k_bitwidth_grad(const float* __restrict__ grad_bt, const float* __restrict__ bt, float delta,
+                                                       float b_target, float lam_over_m, float* __restrict__ grad_bi, int64_t n) {
+  for (int64_t k = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x; k < n; k += static_cast<int64_t>(gridDim.x) * 256) {
+    const float x = __fsub_rn(ld_f32(bt, k), b_target);
+    const float sign = x > 0.0f ? 1.0f : (x < 0.0f ? -1.0f : 0.0f);
+    st_f32(grad_bi, k, __fmul_rn(delta, __fadd_rn(ld_f32(grad_bt, k), __fmul_rn(lam_over_m, sign))));
+  }
+}
+
+// mean_k |b_t,k - b_target| of one layer: one block, every thread a strided partial sum, combined in a fixed order.
+__global__ void __launch_bounds__(1024) k_bitwidth_loss(const float* __restrict__ bt, float b_target, float* __restrict__ out,
+                                                        int64_t m) {
+  __shared__ float red[32];
+  float acc = 0.0f;
+  for (int64_t k = threadIdx.x; k < m; k += 1024) acc += fabsf(__fsub_rn(ld_f32(bt, k), b_target));
+#pragma unroll
+  for (uint32_t o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+  if ((threadIdx.x & 31u) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float total = 0.0f;
+    for (int w = 0; w < 32; ++w) total += red[w];
+    st_f32(out, 0, total / static_cast<float>(m));
+  }
+}
+
 __global__ void __launch_bounds__(256) k_philox_words(uint4* __restrict__ out, uint64_t n_vec, uint64_t first_vec,
                                                       uint32_t seed_lo, uint32_t seed_hi, uint32_t step_lo,
                                                       uint32_t step_hi) {
