@@ -36,11 +36,13 @@
  *     computed in double then rounded to float otherwise.
  *   - sample: y = fl32( float(w) + float(R) * scale_g ) (the product is exact, no FMA
  *     contraction), w_hat = IEEE round-to-nearest-even of y to BF16.  R == 0 adds +0.0.
- *   - Fast kernels need: 16-byte aligned tensor pointers, cols % 8 == 0, ld == cols,
- *     elem_offset % 8 == 0, group_rows == 1 and group_cols in {8,16,32,64,128,256} dividing
- *     cols, or whole-row groups with cols <= 65536.  Every other legal shape (ragged groups,
- *     ld > cols, the paper's 32x32 square blocks, odd cols) runs on a slower general kernel
- *     with identical results.
+ *   - Fast kernels cover dense tensors (ld == cols) with 16-byte aligned pointers, cols % 8 == 0,
+ *     elem_offset % 8 == 0 and: group_rows == 1 with group_cols in {8,16,32,64,128,256} dividing
+ *     cols; whole-row groups with cols <= 65536; the paper's 32 x 32 blocks when rows and cols are
+ *     multiples of 32.  They are fastest with 32-byte aligned pointers (and, for whole rows, cols a
+ *     multiple of 32 up to 32768).  Every other legal shape (ragged groups, ld > cols, other 2-D
+ *     groups, odd cols, a tensor whose element indices straddle a multiple of 2^35) runs on a
+ *     slower general kernel with identical results.
  *   - NaN / Inf in the inputs give unspecified values but never a fault.
  *
  * Every function returns 0 (GWS_OK) or a negative gws_status.  Arguments are validated on
