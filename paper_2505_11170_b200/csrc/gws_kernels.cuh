@@ -216,18 +216,25 @@ __device__ __forceinline__ uint4 sample_vec(const uint4& w, const Words4& r, con
   return make_uint4(sample_pair(w.x, p[0], k), sample_pair(w.y, p[1], k), sample_pair(w.z, p[2], k), sample_pair(w.w, p[3], k));
 }
 
-// acc + sum over the vector of float(g) * 2R, accumulated in element-pair order (low, high).
-__device__ __forceinline__ float dot_pair(uint32_t g, uint32_t pair, float acc) {
-  acc = __fmaf_rn(__uint_as_float(g << 16), __uint_as_float(pair << 16), acc);
-  return fma_bf16(hi16(g), hi16(pair), acc);
+// Running sum of float(g) * 2R: low and high BF16 halves of every pair go to their own accumulator
+// (two independent FMA chains), both through fma.rn.f32.bf16, which widens the operands exactly
+// and takes them straight from the halves of the 32-bit words.  The order is fixed, so results
+// repeat bit for bit.
+struct DotAcc {
+  float lo = 0.0f, hi = 0.0f;
+  __device__ __forceinline__ float total() const { return __fadd_rn(lo, hi); }
+};
+__device__ __forceinline__ void dot_pair(uint32_t g, uint32_t pair, DotAcc& acc) {
+  acc.lo = fma_bf16(static_cast<uint16_t>(g & 0xFFFFu), static_cast<uint16_t>(pair & 0xFFFFu), acc.lo);
+  acc.hi = fma_bf16(hi16(g), hi16(pair), acc.hi);
 }
-__device__ __forceinline__ float dot_vec(const uint4& g, const Words4& r, float acc) {
+__device__ __forceinline__ void dot_vec(const uint4& g, const Words4& r, DotAcc& acc) {
   uint32_t p[4];
   decode8(r, p);
-  acc = dot_pair(g.x, p[0], acc);
-  acc = dot_pair(g.y, p[1], acc);
-  acc = dot_pair(g.z, p[2], acc);
-  return dot_pair(g.w, p[3], acc);
+  dot_pair(g.x, p[0], acc);
+  dot_pair(g.y, p[1], acc);
+  dot_pair(g.z, p[2], acc);
+  dot_pair(g.w, p[3], acc);
 }
 // dL/db_t of a group from its scale and the sum of g * 2R.
 __device__ __forceinline__ float grad_bt_of(float scale, float sum_g_2r) {
@@ -373,12 +380,13 @@ __device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t first_chunk
     const bool writer = ok[i] && writer_lane;
     const uint32_t v0 = e.vec_lo + chunk[i] * 4u;
     if (MODE == kBwd) {
-      float acc = 0.0f;
+      DotAcc dot;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
-        acc = dot_vec(make_uint4(c[i].x[4 * k], c[i].x[4 * k + 1], c[i].x[4 * k + 2], c[i].x[4 * k + 3]), r, acc);
+        dot_vec(make_uint4(c[i].x[4 * k], c[i].x[4 * k + 1], c[i].x[4 * k + 2], c[i].x[4 * k + 3]), r, dot);
       }
+      float acc = dot.total();
       for (uint32_t o = 1; o < lanes; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
       if (writer) st_f32(e.gout, g, grad_bt_of(gv[i], acc));
       if (ok[i] && e.out != nullptr) store_chunk<USE32>(e.out, chunk[i], 4, c[i]);
@@ -428,11 +436,13 @@ __device__ __forceinline__ void flat_narrow(const FlatRec& e, uint32_t chunk, ui
     const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
     if (MODE == kBwd) {
       if (writer) {
-        float acc = dot_vec(xv, r, 0.0f);
+        DotAcc dot;
+        dot_vec(xv, r, dot);
         if (ll == 1u) {
           const Words4 r2 = philox4x32_10_pre(v0 + mate, e.k0, e.k1, e.pre);
-          acc = dot_vec(make_uint4(c.x[4 * mate], c.x[4 * mate + 1], c.x[4 * mate + 2], c.x[4 * mate + 3]), r2, acc);
+          dot_vec(make_uint4(c.x[4 * mate], c.x[4 * mate + 1], c.x[4 * mate + 2], c.x[4 * mate + 3]), r2, dot);
         }
+        const float acc = dot.total();
         st_f32(e.gout, g, grad_bt_of(ld_f32(e.gin, g), acc));
       }
       continue;
@@ -561,12 +571,13 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
     const uint32_t chunk = row_chunk0 + q[i];
     const uint32_t v0 = e.vec_lo + chunk * 4u;
     if (MODE == kBwd) {
-      float acc = 0.0f;
+      DotAcc dot;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
-        acc = dot_vec(make_uint4(c[i].x[4 * k], c[i].x[4 * k + 1], c[i].x[4 * k + 2], c[i].x[4 * k + 3]), r, acc);
+        dot_vec(make_uint4(c[i].x[4 * k], c[i].x[4 * k + 1], c[i].x[4 * k + 2], c[i].x[4 * k + 3]), r, dot);
       }
+      float acc = dot.total();
 #pragma unroll
       for (uint32_t o = 1; o < 32u; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
       if (lane == 0u) st_f32(e.gout, g, grad_bt_of(gv[i], acc));
@@ -689,7 +700,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
   const uint32_t span = BLOCK ? 32u : tpr;   // lanes of this warp that share the row
 
   if (MODE == kBwd) {
-    float acc = 0.0f;
+    DotAcc dot;
 #pragma unroll
     for (int k = 0; k < MAXCPT; ++k) {
       if (!ok[k]) continue;
@@ -698,10 +709,11 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
 #pragma unroll
       for (int v = 0; v < 4; ++v) {
         const Words4 r = philox4x32_10_pre(v0 + v, e.k0, e.k1, e.pre);
-        acc = dot_vec(make_uint4(c[k].x[4 * v], c[k].x[4 * v + 1], c[k].x[4 * v + 2], c[k].x[4 * v + 3]), r, acc);
+        dot_vec(make_uint4(c[k].x[4 * v], c[k].x[4 * v + 1], c[k].x[4 * v + 2], c[k].x[4 * v + 3]), r, dot);
       }
       if (okr && e.out != nullptr) store_chunk<true>(e.out, chunk, 4, c[k]);
     }
+    float acc = dot.total();
     for (uint32_t o = 1; o < span; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
     if (BLOCK) {
       if (lane == 0) red_f[warp] = acc;
@@ -802,17 +814,18 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
   const float gvr = (MODE != kAbsmax && okr) ? ld_f32(e.gin, row) : 0.0f;
 
   if (MODE == kBwd) {
-    float acc = 0.0f;
+    DotAcc dot;
 #pragma unroll
     for (int k = 0; k < V; ++k) {
       if (k * 32u < vpr) {
         const uint32_t j = k * 32u + lane;
         const bool ok = okr && j < vpr;
         // vectors past the end of the row are all zero and add nothing
-        acc = dot_vec(x[k], philox_vec(e, vbase + j, step_lo, step_hi), acc);
+        dot_vec(x[k], philox_vec(e, vbase + j, step_lo, step_hi), dot);
         if (ok && e.out != nullptr) st_vec(e.out, vbase + j, x[k]);
       }
     }
+    float acc = dot.total();
 #pragma unroll
     for (uint32_t o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
     if (okr && lane == 0) st_f32(e.gout, row, grad_bt_of(gvr, acc));
@@ -868,15 +881,16 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
   const float gvr = (MODE != kAbsmax) ? ld_f32(e.gin, row) : 0.0f;
 
   if (MODE == kBwd) {
-    float acc = 0.0f;
+    DotAcc dot;
 #pragma unroll
     for (int k = 0; k < V; ++k) {
       if (static_cast<uint32_t>(k) * T < vpr) {
         const uint32_t j = k * T + threadIdx.x;
-        acc = dot_vec(x[k], philox_vec(e, vbase + j, step_lo, step_hi), acc);   // zero vectors past the row add nothing
+        dot_vec(x[k], philox_vec(e, vbase + j, step_lo, step_hi), dot);   // zero vectors past the row add nothing
         if (j < vpr && e.out != nullptr) st_vec(e.out, vbase + j, x[k]);
       }
     }
+    float acc = dot.total();
 #pragma unroll
     for (uint32_t o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
     if (lane == 0) red_f[warp] = acc;
