@@ -350,24 +350,30 @@ int launch_squares(const std::vector<const Entry*>& entries, uint64_t step, cuda
   return GWS_OK;
 }
 
-template <int MODE, bool MULTI>
-int launch_as(int cls, const Entry& single, const Entry* table, int n_or_index, unsigned grid, uint32_t lo, uint32_t hi,
-              cudaStream_t stream) {
+// One tensor on the vector kernels (row classes) or the general kernel.  The general kernel alone also
+// reads its tensor from the device table (entry `index`) in multi-tensor plans.
+template <int MODE>
+int launch_single(int cls, const Entry& single, unsigned grid, uint32_t lo, uint32_t hi, cudaStream_t stream) {
   switch (cls) {
     case gws::kRowWarp:
-      gws::k_row_warp<MODE, MULTI><<<grid, gws::kRowWarpThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      gws::k_row_warp<MODE, false><<<grid, gws::kRowWarpThreads, 0, stream>>>(single, nullptr, 0, lo, hi);
       return check_launch("warp-per-row kernel");
     case gws::kRowCta:
-      gws::k_row_cta<MODE, MULTI><<<grid, gws::kRowCtaThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      gws::k_row_cta<MODE, false><<<grid, gws::kRowCtaThreads, 0, stream>>>(single, nullptr, 0, lo, hi);
       return check_launch("block-per-row kernel");
     default:
-      gws::k_general<MODE, MULTI><<<grid, gws::kGeneralThreads, 0, stream>>>(single, table, n_or_index, lo, hi);
+      gws::k_general<MODE, false><<<grid, gws::kGeneralThreads, 0, stream>>>(single, nullptr, 0, lo, hi);
       return check_launch("general kernel");
   }
 }
+template <int MODE>
+int launch_general_from_table(const Entry& none, const Entry* table, int index, unsigned grid, uint32_t lo, uint32_t hi,
+                              cudaStream_t stream) {
+  gws::k_general<MODE, true><<<grid, gws::kGeneralThreads, 0, stream>>>(none, table, index, lo, hi);
+  return check_launch("general kernel");
+}
 
-// table == nullptr: one tensor, described by `single`; otherwise entry n_or_index (general class) or the
-// n_or_index entries (other classes) of `table`.
+// table == nullptr: one tensor, described by `single`; otherwise entry n_or_index of `table` (general class only).
 template <int MODE>
 int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int64_t tiles, uint64_t step,
            cudaStream_t stream) {
@@ -382,8 +388,8 @@ int launch(int cls, const Entry& single, const Entry* table, int n_or_index, int
   }
   const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
   const unsigned grid = static_cast<unsigned>(tiles);
-  return table == nullptr ? launch_as<MODE, false>(cls, single, table, n_or_index, grid, lo, hi, stream)
-                          : launch_as<MODE, true>(cls, single, table, n_or_index, grid, lo, hi, stream);
+  return table == nullptr ? launch_single<MODE>(cls, single, grid, lo, hi, stream)
+                          : launch_general_from_table<MODE>(single, table, n_or_index, grid, lo, hi, stream);
 }
 
 // Shared checks of the single-tensor calls.  Returns 1 if there is nothing to do.
