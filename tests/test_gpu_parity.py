@@ -313,6 +313,19 @@ def test_multi_tensor_launch_mixed_classes():
     assert plan.launches_per_pass == 6
 
 
+def test_multi_tensor_plan_larger_than_one_parameter_block():
+    # more tensors of a kind than one launch carries in its parameters (192 flat-group, 168 whole-row records):
+    # the plan splits them over several launches and every tensor still matches the oracle
+    T = syn.TensorSpec
+    specs = ([T(f"f{k}", 8 + k % 5, 256, 1, 128) for k in range(200)] + [T(f"n{k}", 3, 48, 1, 16) for k in range(5)] +
+             [T(f"r{k}", 4 + k % 3, 96, 1, 0) for k in range(180)] + [T(f"b{k}", 2, 8192, 1, 0) for k in range(3)] +
+             [T(f"s{k}", 32, 64, 32, 32) for k in range(6)])
+    plan = _run_multi_against_oracle(specs, steps=(5,), with_copy=False)
+    assert list(plan.plan.count) == [205, 180, 3, 6]
+    # flat 200 -> 2, narrow 5 -> 1, shared rows 180 -> 2, block rows 3 -> 1, squares 6 -> 1
+    assert plan.launches_per_pass == 7
+
+
 def test_multi_tensor_empty_entries_and_forward_only():
     T = syn.TensorSpec
     specs = [T("a", 8, 256, 1, 128), T("z", 0, 256, 1, 128), T("b", 8, 768, 1, 0)]
