@@ -137,3 +137,31 @@ def test_config4_stress_sweep(shape):
                 # the outliers are there and the absmax sees them
                 am = gws.group_absmax(d, w)
                 assert float(am.max()) >= 7.9 * sigma
+
+
+def test_config5_sample_then_gemm_unfused():
+    # Up-projection of the Llama2-1B shape: W 5632 x 2048 (rows = outputs), groups of 128, 6 bits; X 16384 x 2048.
+    # The sampled weight is checked bit for bit on row slices; Y = X W_hat^T (the stock BF16 GEMM the paper keeps) is
+    # checked on sampled outputs against a float64 dot product with the oracle's W_hat.
+    spec = syn.TensorSpec("up", 5632, 2048, 1, 128)
+    w = syn.weights(spec, 0, device=DEV)
+    bt = syn.bitwidths(spec, 0, fixed=6.0, device=DEV)
+    d = Desc.make(spec.rows, spec.cols, 1, 128, seed=syn.layer_seed(5, 0), step=0)
+    w_hat, sc = gws.sample_fwd(d, w, bt)
+    x = torch.randn(16384, 2048, generator=torch.Generator().manual_seed(3)).to(torch.bfloat16).to(DEV)
+    y = torch.matmul(x, w_hat.t())
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(5)
+    for r0 in (0, spec.rows - 16, int(rng.integers(0, spec.rows - 16))):
+        _slice_check(spec, d.seed, 0, w, bt, w_hat, sc, None, None, r0, 16)
+    rows = sorted({0, spec.rows - 1, *[int(v) for v in rng.integers(0, spec.rows, 6)]})
+    for n in rows:
+        hat, _ = orc.sample_fwd(bits_of(w[n:n + 1]), bt[n * 16:(n + 1) * 16].cpu().numpy(), 1, spec.cols, 1, 128, seed=d.seed,
+                                step=0, elem_offset=n * spec.cols)
+        wn = (hat.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        for m in (0, 16383, int(rng.integers(0, 16384))):
+            want = float(x[m].double().cpu().numpy() @ wn)
+            got = float(y[m, n])
+            # BF16 output rounding (2^-8 relative, with margin) plus FP32 accumulation error relative to sum |x||w|
+            budget = 2.0 ** -8 * abs(want) + 1e-5 * float(np.abs(x[m].double().cpu().numpy()) @ np.abs(wn)) + 1e-30
+            assert abs(got - want) <= budget, (m, n, got, want)
