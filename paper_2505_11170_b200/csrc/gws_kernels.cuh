@@ -1,26 +1,31 @@
 // Device code of the sampling pass for sm_100a.
 //
 // The pass is elementwise plus a small per-group reduction.  Its algorithmic cost is 4 bytes per
-// element forward and 2 backward, but every element also needs 16 random bits, so the instruction
-// issue rate (Philox4x32-10: 20 wide multiplies + 20 three-input XORs per 8 elements; the AND / OR
-// decode; the FP32 add) is the ceiling that binds before HBM does for backward and close to it for
-// forward.  The kernels are therefore written for instruction count first:
+// element forward and 2 backward, but every element also needs 16 random bits (Philox4x32-10: 18
+// wide multiplies + 19 three-input XORs per 8 elements once the launch-uniform part is hoisted).
+// On B200 that generation alone runs at about 2.8 T elements/s: well above the HBM bound of the
+// forward pass (1.6 T), below that of the backward pass (3.1 T).  So forward is HBM-bound, backward
+// is bound by instruction issue, and everything besides Philox is written for instruction count:
 //
 //   * one Philox call and one whole-word decode serve the 8 elements of a 16-byte vector;
-//   * the noise reaches the FP32 pipe as a BF16 bit pattern (2R), low halves widened by a shift,
-//     high halves consumed directly by the mixed-precision add / fma of sm_100;
-//   * a thread owns 64 contiguous bytes (4 vectors) of a flat group, loaded with two 32-byte loads,
-//     so a group of 128 elements is 4 lanes and needs two shuffle steps;
-//   * |w| maxima are taken on packed BF16 pairs (max.xorsign.abs), never widened.
+//   * the noise reaches the FP32 pipe as a BF16 bit pattern (2R); high halves (and in backward
+//     both halves) are consumed directly by the mixed-precision add / fma of sm_100;
+//   * a thread owns 64 contiguous bytes (a chunk: 4 vectors, 32 elements), moved with two 32-byte
+//     accesses, so a group of 128 elements is 4 lanes and needs two shuffle steps;
+//   * |w| maxima are taken on packed BF16 pairs (max.xorsign.abs), never widened;
+//   * the tensors of a launch are described by compact records passed BY VALUE in the kernel
+//     parameters, so a thread block (a few microseconds of work) finds its tensor without a
+//     global-memory access.
 //
-// Four tilings:
-//   flat      group = 8 << k contiguous elements (k = 0..5) of a dense tensor: the tensor is a flat
-//             run of 64-byte chunks, one per thread; groups up to a chunk live inside the thread.
-//   row-warp  group = one row of up to 4096 elements: one warp per row, up to 16 vectors per lane
-//             kept in registers between the max and the add (single pass over W).
-//   row-cta   group = one row of up to 65536 elements: one 512-thread block per row.
-//   general   every other shape: one block per group, scalar accesses.
-// All kernels read their tensor from a table so that one launch serves many tensors.
+// Kernels:
+//   k_flat    group = 8 << k contiguous elements (k = 0..5) of a dense tensor: the tensor is a flat
+//             run of chunks; groups up to a chunk live inside the thread.
+//   k_row     group = one row (a multiple of 32 elements, up to 32768): 1..32 lanes or one block
+//             share a row, whose chunks stay in registers between the max and the add.
+//   k_square  group = the paper's 32 x 32 block: a warp per block, lane = row.
+//   k_row_warp / k_row_cta   whole rows the chunk kernel does not take (16-byte vectors), one tensor
+//             per launch;  k_general  every other shape: one block per group, scalar accesses,
+//             tensor record read from a device table in multi-tensor plans.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -33,7 +38,8 @@ namespace gws {
 enum Mode { kAbsmax = 0, kFwd = 1, kBwd = 2 };
 enum KernelClass { kFlat = 0, kRowWarp = 1, kRowCta = 2, kGeneral = 3 };
 
-// One tensor of a launch.  `in`/`out`/`gin`/`gout` change meaning with the mode:
+// Full description of one tensor: the record of the multi-tensor tables and the parameter of the
+// vector and general kernels.  `in`/`out`/`gin`/`gout` change meaning with the mode:
 //   absmax: in = w,           gout = absmax
 //   fwd:    in = w,           out = w_hat,           gin = bt,    gout = scale_out or null
 //   bwd:    in = grad_w_hat,  out = grad_w or null,  gin = scale, gout = grad_bt
