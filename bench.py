@@ -43,15 +43,23 @@ def measured_peaks():
 
 
 PROFILE = os.path.join(ROOT, "profiles", "k_flat_llama2_1b_g128.md")
-KERNEL_SOURCES = [os.path.join(ROOT, "paper_2505_11170_b200", "csrc", f) for f in ("gws_api.cu", "gws_kernels.cuh", "gws_math.cuh")]
+CSRC = os.path.join(ROOT, "paper_2505_11170_b200", "csrc")
 
 
 def kernel_source_hash() -> str:
+    """Hash of the device code (comments and white space removed) and of the tile-shape macros of the host file:
+    what has to be unchanged for ncu counters to still describe the kernels."""
     import hashlib
+    import re
     h = hashlib.sha256()
-    for path in KERNEL_SOURCES:
-        with open(path, "rb") as f:
-            h.update(f.read())
+    for name in ("gws_kernels.cuh", "gws_math.cuh"):
+        with open(os.path.join(CSRC, name)) as f:
+            text = f.read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", "", text)
+        h.update(re.sub(r"\s+", " ", text).encode())
+    with open(os.path.join(CSRC, "gws_api.cu")) as f:
+        h.update(" ".join(sorted(re.findall(r"#define\s+GWS_FLAT_CPT_\w+\s+\d+", f.read()))).encode())
     return h.hexdigest()[:16]
 
 
