@@ -220,6 +220,19 @@ def test_nan_and_inf_inputs_never_fault(case):
         assert torch.equal(w_hat[-1].view(torch.int16), clean_hat[-1].view(torch.int16))
 
 
+@pytest.mark.parametrize("case", [(131, 2048, 1, 128, None), (50, 160, 1, 32, None), (21, 768, 1, 0, None), (5, 8192, 1, 0, None),
+                                  (96, 608, 32, 32, None), (70, 520, 1, 0, None), (33, 40, 32, 32, None)])
+def test_backward_reductions_repeat_bit_for_bit(case):
+    # fixed summation order, no atomics: two runs give identical bits (and a race in a reduction would not)
+    rows, cols, gr, gc, ld = case
+    d = _desc(case)
+    g = _make(rows, cols, ld, 51, sigma=1e-4).to(DEV)
+    sc = torch.rand(gws.n_groups(d), device=DEV) * 1e-3
+    runs = [gws.sample_bwd(d, g, sc)[1].clone() for _ in range(3)]
+    assert torch.equal(runs[0].view(torch.int32), runs[1].view(torch.int32))
+    assert torch.equal(runs[0].view(torch.int32), runs[2].view(torch.int32))
+
+
 def test_elem_offset_reproduces_the_unsharded_tensor():
     rows, cols = 64, 512
     w = _make(rows, cols, None, 8)
