@@ -205,21 +205,48 @@ __device__ __forceinline__ Scale make_scale(float s) {
   k.tiny = s < 0x1p-120f;
   return k;
 }
+template <bool TINY>
 __device__ __forceinline__ float noise_term(float two_r, const Scale& k) {
-  return k.tiny ? __fmul_rn(__fmul_rn(two_r, 0.5f), k.s) : __fmul_rn(two_r, k.half);
+  return TINY ? __fmul_rn(__fmul_rn(two_r, 0.5f), k.s) : __fmul_rn(two_r, k.half);
 }
 
 // Eq. 3 + cast for one pair word: 2 x ( bf16_rne( fl32(w + R*s) ) ).  R*s is exact, the add rounds
 // once in FP32 (a separate instruction: never contracted), the pack rounds to nearest even.
-__device__ __forceinline__ uint32_t sample_pair(uint32_t w, uint32_t pair, const Scale& k) {
-  const float ql = noise_term(__uint_as_float(pair << 16), k);
-  const float qh = noise_term(__uint_as_float(pair & 0xFFFF0000u), k);
+template <bool TINY>
+__device__ __forceinline__ uint32_t sample_pair_t(uint32_t w, uint32_t pair, const Scale& k) {
+  const float ql = noise_term<TINY>(__uint_as_float(pair << 16), k);
+  const float qh = noise_term<TINY>(__uint_as_float(pair & 0xFFFF0000u), k);
   return pack_bf16_rne(__fadd_rn(__uint_as_float(w << 16), ql), add_bf16(hi16(w), qh));
 }
-__device__ __forceinline__ uint4 sample_vec(const uint4& w, const Words4& r, const Scale& k) {
+template <bool TINY>
+__device__ __forceinline__ uint4 sample_vec_t(const uint4& w, const Words4& r, const Scale& k) {
   uint32_t p[4];
   decode8(r, p);
-  return make_uint4(sample_pair(w.x, p[0], k), sample_pair(w.y, p[1], k), sample_pair(w.z, p[2], k), sample_pair(w.w, p[3], k));
+  return make_uint4(sample_pair_t<TINY>(w.x, p[0], k), sample_pair_t<TINY>(w.y, p[1], k), sample_pair_t<TINY>(w.z, p[2], k),
+                    sample_pair_t<TINY>(w.w, p[3], k));
+}
+// The tiny-scale form is chosen once per vector / chunk (it is a property of the group), so the common
+// path carries one multiply per element.
+__device__ __forceinline__ uint4 sample_vec(const uint4& w, const Words4& r, const Scale& k) {
+  return k.tiny ? sample_vec_t<true>(w, r, k) : sample_vec_t<false>(w, r, k);
+}
+// One 64-byte chunk whose first vector has the (low) Philox counter word v0.
+template <bool TINY>
+__device__ __forceinline__ void sample_chunk_t(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
+                                               const Scale& sc, uint32_t* y) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const Words4 r = philox4x32_10_pre(v0 + k, k0, k1, pre);
+    uint32_t p[4];
+    decode8(r, p);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) y[4 * k + j] = sample_pair_t<TINY>(x[4 * k + j], p[j], sc);
+  }
+}
+__device__ __forceinline__ void sample_chunk(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
+                                             const Scale& sc, uint32_t* y) {
+  if (sc.tiny) sample_chunk_t<true>(x, v0, k0, k1, pre, sc, y);
+  else sample_chunk_t<false>(x, v0, k0, k1, pre, sc, y);
 }
 
 // Running sum of float(g) * 2R: low and high BF16 halves of every pair go to their own accumulator
@@ -408,14 +435,7 @@ __device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t first_chunk
     }
     const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv[i])));
     Chunk y;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
-      uint32_t p[4];
-      decode8(r, p);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) y.x[4 * k + j] = sample_pair(c[i].x[4 * k + j], p[j], sc);
-    }
+    sample_chunk(c[i].x, v0, e.k0, e.k1, e.pre, sc, y.x);
     if (ok[i]) {
       store_chunk<USE32>(e.out, chunk[i], 4, y);
       if (writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
@@ -601,14 +621,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
     }
     const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv[i])));
     Chunk y;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
-      uint32_t p[4];
-      decode8(r, p);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) y.x[4 * k + j] = sample_pair(c[i].x[4 * k + j], p[j], sc);
-    }
+    sample_chunk(c[i].x, v0, e.k0, e.k1, e.pre, sc, y.x);
     store_chunk<true>(e.out, chunk, 4, y);
     if (lane == 0u && e.gout != nullptr) st_f32(e.gout, g, sc.s);
   }
@@ -757,14 +770,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
     const uint32_t chunk = row_chunk0 + static_cast<uint32_t>(k) * tpr + t;
     const uint32_t v0 = e.vec_lo + chunk * 4u;
     Chunk y;
-#pragma unroll
-    for (int v = 0; v < 4; ++v) {
-      const Words4 r = philox4x32_10_pre(v0 + v, e.k0, e.k1, e.pre);
-      uint32_t p[4];
-      decode8(r, p);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) y.x[4 * v + j] = sample_pair(c[k].x[4 * v + j], p[j], sc);
-    }
+    sample_chunk(c[k].x, v0, e.k0, e.k1, e.pre, sc, y.x);
     if (okr) store_chunk<true>(e.out, chunk, 4, y);
   }
   if (okr && t == 0u && e.gout != nullptr) st_f32(e.gout, row, sc.s);
