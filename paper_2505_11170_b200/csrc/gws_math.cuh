@@ -21,10 +21,18 @@ struct Words4 {
   uint32_t o[4];
 };
 
+// Rounds of the Philox4x32 block function.  The library, its oracle and every test use 10.  The switch
+// exists only to measure how much of the backward pass is random-bit generation (a build with another
+// value has no oracle to be checked against).
+#ifndef GWS_PHILOX_ROUNDS
+#define GWS_PHILOX_ROUNDS 10
+#endif
+static_assert(GWS_PHILOX_ROUNDS >= 2, "the hoisted form below takes rounds 1 and 2 apart");
+
 // Ten rounds of the Philox4x32 block function.  Counter (c0..c3), key (k0, k1).
 GWS_HD Words4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1) {
 #pragma unroll
-  for (int r = 0; r < 10; ++r) {
+  for (int r = 0; r < GWS_PHILOX_ROUNDS; ++r) {
     const uint64_t p0 = static_cast<uint64_t>(kPhiloxM0) * c0;
     const uint64_t p1 = static_cast<uint64_t>(kPhiloxM1) * c2;
     // round key r is k + r*W (mod 2^32); r*W folds to a constant after unrolling
@@ -81,7 +89,7 @@ GWS_HD Words4 philox4x32_10_pre(uint32_t v_lo, uint32_t k0, uint32_t k1, const P
   c2 = c3 ^ q.y2;
   c3 = q.l3;
 #pragma unroll
-  for (int r = 2; r < 10; ++r) {
+  for (int r = 2; r < GWS_PHILOX_ROUNDS; ++r) {
     const uint64_t p0 = static_cast<uint64_t>(kPhiloxM0) * c0;
     const uint64_t p1 = static_cast<uint64_t>(kPhiloxM1) * c2;
     const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ (k0 + static_cast<uint32_t>(r) * kPhiloxW0);
