@@ -129,9 +129,9 @@ int gws_sample_bwd(const gws_desc* desc, const void* grad_w_hat, const float* sc
 
 /* ---- many tensors per launch ---------------------------------------------------------------
  * One linear layer of a 1B-parameter model is a few microseconds of HBM time, so a training
- * step samples all layers with one launch per kernel class.  The tensor set is described
- * once (gws_multi_prepare uploads a table into caller-owned device workspace); each step then
- * calls gws_sample_fwd_multi / gws_sample_bwd_multi with only the step counter changing.
+ * step samples all layers with as few launches as possible: tensors that run on the same kernel
+ * share a launch.  The tensor set is described once (gws_multi_prepare); each step then calls
+ * gws_sample_fwd_multi / gws_sample_bwd_multi with only the step counter changing.
  */
 
 /* Host arrays of n device pointers each; the meaning of every pointer is that of the
@@ -153,9 +153,9 @@ typedef struct gws_multi_plan {
   const void* host_tables; /* the host copy of the tables (host_workspace of gws_multi_prepare)          */
   int32_t n_tensors;
   int32_t has_fwd, has_bwd;
-  int32_t count[4];     /* tensors per kernel class: flat groups, warp-per-row, CTA-per-row, general */
-  int64_t tiles[4];     /* thread-block tiles per class                                             */
-  int64_t fwd_offset[4], bwd_offset[4]; /* byte offsets of the class tables inside workspace         */
+  int32_t count[4];     /* tensors per class: flat groups, rows <= 4096, rows <= 65536, general (gws_kernel_class) */
+  int64_t tiles[4];     /* size of each class in its table's units: 1024-vector tiles, 8-row tiles, rows, blocks  */
+  int64_t fwd_offset[4], bwd_offset[4]; /* byte offsets of the class tables inside both workspaces          */
   int64_t total_elements;
 } gws_multi_plan;
 
@@ -167,10 +167,11 @@ size_t gws_workspace_bytes(int n_tensors);
  * Validate n descriptors and pointer sets, build the tile tables, keep one copy in `host_workspace`
  * (HOST memory, caller-owned, at least gws_workspace_bytes(n)) and copy them into `workspace`
  * (DEVICE memory) on `stream`; the call waits for that copy, so call it outside the training loop.
- * desc[i].step is ignored.  Both workspaces must stay untouched for as long as the plan is used:
- * row and general kernels read their tensor records from the device copy; flat-group launches
- * (groups of 8..256 contiguous elements) take theirs from the host copy and pass up to 240 of them
- * by value in the kernel parameters, so that a thread block finds its tensor without a memory access.
+ * desc[i].step is ignored.  Both workspaces must stay untouched for as long as the plan is used.
+ * Launches take their tensor records from the host copy and pass them by value in the kernel
+ * parameters (up to 192 flat-group or 168 whole-row records per launch), so that a thread block
+ * finds its tensor without a memory access; only the general kernel (ragged groups, padded rows,
+ * odd shapes) reads its record from the device copy.
  */
 int gws_multi_prepare(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs, void* workspace,
                       size_t workspace_bytes, void* host_workspace, size_t host_workspace_bytes,
