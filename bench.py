@@ -32,6 +32,7 @@ WORKLOAD = "llama2_1b_linear_set_g128"
 FWD_BYTES_PER_ELEM = 2 + 2 + 8 / 128      # read w, write w_hat, read b_t + write scale per 128 elements
 BWD_BYTES_PER_ELEM = 2 + 8 / 128          # read dL/dw_hat, read scale + write dL/db_t per 128 elements
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0                   # B200 HBM3e data-sheet figure, for context beside the measured copy peak
 
 
 def measured_peaks():
@@ -395,9 +396,10 @@ def main():
                    "bits": "uniform integers 4..9", "passes": "forward + backward (identity grad_w), one launch each",
                    "l2": "inputs larger than L2: each pass streams %.2f GB" % (n_elem * 2 / 1e9),
                    "multi_gpu": "replicas only (no exchange step in the path)"},
-        "gelem_per_s": gelem, "hbm_frac": value / world / peak,
+        "gelem_per_s": gelem, "hbm_frac": value / world / peak, "hbm_frac_of_nominal_8000": value / world / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "k_flat<fwd> (gws_sample_fwd_multi)", "achieved": fwd_gbs, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": fwd_gbs / peak, "ms_per_launch": fwd_ms,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": fwd_gbs / peak, "frac_of_nominal_8000": fwd_gbs / NOMINAL_HBM_GBS,
+                     "ms_per_launch": fwd_ms,
                      "algorithmic_bytes_per_launch": fwd_bytes, "traffic": traffic.get("fwd_bytes_per_launch")},
         "roofline_bwd": {"bound": "hbm", "kernel": "k_flat<bwd> (gws_sample_bwd_multi)", "achieved": bwd_gbs, "peak": peak,
                          "unit": "GB/s", "frac": bwd_gbs / peak, "ms_per_launch": bwd_ms,
