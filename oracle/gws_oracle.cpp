@@ -44,7 +44,9 @@
 // Pins (tests/test_oracle_*.py): Philox known-answer vectors; exhaustive
 // decode counts against Eq. 10; closed-form moments; KS / chi-square over
 // 10^7 draws; hand-computed add-then-cast cases; library BF16 casts;
-// finite-difference gradients; the Lemma 1 and Proposition 2 invariants.
+// finite-difference gradients; the Lemma 1 and Proposition 2 invariants;
+// the given-scale forward against the fused one and a numpy restatement, and
+// the facts a sharded pass rests on (partial maxima, partial sums).
 // The only thing left unpinned is which of the equally valid bit assignments
 // the authors' own kernels used; their stream cannot be reproduced.
 
@@ -289,6 +291,24 @@ void gwso_sample_fwd(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows,
     }
   if (scale_out)
     for (int64_t g = 0; g < geo.n_groups; ++g) scale_out[g] = scale_of(absmax_scratch[g], bt[g]);
+}
+
+// Eq. 3 + cast for a tensor whose group maxima were taken elsewhere: scale[g]
+// is s_g = max_g|w| * 2^(1 - b_g) as the caller has it (for a tensor cut into
+// shards the maximum runs over the whole group, parts held by other shards
+// included).  Same noise, add and cast as gwso_sample_fwd; nothing is reduced.
+void gwso_sample_fwd_scaled(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols,
+                            uint64_t seed, uint64_t step, uint64_t elem_offset, const uint16_t* w,
+                            const float* scale, uint16_t* w_hat) {
+  const Geometry geo = make_geometry(rows, cols, ld, group_rows, group_cols);
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const uint64_t e = elem_offset + static_cast<uint64_t>(i * cols + j);
+      const int r = noise_of_element(seed, step, e);
+      const float pqn = static_cast<float>(r) * scale[group_of(geo, i, j)];
+      const float y = bf16_to_f32(w[i * ld + j]) + pqn;
+      w_hat[i * ld + j] = f32_to_bf16_rne(y);
+    }
 }
 
 // Eq. 4 with R supplied.  grad_w (may be null) receives the upstream gradient

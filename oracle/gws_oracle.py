@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.gwso_sample_fwd_injected.restype = None
         L.gwso_sample_fwd.argtypes = [c_int64] * 5 + [c_uint64] * 3 + [u16p, f32p, u16p, f32p, f32p]
         L.gwso_sample_fwd.restype = None
+        L.gwso_sample_fwd_scaled.argtypes = [c_int64] * 5 + [c_uint64] * 3 + [u16p, f32p, u16p]
+        L.gwso_sample_fwd_scaled.restype = None
         L.gwso_sample_bwd_injected.argtypes = [c_int64] * 5 + [u16p, f32p, i8p, u16p, f32p, f64p]
         L.gwso_sample_bwd_injected.restype = None
         L.gwso_sample_bwd.argtypes = [c_int64] * 5 + [c_uint64] * 3 + [u16p, f32p, u16p, f32p, f64p]
@@ -198,6 +200,18 @@ def sample_fwd(w, bt, rows, cols, group_rows=1, group_cols=0, seed=0, step=0, el
         lib().gwso_sample_fwd_injected(rows, cols, ld, group_rows, group_cols, _p(w, c_uint16), _p(bt, c_float),
                                        _p(r, c_int8), _p(w_hat, c_uint16), _p(sc, c_float), _p(scratch, c_float))
     return w_hat, sc
+
+
+def sample_fwd_scaled(w, scale_, rows, cols, group_rows=1, group_cols=0, seed=0, step=0, elem_offset=0, ld=None):
+    """Eq. 3 + cast with the per-group factor s_g supplied (its maximum taken elsewhere).  Returns w_hat uint16."""
+    ld = cols if ld is None else ld
+    w = _check_w(w, rows, cols, ld)
+    sc = _c(scale_, np.float32)
+    assert sc.size == n_groups(rows, cols, group_rows, group_cols)
+    w_hat = w.copy()
+    lib().gwso_sample_fwd_scaled(rows, cols, ld, group_rows, group_cols, seed, step, elem_offset, _p(w, c_uint16),
+                                 _p(sc, c_float), _p(w_hat, c_uint16))
+    return w_hat
 
 
 def sample_bwd(g, scale_, rows, cols, group_rows=1, group_cols=0, seed=0, step=0, elem_offset=0, ld=None, r=None):
