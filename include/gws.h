@@ -127,6 +127,35 @@ int gws_sample_fwd(const gws_desc* desc, const void* w, const float* bt, void* w
 int gws_sample_bwd(const gws_desc* desc, const void* grad_w_hat, const float* scale, void* grad_w,
                    float* grad_bt, void* stream);
 
+/* ---- tensors held in parts (shards) ---------------------------------------------------------
+ * Section 3.5 leaves the 2 bytes per parameter of w_hat to training parallelism: each rank then
+ * holds a run of a tensor's elements, and a group can reach across two ranks.  Eq. 3 needs the
+ * maximum over the WHOLE group and Eq. 4 the sum over the whole group, so the fused calls above
+ * are right only for groups a rank holds completely.  For the others the steps are taken apart:
+ * gws_group_absmax on the part (a partial maximum), a MAX reduction between the ranks (the
+ * caller's: NCCL or any other), gws_scale_from_absmax, gws_sample_fwd_scaled on the part; in
+ * backward gws_sample_bwd on the part with that scale (a partial gradient: Eq. 4 is linear in
+ * the group sum) and a SUM reduction.  A part states the logical index of its first element in
+ * elem_offset, so it draws the noise the uncut tensor would: the result has the uncut tensor's bits.
+ */
+
+/*
+ * The per-group factor of Eq. 3, s_g = fl32(absmax_g * 2^(1 - b_g)), from maxima taken earlier:
+ * bit-identical to what gws_sample_fwd writes to scale_out for the same maxima and bit-widths.
+ *   absmax, bt  device, FP32 [n_groups], read only
+ *   scale       device, FP32 [n_groups], written (may be absmax itself)
+ * n_groups == 0 does nothing; negative is GWS_ERR_SHAPE.
+ */
+int gws_scale_from_absmax(int64_t n_groups, const float* absmax, const float* bt, float* scale, void* stream);
+
+/*
+ * Forward sampling with the per-group factor supplied: noise, add and BF16 cast of Eq. 3, no
+ * maximum taken.  Arguments as gws_sample_fwd, except
+ *   scale  device, FP32 [n_groups of desc], read only: s_g of each group of the descriptor.
+ * With scale as written by gws_sample_fwd the output equals that call's w_hat bit for bit.
+ */
+int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scale, void* w_hat, void* stream);
+
 /* ---- many tensors per launch ---------------------------------------------------------------
  * One linear layer of a 1B-parameter model is a few microseconds of HBM time, so a training
  * step samples all layers with as few launches as possible: tensors that run on the same kernel

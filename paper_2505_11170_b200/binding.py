@@ -64,6 +64,8 @@ _SIGNATURES = {
     "gws_noise": (c_int, [POINTER(Desc), c_void_p, c_void_p]),
     "gws_sample_fwd": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gws_sample_bwd": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gws_scale_from_absmax": (c_int, [c_int64, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gws_sample_fwd_scaled": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p]),
     "gws_workspace_bytes": (c_size_t, [c_int]),
     "gws_multi_prepare": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, c_void_p, c_size_t,
                                   POINTER(_MultiPlan), c_void_p]),
@@ -183,6 +185,27 @@ def sample_fwd(desc: Desc, w: torch.Tensor, bt: torch.Tensor, w_hat: Optional[to
         scale_out = torch.empty(n_groups(desc), dtype=torch.float32, device=w.device)
     _check(load_library().gws_sample_fwd(ctypes.byref(desc), _ptr(w), _ptr(bt), _ptr(w_hat), _ptr(scale_out), _stream(stream)))
     return w_hat, scale_out
+
+
+def scale_from_absmax(absmax: torch.Tensor, bt: torch.Tensor, scale: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """s_g = fl32(absmax_g * 2^(1 - b_g)); ``scale`` may be ``absmax`` itself."""
+    _require_cuda(absmax, bt, scale)
+    if absmax.numel() != bt.numel():
+        raise ValueError("gws: absmax and bt differ in length")
+    if scale is None:
+        scale = torch.empty_like(absmax)
+    _check(load_library().gws_scale_from_absmax(absmax.numel(), _ptr(absmax), _ptr(bt), _ptr(scale), _stream(stream)))
+    return scale
+
+
+def sample_fwd_scaled(desc: Desc, w: torch.Tensor, scale: torch.Tensor, w_hat: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    """Forward with the per-group factor supplied (its maximum taken, and reduced, elsewhere)."""
+    _require_cuda(w, scale, w_hat)
+    if w_hat is None:
+        w_hat = torch.empty_like(w)
+    _check(load_library().gws_sample_fwd_scaled(ctypes.byref(desc), _ptr(w), _ptr(scale), _ptr(w_hat), _stream(stream)))
+    return w_hat
 
 
 def sample_bwd(desc: Desc, grad_w_hat: torch.Tensor, scale: torch.Tensor, grad_w: Optional[torch.Tensor] = None,

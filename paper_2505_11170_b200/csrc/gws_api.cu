@@ -150,7 +150,7 @@ gws::FlatRec to_flat_rec(const Entry& e) {
 // Chunks (64 bytes) a thread handles in each mode.
 template <int MODE, int VARIANT>
 constexpr int flat_cpt() {
-  return VARIANT == gws::kNarrow ? 1 : (MODE == gws::kFwd ? GWS_FLAT_CPT_FWD : GWS_FLAT_CPT_BWD);
+  return VARIANT == gws::kNarrow ? 1 : (MODE == gws::kBwd ? GWS_FLAT_CPT_BWD : GWS_FLAT_CPT_FWD);
 }
 
 template <int MODE, int VARIANT, int CAP>
@@ -438,6 +438,27 @@ int gws_sample_fwd(const gws_desc* desc, const void* w, const float* bt, void* w
   const int cls = classify(desc, aligned(w, 16) && aligned(w_hat, 16));
   const Entry e = make_entry(desc, cls, w, w_hat, bt, scale_out);
   return launch<gws::kFwd>(cls, e, nullptr, 0, tiles_of(desc, cls), desc->step, static_cast<cudaStream_t>(stream));
+}
+
+int gws_scale_from_absmax(int64_t n_groups, const float* absmax, const float* bt, float* scale, void* stream) {
+  if (n_groups < 0) return GWS_ERR_SHAPE;
+  if (n_groups == 0) return GWS_OK;
+  if (absmax == nullptr || bt == nullptr || scale == nullptr) return GWS_ERR_NULL;
+  if (!aligned(absmax, 4) || !aligned(bt, 4) || !aligned(scale, 4)) return GWS_ERR_ALIGN;
+  const int64_t blocks = std::min<int64_t>((n_groups + 255) / 256, 148 * 8);
+  gws::k_scale<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(absmax, bt, scale, n_groups);
+  return check_launch("scale kernel");
+}
+
+int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scale, void* w_hat, void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (w == nullptr || scale == nullptr || w_hat == nullptr) return GWS_ERR_NULL;
+  if (!aligned(w, 2) || !aligned(w_hat, 2) || !aligned(scale, 4)) return GWS_ERR_ALIGN;
+  if (overlaps(w, span_bytes(desc), w_hat, span_bytes(desc))) return GWS_ERR_ALIAS;
+  const int cls = classify(desc, aligned(w, 16) && aligned(w_hat, 16));
+  const Entry e = make_entry(desc, cls, w, w_hat, scale, nullptr);
+  return launch<gws::kFwdScaled>(cls, e, nullptr, 0, tiles_of(desc, cls), desc->step, static_cast<cudaStream_t>(stream));
 }
 
 int gws_sample_bwd(const gws_desc* desc, const void* grad_w_hat, const float* scale, void* grad_w, float* grad_bt,

@@ -35,13 +35,16 @@
 
 namespace gws {
 
-enum Mode { kAbsmax = 0, kFwd = 1, kBwd = 2 };
+// kFwdScaled: forward with the per-group factor s_g supplied (in `gin`) instead of derived from this tensor's own
+// maxima: the add and cast of Eq. 3 for a tensor whose groups reach into memory this call does not see.
+enum Mode { kAbsmax = 0, kFwd = 1, kBwd = 2, kFwdScaled = 3 };
 enum KernelClass { kFlat = 0, kRowWarp = 1, kRowCta = 2, kGeneral = 3 };
 
 // Full description of one tensor: the record of the multi-tensor tables and the parameter of the
 // vector and general kernels.  `in`/`out`/`gin`/`gout` change meaning with the mode:
 //   absmax: in = w,           gout = absmax
 //   fwd:    in = w,           out = w_hat,           gin = bt,    gout = scale_out or null
+//   scaled: in = w,           out = w_hat,           gin = scale
 //   bwd:    in = grad_w_hat,  out = grad_w or null,  gin = scale, gout = grad_bt
 struct __align__(16) Entry {
   const void* in;
@@ -425,6 +428,12 @@ __device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t first_chunk
       if (ok[i] && e.out != nullptr) store_chunk<USE32>(e.out, chunk[i], 4, c[i]);
       continue;
     }
+    if (MODE == kFwdScaled) {
+      Chunk y;
+      sample_chunk(c[i].x, v0, e.k0, e.k1, e.pre, make_scale(gv[i]), y.x);
+      if (ok[i]) store_chunk<USE32>(e.out, chunk[i], 4, y);
+      continue;
+    }
     uint32_t m = maxabs2(maxabs2(absmax_words4(c[i].x), absmax_words4(c[i].x + 4)),
                          maxabs2(absmax_words4(c[i].x + 8), absmax_words4(c[i].x + 12)));
     for (uint32_t o = 1; o < lanes; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
@@ -473,6 +482,11 @@ __device__ __forceinline__ void flat_narrow(const FlatRec& e, uint32_t chunk, ui
       }
       continue;
     }
+    if (MODE == kFwdScaled) {
+      const uint4 yv = sample_vec(xv, r, make_scale(ld_f32(e.gin, g)));
+      y.x[4 * k] = yv.x; y.x[4 * k + 1] = yv.y; y.x[4 * k + 2] = yv.z; y.x[4 * k + 3] = yv.w;
+      continue;
+    }
     uint32_t m = absmax_vec(xv);
     if (ll == 1u) m = maxabs2(m, absmax_words4(c.x + 4 * mate));
     const float a = absmax_finish(m);
@@ -485,7 +499,7 @@ __device__ __forceinline__ void flat_narrow(const FlatRec& e, uint32_t chunk, ui
     y.x[4 * k] = yv.x; y.x[4 * k + 1] = yv.y; y.x[4 * k + 2] = yv.z; y.x[4 * k + 3] = yv.w;
     if (writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
   }
-  if (MODE == kFwd) store_chunk<false>(e.out, chunk, n_valid, y);
+  if (MODE == kFwd || MODE == kFwdScaled) store_chunk<false>(e.out, chunk, n_valid, y);
   if (MODE == kBwd && e.out != nullptr) store_chunk<false>(e.out, chunk, n_valid, c);
 }
 
@@ -608,6 +622,12 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
       for (uint32_t o = 1; o < 32u; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
       if (lane == 0u) st_f32(e.gout, g, grad_bt_of(gv[i], acc));
       if (e.out != nullptr) store_chunk<true>(e.out, chunk, 4, c[i]);
+      continue;
+    }
+    if (MODE == kFwdScaled) {
+      Chunk y;
+      sample_chunk(c[i].x, v0, e.k0, e.k1, e.pre, make_scale(gv[i]), y.x);
+      store_chunk<true>(e.out, chunk, 4, y);
       continue;
     }
     uint32_t m = maxabs2(maxabs2(absmax_words4(c[i].x), absmax_words4(c[i].x + 4)),
@@ -745,25 +765,28 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
     return;
   }
 
-  uint32_t m = 0u;
+  float a = 0.0f;
+  if (MODE != kFwdScaled) {
+    uint32_t m = 0u;
 #pragma unroll
-  for (int k = 0; k < MAXCPT; ++k)
-    m = maxabs2(m, maxabs2(maxabs2(absmax_words4(c[k].x), absmax_words4(c[k].x + 4)),
-                           maxabs2(absmax_words4(c[k].x + 8), absmax_words4(c[k].x + 12))));
-  for (uint32_t o = 1; o < span; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-  if (BLOCK) {
-    if (lane == 0) red_u[warp] = m;
-    __syncthreads();
-    m = red_u[0];
+    for (int k = 0; k < MAXCPT; ++k)
+      m = maxabs2(m, maxabs2(maxabs2(absmax_words4(c[k].x), absmax_words4(c[k].x + 4)),
+                             maxabs2(absmax_words4(c[k].x + 8), absmax_words4(c[k].x + 12))));
+    for (uint32_t o = 1; o < span; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if (BLOCK) {
+      if (lane == 0) red_u[warp] = m;
+      __syncthreads();
+      m = red_u[0];
 #pragma unroll
-    for (int w = 1; w < kRowThreads / 32; ++w) m = maxabs2(m, red_u[w]);
+      for (int w = 1; w < kRowThreads / 32; ++w) m = maxabs2(m, red_u[w]);
+    }
+    a = absmax_finish(m);
   }
-  const float a = absmax_finish(m);
   if (MODE == kAbsmax) {
     if (okr && t == 0u) st_f32(e.gout, row, a);
     return;
   }
-  const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv)));
+  const Scale sc = make_scale(MODE == kFwdScaled ? gv : __fmul_rn(a, pow2_one_minus(gv)));
 #pragma unroll
   for (int k = 0; k < MAXCPT; ++k) {
     if (!ok[k]) continue;
@@ -773,7 +796,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
     sample_chunk(c[k].x, v0, e.k0, e.k1, e.pre, sc, y.x);
     if (okr) store_chunk<true>(e.out, chunk, 4, y);
   }
-  if (okr && t == 0u && e.gout != nullptr) st_f32(e.gout, row, sc.s);
+  if (MODE == kFwd && okr && t == 0u && e.gout != nullptr) st_f32(e.gout, row, sc.s);
 }
 
 // Host side: as fill_flat_batch.  Tiles: rows per block for shared rows (256 / threads per row), one row per block else.
@@ -842,17 +865,20 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
     for (uint32_t o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
     if (okr && lane == 0) st_f32(e.gout, row, grad_bt_of(gvr, acc));
   } else {
-    uint32_t m = 0;
+    float a = 0.0f;
+    if (MODE != kFwdScaled) {
+      uint32_t m = 0;
 #pragma unroll
-    for (int k = 0; k < V; ++k)
-      if (k * 32u < vpr) m = maxabs2(m, absmax_vec(x[k]));
+      for (int k = 0; k < V; ++k)
+        if (k * 32u < vpr) m = maxabs2(m, absmax_vec(x[k]));
 #pragma unroll
-    for (uint32_t o = 16; o > 0; o >>= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    const float a = absmax_finish(m);
+      for (uint32_t o = 16; o > 0; o >>= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+      a = absmax_finish(m);
+    }
     if (MODE == kAbsmax) {
       if (okr && lane == 0) st_f32(e.gout, row, a);
     } else {
-      const Scale s = make_scale(__fmul_rn(a, pow2_one_minus(gvr)));
+      const Scale s = make_scale(MODE == kFwdScaled ? gvr : __fmul_rn(a, pow2_one_minus(gvr)));
 #pragma unroll
       for (int k = 0; k < V; ++k) {
         if (k * 32u < vpr) {
@@ -861,7 +887,7 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
           if (okr && j < vpr) st_vec(e.out, vbase + j, y);
         }
       }
-      if (okr && lane == 0 && e.gout != nullptr) st_f32(e.gout, row, s.s);
+      if (MODE == kFwd && okr && lane == 0 && e.gout != nullptr) st_f32(e.gout, row, s.s);
     }
   }
 }
@@ -913,22 +939,25 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
       st_f32(e.gout, row, grad_bt_of(gvr, total));
     }
   } else {
-    uint32_t m = 0;
+    float a = 0.0f;
+    if (MODE != kFwdScaled) {
+      uint32_t m = 0;
 #pragma unroll
-    for (int k = 0; k < V; ++k)
-      if (static_cast<uint32_t>(k) * T < vpr) m = maxabs2(m, absmax_vec(x[k]));
+      for (int k = 0; k < V; ++k)
+        if (static_cast<uint32_t>(k) * T < vpr) m = maxabs2(m, absmax_vec(x[k]));
 #pragma unroll
-    for (uint32_t o = 16; o > 0; o >>= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    if (lane == 0) red_u[warp] = m;
-    __syncthreads();
-    uint32_t mm = red_u[0];
+      for (uint32_t o = 16; o > 0; o >>= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+      if (lane == 0) red_u[warp] = m;
+      __syncthreads();
+      uint32_t mm = red_u[0];
 #pragma unroll
-    for (int w = 1; w < WARPS; ++w) mm = maxabs2(mm, red_u[w]);
-    const float a = absmax_finish(mm);
+      for (int w = 1; w < WARPS; ++w) mm = maxabs2(mm, red_u[w]);
+      a = absmax_finish(mm);
+    }
     if (MODE == kAbsmax) {
       if (threadIdx.x == 0) st_f32(e.gout, row, a);
     } else {
-      const Scale s = make_scale(__fmul_rn(a, pow2_one_minus(gvr)));
+      const Scale s = make_scale(MODE == kFwdScaled ? gvr : __fmul_rn(a, pow2_one_minus(gvr)));
 #pragma unroll
       for (int k = 0; k < V; ++k) {
         if (static_cast<uint32_t>(k) * T < vpr) {
@@ -937,7 +966,7 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
           if (j < vpr) st_vec(e.out, vbase + j, y);
         }
       }
-      if (threadIdx.x == 0 && e.gout != nullptr) st_f32(e.gout, row, s.s);
+      if (MODE == kFwd && threadIdx.x == 0 && e.gout != nullptr) st_f32(e.gout, row, s.s);
     }
   }
 }
@@ -965,7 +994,8 @@ __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_consta
     const int64_t h = min(gr, e.rows - r0), wd = min(gc, e.cols - c0);
     const int64_t count = h * wd;
     float scale = 0.0f;
-    if (MODE != kBwd) {
+    if (MODE == kFwdScaled) scale = ld_f32(e.gin, g);
+    if (MODE == kAbsmax || MODE == kFwd) {
       float m = 0.0f;
       for (int64_t k = threadIdx.x; k < count; k += T) {
         const int64_t i = r0 + k / wd, j = c0 + k % wd;
@@ -1000,7 +1030,7 @@ __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_consta
         const int r = r_from_pairs(pairs, static_cast<unsigned>(el & 7u));
         const uint16_t bits = ld_u16(in, i * e.ld + j);
         const float val = __uint_as_float(static_cast<uint32_t>(bits) << 16);
-        if (MODE == kFwd) {
+        if (MODE == kFwd || MODE == kFwdScaled) {
           const float q = __fmul_rn(static_cast<float>(r), scale);
           const float y = __fadd_rn(val, q);
           st_u16(out, i * e.ld + j, static_cast<uint16_t>(pack_bf16_rne(y, 0.0f) & 0xFFFFu));
@@ -1068,6 +1098,14 @@ __global__ void __launch_bounds__(256) k_noise_probe(uint32_t* __restrict__ sink
     for (int w = 0; w < 8; ++w) t ^= red[w];
     sink[blockIdx.x] = t;
   }
+}
+
+// s_g = fl32(absmax_g * 2^(1 - b_g)) for a run of groups whose maxima were taken (and, for a sharded tensor,
+// reduced across shards) beforehand: the factor of Eq. 3 as the fused forward kernels form it.
+__global__ void __launch_bounds__(256) k_scale(const float* __restrict__ absmax, const float* __restrict__ bt,
+                                               float* __restrict__ scale, int64_t n) {
+  for (int64_t k = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x; k < n; k += static_cast<int64_t>(gridDim.x) * 256)
+    st_f32(scale, k, __fmul_rn(ld_f32(absmax, k), pow2_one_minus(ld_f32(bt, k))));
 }
 
 // ---- bit-width parametrisation (Eq. 11), its loss term (Eq. 12) and the chain rule back to b_i ----------
