@@ -26,9 +26,13 @@
  *   - Random bits: Philox4x32 with 10 rounds (Section 3.4 names Philox).  Element (i, j) has
  *     the logical index e = elem_offset + i*cols + j (independent of ld).  Counter =
  *     (lo32(e>>3), hi32(e>>3), lo32(step), hi32(step)), key = (lo32(seed), hi32(seed)).  One
- *     call yields 128 bits = eight 16-bit fields; element e uses field e & 7, counted from
- *     the least significant bits of output word 0.
- *   - Field bits x0 (LSB) .. x15:  m2 = x0&...&x7&(x8|x9);  m1 = (x10|x11)&(x12|x13)&x14;
+ *     call yields four 32-bit words = 128 bits, 16 for each of 8 consecutive elements.
+ *     Section 3.4 combines whole random integers with AND / OR, one bit position per element,
+ *     so an element's 16 bits are bit columns of the four words, not a run inside one word:
+ *     element t = e & 7 (j = t >> 1, h = t & 1) owns columns c+1, c, c-7, c-8 of every word,
+ *     c = 16h + 14 - 2j.  Its field bit x_k is bit c + D[k] of word W[k] with
+ *     W = {0,1,2,3, 1,2,3, 0,1,2, 0,1,2,3, 0, 3},  D = {-7,-7,-7,-7, -8,-8,-8, 1,1,1, 0,0,0,0, -8, 1}.
+ *   - Field bits x0 .. x15:  m2 = x0&...&x7&(x8|x9);  m1 = (x10|x11)&(x12|x13)&x14;
  *     |R| = 2 if m2 else 1 if m1 else 0;  R is negative iff x15 is set and |R| != 0.
  *     This gives exactly Eq. 10: Pr(+-2) = 3/4 * 2^-9 each, Pr(+-1) = (3/4)^2 * 2^-2 *
  *     (1 - 3/1024) each.
@@ -234,6 +238,12 @@ int gws_multi_launch_count(const gws_multi_plan* plan, int backward);
 /* Forward / backward of every tensor of the plan for gradient-update counter `step`. */
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
 int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
+
+/* gws_sample_fwd_scaled for every tensor of the plan, with the launches of gws_sample_fwd_multi: the
+ * `scale` array each tensor was prepared with is READ (the per-group factor, e.g. after a reduction
+ * between ranks) instead of written; `bt` is not used.  GWS_ERR_NULL if the plan has no forward side
+ * or a tensor was prepared without a scale array. */
+int gws_sample_fwd_scaled_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
 
 /* ---- bit-width parametrisation and seeds (Section 3.6, "Bitwidth" and "Managing seed") ---------------
  *

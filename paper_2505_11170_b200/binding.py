@@ -74,6 +74,7 @@ _SIGNATURES = {
     "gws_multi_launch_count": (c_int, [POINTER(_MultiPlan), c_int]),
     "gws_sample_fwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_sample_bwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
+    "gws_sample_fwd_scaled_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_bitwidth": (c_int, [c_int64, c_void_p, c_float, c_float, c_void_p, c_void_p]),
     "gws_bitwidth_loss": (c_int, [c_int64, c_void_p, c_float, c_void_p, c_void_p]),
     "gws_bitwidth_grad": (c_int, [c_int64, c_void_p, c_void_p, c_float, c_float, ctypes.c_double, c_void_p, c_void_p]),
@@ -290,6 +291,10 @@ class MultiPlan:
 
     def sample_bwd_multi(self, step: int, stream=None) -> None:
         _check(load_library().gws_sample_bwd_multi(ctypes.byref(self.plan), step, _stream(stream)))
+
+    def sample_fwd_scaled_multi(self, step: int, stream=None) -> None:
+        """Forward with the factors already in the plan's ``scale`` arrays (read, not written)."""
+        _check(load_library().gws_sample_fwd_scaled_multi(ctypes.byref(self.plan), step, _stream(stream)))
 
 
 def bitwidth(bi: torch.Tensor, b_init: float, b_target: float, bt: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

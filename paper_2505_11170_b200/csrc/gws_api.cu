@@ -457,7 +457,7 @@ int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scal
   if (!aligned(w, 2) || !aligned(w_hat, 2) || !aligned(scale, 4)) return GWS_ERR_ALIGN;
   if (overlaps(w, span_bytes(desc), w_hat, span_bytes(desc))) return GWS_ERR_ALIAS;
   const int cls = classify(desc, aligned(w, 16) && aligned(w_hat, 16));
-  const Entry e = make_entry(desc, cls, w, w_hat, scale, nullptr);
+  const Entry e = make_entry(desc, cls, w, w_hat, nullptr, const_cast<float*>(scale));   // this mode only reads it
   return launch<gws::kFwdScaled>(cls, e, nullptr, 0, tiles_of(desc, cls), desc->step, static_cast<cudaStream_t>(stream));
 }
 
@@ -659,44 +659,53 @@ int64_t gws_multi_table_image(int n, const gws_desc* descs, const gws_multi_ptrs
   return static_cast<int64_t>(image.size());
 }
 
-static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream, bool backward) {
+}  // extern "C" (a template cannot have C linkage)
+
+// One pass over the tensors of a plan.  MODE kFwd and kFwdScaled read the forward tables, kBwd the backward ones.
+template <int MODE>
+static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
+  constexpr bool backward = MODE == gws::kBwd;
   if (plan == nullptr) return GWS_ERR_NULL;
   if (plan->workspace == nullptr || plan->host_tables == nullptr) return GWS_ERR_WORKSPACE;
   if (backward ? !plan->has_bwd : !plan->has_fwd) return GWS_ERR_NULL;
   const Entry none{};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  auto host_table = [&](int cls) {
+    return reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
+                                          (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
+  };
+  if (MODE == gws::kFwdScaled)   // every tensor must come with its scale array
+    for (int cls = 0; cls < 4; ++cls)
+      for (int i = 0; i < plan->count[cls]; ++i)
+        if (host_table(cls)[i].gout == nullptr) return GWS_ERR_NULL;
   for (int cls = 0; cls < 4; ++cls) {
     const int count = plan->count[cls];
     if (count == 0) continue;
     const Entry* table = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->workspace) +
                                                         (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
+    const Entry* host = host_table(cls);
     if (cls == gws::kFlat) {
-      const Entry* host = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
-                                                         (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
-      const int st = backward ? launch_flat<gws::kBwd>(host, count, step, s) : launch_flat<gws::kFwd>(host, count, step, s);
+      const int st = launch_flat<MODE>(host, count, step, s);
       if (st != GWS_OK) return st;
     } else if (cls != gws::kGeneral) {
-      const Entry* host = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
-                                                         (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
-      const int st = backward ? launch_rows<gws::kBwd>(cls, host, count, step, s) : launch_rows<gws::kFwd>(cls, host, count, step, s);
+      const int st = launch_rows<MODE>(cls, host, count, step, s);
       if (st != GWS_OK) return st;
     } else {
       // whole 32 x 32 blocks share launches of the square-block kernel; every other shape: one launch per tensor
-      const Entry* host = reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) +
-                                                         (backward ? plan->bwd_offset[cls] : plan->fwd_offset[cls]));
       std::vector<const Entry*> squares;
       for (int i = 0; i < count; ++i) {
         if (square_eligible(host[i])) { squares.push_back(&host[i]); continue; }
-        const int st = backward ? launch<gws::kBwd>(cls, none, table, i, kGeneralGrid, step, s)
-                                : launch<gws::kFwd>(cls, none, table, i, kGeneralGrid, step, s);
+        const int st = launch<MODE>(cls, none, table, i, kGeneralGrid, step, s);
         if (st != GWS_OK) return st;
       }
-      const int st = backward ? launch_squares<gws::kBwd>(squares, step, s) : launch_squares<gws::kFwd>(squares, step, s);
+      const int st = launch_squares<MODE>(squares, step, s);
       if (st != GWS_OK) return st;
     }
   }
   return GWS_OK;
 }
+
+extern "C" {
 
 int gws_multi_launch_count(const gws_multi_plan* plan, int backward) {
   if (plan == nullptr) return GWS_ERR_NULL;
@@ -725,11 +734,15 @@ int gws_multi_launch_count(const gws_multi_plan* plan, int backward) {
 }
 
 int gws_sample_fwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
-  return run_multi(plan, step, stream, false);
+  return run_multi<gws::kFwd>(plan, step, stream);
 }
 
 int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
-  return run_multi(plan, step, stream, true);
+  return run_multi<gws::kBwd>(plan, step, stream);
+}
+
+int gws_sample_fwd_scaled_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
+  return run_multi<gws::kFwdScaled>(plan, step, stream);
 }
 
 int gws_multi_locate_probe(const gws_multi_plan* plan, int backward, int kernel_class, const int64_t* tiles, int n_tiles,
@@ -871,7 +884,7 @@ int gws_sample_fwd_multi_static(int n, const gws_desc* descs, const gws_multi_pt
                                           static_cast<cudaStream_t>(stream));
   if (err != cudaSuccess) return cuda_fail(err, "upload into the built-in table array");
   plan.host_tables = image.data();   // lives until the launches below have copied their parameters
-  return run_multi(&plan, step, stream, false);
+  return run_multi<gws::kFwd>(&plan, step, stream);
 }
 
 // ---- bit-width parametrisation and seeds (Section 3.6) ------------------------------------------------

@@ -44,7 +44,7 @@ enum KernelClass { kFlat = 0, kRowWarp = 1, kRowCta = 2, kGeneral = 3 };
 // vector and general kernels.  `in`/`out`/`gin`/`gout` change meaning with the mode:
 //   absmax: in = w,           gout = absmax
 //   fwd:    in = w,           out = w_hat,           gin = bt,    gout = scale_out or null
-//   scaled: in = w,           out = w_hat,           gin = scale
+//   scaled: in = w,           out = w_hat,           gout = scale (read only): the forward record serves both forms
 //   bwd:    in = grad_w_hat,  out = grad_w or null,  gin = scale, gout = grad_bt
 struct __align__(16) Entry {
   const void* in;
@@ -408,7 +408,7 @@ __device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t first_chunk
     ok[i] = chunk0 < n_chunks;
     chunk[i] = ok[i] ? chunk0 : n_chunks - 1u;   // keeps the warp whole for the shuffles
     c[i] = load_chunk<USE32>(e.in, chunk[i], 4);
-    gv[i] = (MODE != kAbsmax) ? ld_f32(e.gin, chunk[i] >> lanes_log2) : 0.0f;
+    gv[i] = (MODE != kAbsmax) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, chunk[i] >> lanes_log2) : 0.0f;
   }
 #pragma unroll
   for (int i = 0; i < CPT; ++i) {
@@ -483,7 +483,7 @@ __device__ __forceinline__ void flat_narrow(const FlatRec& e, uint32_t chunk, ui
       continue;
     }
     if (MODE == kFwdScaled) {
-      const uint4 yv = sample_vec(xv, r, make_scale(ld_f32(e.gin, g)));
+      const uint4 yv = sample_vec(xv, r, make_scale(ld_f32(e.gout, g)));
       y.x[4 * k] = yv.x; y.x[4 * k + 1] = yv.y; y.x[4 * k + 2] = yv.z; y.x[4 * k + 3] = yv.w;
       continue;
     }
@@ -601,7 +601,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
     ok[i] = q[i] < cpr;
     if (ok[i]) {
       c[i] = load_chunk<true>(e.in, row_chunk0 + q[i], 4);
-      gv[i] = (MODE != kAbsmax) ? ld_f32(e.gin, band * cpr + q[i]) : 0.0f;
+      gv[i] = (MODE != kAbsmax) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, band * cpr + q[i]) : 0.0f;
     }
   }
 #pragma unroll
@@ -734,7 +734,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
       for (int i = 0; i < 16; ++i) c[k].x[i] = 0u;
     }
   }
-  const float gv = (MODE != kAbsmax) ? ld_f32(e.gin, row) : 0.0f;
+  const float gv = (MODE != kAbsmax) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, row) : 0.0f;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const uint32_t span = BLOCK ? 32u : tpr;   // lanes of this warp that share the row
 
@@ -846,7 +846,7 @@ __global__ void __launch_bounds__(kRowWarpThreads) k_row_warp(const __grid_const
       if (okr && j < vpr) x[k] = ld_vec(e.in, vbase + j);
     }
   }
-  const float gvr = (MODE != kAbsmax && okr) ? ld_f32(e.gin, row) : 0.0f;
+  const float gvr = (MODE != kAbsmax && okr) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, row) : 0.0f;
 
   if (MODE == kBwd) {
     DotAcc dot;
@@ -916,7 +916,7 @@ __global__ void __launch_bounds__(kRowCtaThreads) k_row_cta(const __grid_constan
       if (j < vpr) x[k] = ld_vec(e.in, vbase + j);
     }
   }
-  const float gvr = (MODE != kAbsmax) ? ld_f32(e.gin, row) : 0.0f;
+  const float gvr = (MODE != kAbsmax) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, row) : 0.0f;
 
   if (MODE == kBwd) {
     DotAcc dot;
@@ -994,7 +994,7 @@ __global__ void __launch_bounds__(kGeneralThreads) k_general(const __grid_consta
     const int64_t h = min(gr, e.rows - r0), wd = min(gc, e.cols - c0);
     const int64_t count = h * wd;
     float scale = 0.0f;
-    if (MODE == kFwdScaled) scale = ld_f32(e.gin, g);
+    if (MODE == kFwdScaled) scale = ld_f32(e.gout, g);
     if (MODE == kAbsmax || MODE == kFwd) {
       float m = 0.0f;
       for (int64_t k = threadIdx.x; k < count; k += T) {

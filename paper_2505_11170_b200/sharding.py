@@ -30,12 +30,13 @@ from . import binding
 from .binding import Desc
 
 
-def even_bounds(n_elements: int, world: int) -> List[int]:
-    """Cuts of ``n_elements`` into ``world`` runs of equal length, rounded up to 8 elements (16 bytes of BF16)."""
-    if n_elements < 0 or world < 1:
-        raise ValueError("even_bounds: n_elements >= 0 and world >= 1 expected")
+def even_bounds(n_elements: int, world: int, align: int = 32) -> List[int]:
+    """Cuts of ``n_elements`` into ``world`` runs of equal length, rounded up to ``align`` elements.  The default, 32
+    elements = 64 bytes of BF16, keeps every piece on the kernels that move 64-byte chunks; 8 is the minimum."""
+    if n_elements < 0 or world < 1 or align < 8 or align % 8 != 0:
+        raise ValueError("even_bounds: n_elements >= 0, world >= 1 and align a multiple of 8 expected")
     per = -(-n_elements // world)
-    per = -(-per // 8) * 8
+    per = -(-per // align) * align
     return [min(r * per, n_elements) for r in range(world + 1)]
 
 
@@ -234,3 +235,125 @@ class ShardedSampler:
         if self.plan.world > 1:
             all_reduce_slots(buf, "sum", self.process_group)
         self.backward_finish(buf, grad_bt)
+
+
+class ShardedSetSampler:
+    """All sharded tensors of a rank in a few launches per pass (the per-tensor sampler above takes several per tensor).
+
+    Every whole-group body and every end piece is one tensor of a multi-tensor plan, so one forward pass of that plan
+    samples the bodies for good and leaves, for each end piece, the factor its PART of the group would give:
+    fl32(partial max * 2^(1 - b)).  Rounding is monotonic and every rank multiplies by the same power, so the
+    maximum of those over the ranks is the factor of the whole group, fl32(max * 2^(1 - b)), bit for bit: the
+    factors themselves go through the MAX all-reduce, and a second, small plan re-samples the end pieces with
+    them (gws_sample_fwd_scaled_multi).  Backward is one pass of the plan, then the SUM all-reduce.
+
+    ``w[t]`` / ``w_hat[t]`` / ``grad_w_hat[t]``: BF16 shard of tensor t; ``bt[t]``: FP32 [plans[t].n_local_groups].
+    The sampler owns the flat ``scale_all`` / ``grad_bt_all`` arrays; ``scale[t]`` and ``grad_bt[t]`` are views.
+    """
+
+    def __init__(self, plans: Sequence[FlatShardPlan], seeds: Sequence[int], w: Sequence[torch.Tensor], bt: Sequence[torch.Tensor],
+                 w_hat: Sequence[torch.Tensor], grad_w_hat: Optional[Sequence[torch.Tensor]] = None, process_group=None):
+        if not (len(plans) == len(seeds) == len(w) == len(bt) == len(w_hat)) or (grad_w_hat is not None and len(grad_w_hat) != len(plans)):
+            raise ValueError("ShardedSetSampler: one plan, seed and buffer set per tensor expected")
+        if len({p.world for p in plans}) > 1:
+            raise ValueError("ShardedSetSampler: every plan must have the same world size")
+        self.plans = list(plans)
+        self.process_group = process_group
+        self.world = plans[0].world if plans else 1
+        device = w[0].device if w else torch.device("cuda")
+        offsets, total = [], 0
+        for p in plans:
+            offsets.append(total)
+            total += p.n_local_groups
+        self.scale_all = torch.zeros(max(total, 1), dtype=torch.float32, device=device)
+        self.grad_bt_all = torch.zeros(max(total, 1), dtype=torch.float32, device=device)
+        self.scale = [self.scale_all[o:o + p.n_local_groups] for o, p in zip(offsets, plans)]
+        self.grad_bt = [self.grad_bt_all[o:o + p.n_local_groups] for o, p in zip(offsets, plans)]
+        n_slots = self.world + 1
+        self._buf = torch.zeros(max(len(plans) * n_slots, 1), dtype=torch.float32, device=device)
+
+        descs, sel = [], []            # sel: (tensor, element slice, group slice) of every plan entry
+        piece_entries = []
+        src, dst, grp, read = [], [], [], []
+        for t, p in enumerate(plans):
+            for buf, name in ((w[t], "w"), (w_hat[t], "w_hat")) + (((grad_w_hat[t], "grad_w_hat"),) if grad_w_hat is not None else ()):
+                if buf.numel() != p.n_elements or buf.dtype != torch.bfloat16 or not buf.is_contiguous():
+                    raise ValueError(f"ShardedSetSampler: {name}[{t}] must be a contiguous BF16 buffer of the shard's length")
+            if bt[t].numel() != p.n_local_groups or bt[t].dtype != torch.float32 or not bt[t].is_contiguous():
+                raise ValueError(f"ShardedSetSampler: bt[{t}] must be a contiguous FP32 array of n_local_groups entries")
+            if p.body is not None:
+                b = p.body
+                descs.append(Desc.make(b.n_groups, p.group, 1, p.group, seed=seeds[t], elem_offset=b.elem_offset))
+                sel.append((t, slice(b.local_begin, b.local_begin + b.n_groups * p.group), slice(b.local_group, b.local_group + b.n_groups)))
+            for piece in p.pieces:
+                descs.append(Desc.make(1, piece.n_elements, 1, 0, seed=seeds[t], elem_offset=piece.elem_offset))
+                sel.append((t, slice(piece.local_begin, piece.local_begin + piece.n_elements), slice(piece.local_group, piece.local_group + 1)))
+                piece_entries.append(len(descs) - 1)
+                for s in piece.slots:
+                    src.append(offsets[t] + piece.local_group)
+                    dst.append(t * n_slots + s)
+                grp.append(offsets[t] + piece.local_group)
+                read.append(t * n_slots + piece.read_slot)
+        index = lambda v: torch.tensor(v, dtype=torch.int64, device=device)
+        self._src, self._dst, self._grp, self._read = index(src), index(dst), index(grp), index(read)
+        self.n_pieces = len(piece_entries)
+
+        def views(entries):
+            pick = lambda bufs, groups: [bufs[t][gs] if groups else bufs[t][es] for t, es, gs in (sel[k] for k in entries)]
+            return dict(w=pick(w, False), bt=pick(bt, True), w_hat=pick(w_hat, False), scale=pick(self.scale, True),
+                        grad_w_hat=pick(grad_w_hat, False) if grad_w_hat is not None else None,
+                        grad_bt=pick(self.grad_bt, True) if grad_w_hat is not None else None)
+
+        everything = list(range(len(descs)))
+        self._plan_all = binding.MultiPlan(descs, **views(everything)) if descs else None
+        self._plan_pieces = None
+        if piece_entries:
+            v = views(piece_entries)
+            self._plan_pieces = binding.MultiPlan([descs[k] for k in piece_entries], w=v["w"], bt=v["bt"], w_hat=v["w_hat"], scale=v["scale"])
+
+    def _gather(self, values: torch.Tensor) -> torch.Tensor:
+        self._buf.zero_()
+        if self.n_pieces:
+            self._buf.index_copy_(0, self._dst, values.index_select(0, self._src))    # copies only
+        return self._buf
+
+    def _scatter(self, reduced: torch.Tensor, values: torch.Tensor) -> None:
+        if self.n_pieces:
+            values.index_copy_(0, self._grp, reduced.index_select(0, self._read))
+
+    def forward_local(self, step: int) -> torch.Tensor:
+        """Returns the slot buffer (W+1 slots per tensor) to be reduced with MAX over the ranks."""
+        if self._plan_all is not None:
+            self._plan_all.sample_fwd_multi(step)
+        return self._gather(self.scale_all)
+
+    def forward_finish(self, step: int, reduced: torch.Tensor) -> None:
+        self._scatter(reduced, self.scale_all)
+        if self._plan_pieces is not None:
+            self._plan_pieces.sample_fwd_scaled_multi(step)
+
+    def forward(self, step: int) -> None:
+        buf = self.forward_local(step)
+        if self.world > 1:
+            all_reduce_slots(buf, "max", self.process_group)
+        self.forward_finish(step, buf)
+
+    def backward_local(self, step: int) -> torch.Tensor:
+        """Returns the slot buffer to be reduced with SUM over the ranks."""
+        if self._plan_all is not None:
+            self._plan_all.sample_bwd_multi(step)
+        return self._gather(self.grad_bt_all)
+
+    def backward_finish(self, reduced: torch.Tensor) -> None:
+        self._scatter(reduced, self.grad_bt_all)
+
+    def backward(self, step: int) -> None:
+        buf = self.backward_local(step)
+        if self.world > 1:
+            all_reduce_slots(buf, "sum", self.process_group)
+        self.backward_finish(buf)
+
+    @property
+    def launches_per_forward(self) -> int:
+        return (self._plan_all.launches_per_pass if self._plan_all is not None else 0) + \
+               (self._plan_pieces.launches_per_pass if self._plan_pieces is not None else 0)

@@ -105,3 +105,60 @@ def test_sampler_rejects_buffers_of_the_wrong_size():
     with pytest.raises(ValueError):
         s.forward_local(0, w[:-8], torch.zeros(plan.n_local_groups, device=DEV), torch.empty_like(w),
                         torch.zeros(plan.n_local_groups, device=DEV))
+
+
+def _set_inputs(shapes, seed):
+    out = []
+    for k, (n_groups, group) in enumerate(shapes):
+        out.append(_inputs(n_groups * group, n_groups, seed + k))
+    return out
+
+
+@pytest.mark.parametrize("world,align", [(4, 32), (3, 8), (1, 32), (8, 32)])
+def test_tensor_set_sampler_carries_the_bits_of_the_uncut_tensors(world, align):
+    from paper_2505_11170_b200.sharding import ShardedSetSampler, even_bounds
+    # (groups, group size): groups of 128, of 32, whole rows of 2048 and 4096 + 32, narrow groups, a tensor smaller than the world
+    shapes = [(90, 128), (77, 32), (10, 2048), (3, 4128), (200, 8), (1, 64), (50, 256)]
+    step, user_seed = 21, 0xABCDEF12345
+    inputs = _set_inputs(shapes, 300)
+    seeds = [user_seed + 977 * k for k in range(len(shapes))]
+    want = []
+    for (n_groups, group), (w, grad, bt), seed in zip(shapes, inputs, seeds):
+        hat, scale = orc.sample_fwd(bits_of(w), bt.numpy(), n_groups, group, seed=seed, step=step)
+        _, gbt = orc.sample_bwd(bits_of(grad), scale, n_groups, group, seed=seed, step=step)
+        r = orc.noise_r(seed, step, 0, n_groups * group).astype(np.float64)
+        absprod = np.abs(f32_of_bits(bits_of(grad)).astype(np.float64) * r).reshape(n_groups, group).sum(axis=1)
+        want.append((hat, scale, gbt, 1e-5 * LN2 * scale.astype(np.float64) * absprod + 1e-45))
+
+    ranks = []
+    for r in range(world):
+        plans = [plan_flat_shard(ng * g, g, r, world, even_bounds(ng * g, world, align)) for ng, g in shapes]
+        loc = lambda p, t: t[p.begin:p.end].to(DEV)
+        grp = lambda p, t: t[p.first_group:p.first_group + p.n_local_groups].to(DEV)
+        w = [loc(p, x[0]) for p, x in zip(plans, inputs)]
+        grad = [loc(p, x[1]) for p, x in zip(plans, inputs)]
+        bt = [grp(p, x[2]) for p, x in zip(plans, inputs)]
+        w_hat = [torch.full_like(t, float("nan")) for t in w]
+        ranks.append(dict(plans=plans, w_hat=w_hat, sampler=ShardedSetSampler(plans, seeds, w, bt, w_hat, grad)))
+
+    bufs = [k["sampler"].forward_local(step) for k in ranks]
+    reduced = torch.stack(bufs).max(dim=0).values
+    for k in ranks:
+        k["sampler"].forward_finish(step, reduced.clone())
+    bufs = [k["sampler"].backward_local(step) for k in ranks]
+    reduced = torch.stack(bufs).sum(dim=0)
+    for k in ranks:
+        k["sampler"].backward_finish(reduced.clone())
+    torch.cuda.synchronize()
+
+    for k in ranks:
+        for t, p in enumerate(k["plans"]):
+            hat, scale, gbt, tol = want[t]
+            gs = slice(p.first_group, p.first_group + p.n_local_groups)
+            assert np.array_equal(bits_of(k["w_hat"][t]), hat[p.begin:p.end]), (p.rank, t)
+            assert np.array_equal(k["sampler"].scale[t].cpu().numpy().view(np.uint32), scale[gs].view(np.uint32)), (p.rank, t)
+            got = k["sampler"].grad_bt[t].cpu().numpy().astype(np.float64)
+            assert np.all(np.abs(got - gbt[gs].astype(np.float64)) <= tol[gs]), (p.rank, t)
+    if world > 1 and align == 32:
+        # whole groups share one launch; the end pieces (rows of 64-byte chunks) a few more, twice
+        assert max(k["sampler"].launches_per_forward for k in ranks) <= 20

@@ -122,3 +122,16 @@ def test_partial_group_gradients_add_up_to_the_uncut_gradient():
     tol = 4 * 2.0 ** -24 * np.log(2.0) * sc * bound + 1e-45
     assert np.all(np.abs(total - want.astype(np.float64)) <= tol)
     assert np.any(want != 0)
+
+
+def test_factor_of_a_whole_group_is_the_largest_of_its_parts_factors():
+    # fl32(a * p) is non-decreasing in a for p > 0, so reducing the parts' FACTORS by max gives the factor of the
+    # reduced maximum exactly, for integer and fractional bit-widths alike (each part uses the same b)
+    rng = np.random.default_rng(17)
+    n_groups, n_parts = 4000, 5
+    parts = np.abs(rng.normal(0.0, 0.05, (n_parts, n_groups))).astype(np.float32)
+    parts[:, :50] = np.float32(2.0 ** -127) * rng.integers(0, 4, (n_parts, 50)).astype(np.float32)   # subnormal maxima
+    bt = np.where(rng.random(n_groups) < 0.5, rng.integers(2, 12, n_groups), rng.uniform(2.0, 12.0, n_groups)).astype(np.float32)
+    of_parts = np.stack([orc.scale(parts[k], bt) for k in range(n_parts)]).max(axis=0)
+    of_whole = orc.scale(parts.max(axis=0), bt)
+    assert np.array_equal(of_parts.view(np.uint32), of_whole.view(np.uint32))

@@ -20,8 +20,9 @@ from paper_2505_11170_b200.sharding import all_reduce_slots, even_bounds, plan_f
 
 
 def test_even_bounds_are_multiples_of_eight_and_cover_the_tensor():
-    assert even_bounds(1000, 3) == [0, 336, 672, 1000]
-    assert even_bounds(16, 4) == [0, 8, 16, 16, 16]
+    assert even_bounds(1000, 3) == [0, 352, 704, 1000]
+    assert even_bounds(1000, 3, align=8) == [0, 336, 672, 1000]
+    assert even_bounds(16, 4, align=8) == [0, 8, 16, 16, 16]
     assert even_bounds(0, 2) == [0, 0, 0]
     b = even_bounds(2048 * 5632, 8)
     assert b[0] == 0 and b[-1] == 2048 * 5632 and all(x % 8 == 0 for x in b)
