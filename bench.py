@@ -367,7 +367,25 @@ def main():
         probe_desc = Desc.make(n_elem // 2048, 2048, 1, 128, seed=1)
         sink = gws.noise_alu_probe(probe_desc)
         probe_ms = timed(lambda k: gws.noise_alu_probe(probe_desc.with_step(k), sink), 10)
+        # one rank's share of the same set with every tensor cut into 6 flat shards (6 does not divide the tensors, so
+        # every shard has a partial group at each end): the local work of a sharded step, without the two small
+        # all-reduces a real job adds
+        from paper_2505_11170_b200.sharding import ShardedSetSampler, plan_flat_shard
+        shard_world, shard_rank = 6, 2
+        sh_plans = [plan_flat_shard(s_.rows * s_.cols, s_.group_cols or s_.cols, shard_rank, shard_world) for s_ in specs]
+        cut = lambda t, p_: t.view(-1)[p_.begin:p_.end]
+        sh = ShardedSetSampler(sh_plans, [d.seed for d in descs], [cut(W[i], p_) for i, p_ in enumerate(sh_plans)],
+                               [BT[i][p_.first_group:p_.first_group + p_.n_local_groups] for i, p_ in enumerate(sh_plans)],
+                               [cut(WH[i], p_) for i, p_ in enumerate(sh_plans)], [cut(G[i], p_) for i, p_ in enumerate(sh_plans)])
+        sh_elems = sum(p_.n_elements for p_ in sh_plans)
+        sh_fwd_ms = timed(lambda k: sh.forward_finish(k, sh.forward_local(k)), 20)
+        sh_bwd_ms = timed(lambda k: sh.backward_finish(sh.backward_local(k)), 20)
         extras = {
+            "sharded_rank_local_work": {"world": shard_world, "rank": shard_rank, "elements": sh_elems, "end_pieces": sh.n_pieces,
+                                        "fwd_ms": sh_fwd_ms, "bwd_ms": sh_bwd_ms, "launches_per_forward": sh.launches_per_forward,
+                                        "fwd_GB/s": sh_elems * FWD_BYTES_PER_ELEM / (sh_fwd_ms * 1e-3) / 1e9,
+                                        "bwd_GB/s": sh_elems * BWD_BYTES_PER_ELEM / (sh_bwd_ms * 1e-3) / 1e9,
+                                        "note": "each pass reads %.2f GB, more than L2; a real job adds two all-reduces of %d floats" % (sh_elems * 2 / 1e9, len(specs) * (shard_world + 1))},
             "per_layer_launches": {"ms_per_step": per_layer_ms, "launches_per_step": 2 * len(specs),
                                    "GB/s": bytes_per_step / (per_layer_ms * 1e-3) / 1e9},
             "bwd_with_grad_w_copy": {"ms_per_launch": bwd_copy_ms, "GB/s": n_elem * (4 + 8 / 128) / (bwd_copy_ms * 1e-3) / 1e9,
