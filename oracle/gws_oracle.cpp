@@ -46,7 +46,10 @@
 // 10^7 draws; hand-computed add-then-cast cases; library BF16 casts;
 // finite-difference gradients; the Lemma 1 and Proposition 2 invariants;
 // the given-scale forward against the fused one and a numpy restatement, and
-// the facts a sharded pass rests on (partial maxima, partial sums).
+// the facts a sharded pass rests on (partial maxima, partial sums); the MX
+// element grids against their definition, brute-force nearest-even rounding
+// and a library FP8 cast, the shared exponent against its formula, and the
+// transposition property of square blocks.
 // The only thing left unpinned is which of the equally valid bit assignments
 // the authors' own kernels used; their stream cannot be reproduced.
 
@@ -353,6 +356,117 @@ void gwso_sample_bwd(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows,
   const double ln2 = 0.6931471805599453;
   for (int64_t g = 0; g < geo.n_groups; ++g)
     grad_bt[g] = static_cast<float>(-ln2 * static_cast<double>(scale[g]) * acc_scratch[g]);
+}
+
+// ---- w_hat in a microscaling (MX) floating-point format ------------------------------------------------
+//
+// Section 3.1 targets MX formats whose elements are low-precision FP (MXFP), Section 3.2 notes that a
+// square block whose 32-element vectors share one scale is MX-compliant, and Table C.1 lists FP8_e4m3 and
+// FP6_e3m2 as the datatypes that hold w_hat for b_t <= 5 and b_t <= 4.  The paper defines no conversion;
+// this one is the conversion of the OCP Microscaling Formats (MX) specification v1.0 applied to the BF16
+// w_hat, with the paper's sharing rule:
+//   * the scaling block is the sampling group (Eq. 3's b_l x b_l block, or the 1 x G group): every
+//     32-element row vector of a group carries the same scale, so a square block stays consistent under
+//     transposition;
+//   * shared exponent = floor(log2(max_group |w_hat|)) - emax_elem, clamped to the E8M0 range
+//     [-127, 127]; the scale byte is that exponent + 127 (an all-zero or subnormal-only group gets 0);
+//   * element = w_hat / 2^shared_exponent rounded to nearest, ties to even, onto the element grid
+//     (subnormals included); magnitudes beyond the largest normal are clamped to it; the sign of zero
+//     is kept.
+// Element formats: E4M3 = 1 sign, 4 exponent (bias 7), 3 mantissa bits, largest normal 448 = 1.75 * 2^8
+// (emax 8; the code S.1111.111 is NaN and never produced from finite input); E3M2 = 1 sign, 3 exponent
+// (bias 3), 2 mantissa bits, largest normal 28 = 1.75 * 2^4 (emax 4), no NaN or infinity.
+
+struct MxElement {
+  int exponent_bits, mantissa_bits, bias, emax;
+  double max_normal;
+};
+
+static MxElement mx_element(int format) {
+  if (format == 0) return MxElement{4, 3, 7, 8, 448.0};
+  return MxElement{3, 2, 3, 4, 28.0};
+}
+
+// Value of a code of the element format (sign in the top bit of the code's width).
+double gwso_mx_decode(int format, uint32_t code) {
+  const MxElement f = mx_element(format);
+  const int width = 1 + f.exponent_bits + f.mantissa_bits;
+  const uint32_t sign = (code >> (width - 1)) & 1u;
+  const uint32_t e = (code >> f.mantissa_bits) & ((1u << f.exponent_bits) - 1u);
+  const uint32_t m = code & ((1u << f.mantissa_bits) - 1u);
+  double v;
+  if (format == 0 && e == 15u && m == 7u) return std::nan("");
+  if (e == 0)
+    v = std::ldexp(static_cast<double>(m), 1 - f.bias - f.mantissa_bits);
+  else
+    v = std::ldexp(1.0 + std::ldexp(static_cast<double>(m), -f.mantissa_bits), static_cast<int>(e) - f.bias);
+  return sign ? -v : v;
+}
+
+// x (finite) rounded to the element grid: nearest, ties to even, clamped to the largest normal.
+uint32_t gwso_mx_encode(int format, double x) {
+  const MxElement f = mx_element(format);
+  const int width = 1 + f.exponent_bits + f.mantissa_bits;
+  const uint32_t sign = std::signbit(x) ? 1u : 0u;
+  const double a = std::fabs(x);
+  uint32_t magnitude = 0;
+  if (a > 0.0) {
+    int e = static_cast<int>(std::floor(std::log2(a)));
+    if (std::ldexp(1.0, e) > a) --e;          // guard the floating-point log at exact powers of two
+    if (std::ldexp(1.0, e + 1) <= a) ++e;
+    const int e_min = 1 - f.bias;             // exponent of the smallest normal; subnormals share its spacing
+    const int spacing_exp = (e < e_min ? e_min : e) - f.mantissa_bits;
+    const double steps = std::nearbyint(std::ldexp(a, -spacing_exp));   // default rounding mode: ties to even
+    double value = std::ldexp(steps, spacing_exp);
+    if (value > f.max_normal) value = f.max_normal;
+    if (value < std::ldexp(1.0, e_min)) {
+      magnitude = static_cast<uint32_t>(std::ldexp(value, f.bias - 1 + f.mantissa_bits));   // subnormal: exponent field 0
+    } else {
+      int ev = static_cast<int>(std::floor(std::log2(value)));
+      if (std::ldexp(1.0, ev) > value) --ev;
+      if (std::ldexp(1.0, ev + 1) <= value) ++ev;
+      const double frac = std::ldexp(value, -ev) - 1.0;
+      magnitude = (static_cast<uint32_t>(ev + f.bias) << f.mantissa_bits) |
+                  static_cast<uint32_t>(std::ldexp(frac, f.mantissa_bits));
+    }
+  }
+  return (sign << (width - 1)) | magnitude;
+}
+
+// codes[i*cols + j]: one element code per byte (logical order, no ld); scales[i*(cols/32) + j/32]: the
+// E8M0 byte of the 32-element vector.  cols and the resolved group_cols must be multiples of 32.
+void gwso_mx_emit(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols, int format,
+                  const uint16_t* w_hat, uint8_t* codes, uint8_t* scales, float* absmax_scratch) {
+  const MxElement f = mx_element(format);
+  const Geometry geo = make_geometry(rows, cols, ld, group_rows, group_cols);
+  gwso_group_absmax(rows, cols, ld, group_rows, group_cols, w_hat, absmax_scratch);
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const float amax = absmax_scratch[group_of(geo, i, j)];
+      int shared = -127;
+      if (amax > 0.0f) {
+        int e2;
+        std::frexp(amax, &e2);                 // amax = m * 2^e2 with m in [0.5, 1): floor(log2) = e2 - 1
+        shared = (e2 - 1) - f.emax;
+        if (shared < -127) shared = -127;
+        if (shared > 127) shared = 127;
+      }
+      const double scaled = std::ldexp(static_cast<double>(bf16_to_f32(w_hat[i * ld + j])), -shared);
+      codes[i * cols + j] = static_cast<uint8_t>(gwso_mx_encode(format, scaled));
+      if (j % 32 == 0) scales[i * (cols / 32) + j / 32] = static_cast<uint8_t>(shared + 127);
+    }
+}
+
+// Six-bit codes as a little-endian bit stream: code k occupies bits [6k, 6k + 5] of the stream, so 4
+// codes fill 3 bytes and a 32-element vector 24.  n must be a multiple of 4.
+void gwso_mx_pack6(int64_t n, const uint8_t* codes, uint8_t* packed) {
+  for (int64_t b = 0; b < n * 3 / 4; ++b) packed[b] = 0;
+  for (int64_t k = 0; k < n; ++k)
+    for (int bit = 0; bit < 6; ++bit)
+      if ((codes[k] >> bit) & 1u) {
+        const int64_t pos = 6 * k + bit;
+        packed[pos >> 3] |= static_cast<uint8_t>(1u << (pos & 7));
+      }
 }
 
 // ---- bit-width parametrisation and seeds (Section 3.6) ------------------------------------------------

@@ -77,6 +77,15 @@ def lib() -> ctypes.CDLL:
         L.gwso_sample_fwd.restype = None
         L.gwso_sample_fwd_scaled.argtypes = [c_int64] * 5 + [c_uint64] * 3 + [u16p, f32p, u16p]
         L.gwso_sample_fwd_scaled.restype = None
+        u8p = POINTER(ctypes.c_uint8)
+        L.gwso_mx_decode.argtypes = [c_int, c_uint32]
+        L.gwso_mx_decode.restype = c_double
+        L.gwso_mx_encode.argtypes = [c_int, c_double]
+        L.gwso_mx_encode.restype = c_uint32
+        L.gwso_mx_emit.argtypes = [c_int64] * 5 + [c_int, u16p, u8p, u8p, f32p]
+        L.gwso_mx_emit.restype = None
+        L.gwso_mx_pack6.argtypes = [c_int64, u8p, u8p]
+        L.gwso_mx_pack6.restype = None
         L.gwso_sample_bwd_injected.argtypes = [c_int64] * 5 + [u16p, f32p, i8p, u16p, f32p, f64p]
         L.gwso_sample_bwd_injected.restype = None
         L.gwso_sample_bwd.argtypes = [c_int64] * 5 + [c_uint64] * 3 + [u16p, f32p, u16p, f32p, f64p]
@@ -262,3 +271,38 @@ def bitwidth_grad(grad_bt, bt, b_init: float, b_target: float, lam: float) -> np
 
 def layer_seed(user_seed: int, layer: int) -> int:
     return int(lib().gwso_layer_seed(user_seed & 0xFFFFFFFFFFFFFFFF, layer))
+
+
+# ---- w_hat in an MX floating-point format (Section 3.1, Table C.1) ---------------------------------------
+
+MX_E4M3, MX_E3M2 = 0, 1
+
+
+def mx_decode(fmt: int, code: int) -> float:
+    return float(lib().gwso_mx_decode(fmt, code))
+
+
+def mx_encode(fmt: int, x: float) -> int:
+    return int(lib().gwso_mx_encode(fmt, float(x)))
+
+
+def mx_emit(w_hat, rows, cols, group_rows=1, group_cols=0, fmt=MX_E4M3, ld=None):
+    """Returns (codes uint8 [rows*cols], one element code per byte; scales uint8 [rows*cols/32], E8M0)."""
+    ld = cols if ld is None else ld
+    gc = cols if group_cols == 0 else group_cols
+    assert cols % 32 == 0 and gc % 32 == 0, "whole 32-element vectors inside every group expected"
+    w_hat = _check_w(w_hat, rows, cols, ld)
+    codes = np.empty(rows * cols, np.uint8)
+    scales = np.empty(rows * cols // 32, np.uint8)
+    scratch = np.empty(n_groups(rows, cols, group_rows, group_cols), np.float32)
+    lib().gwso_mx_emit(rows, cols, ld, group_rows, group_cols, fmt, _p(w_hat, c_uint16), _p(codes, ctypes.c_uint8),
+                       _p(scales, ctypes.c_uint8), _p(scratch, c_float))
+    return codes, scales
+
+
+def mx_pack6(codes) -> np.ndarray:
+    codes = _c(codes, np.uint8).ravel()
+    assert codes.size % 4 == 0
+    out = np.empty(codes.size * 3 // 4, np.uint8)
+    lib().gwso_mx_pack6(codes.size, _p(codes, ctypes.c_uint8), _p(out, ctypes.c_uint8))
+    return out
