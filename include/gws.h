@@ -160,6 +160,43 @@ int gws_scale_from_absmax(int64_t n_groups, const float* absmax, const float* bt
  */
 int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scale, void* w_hat, void* stream);
 
+/* ---- w_hat in a microscaling (MX) floating-point format -----------------------------------------
+ * Section 3.1 names MX formats with low-precision FP elements as the target of the method and
+ * Table C.1 lists the element types that hold w_hat (FP8_e4m3 up to b_t = 5, FP6_e3m2 up to
+ * b_t = 4); the paper itself stores w_hat in BF16 and defines no conversion.  These calls apply
+ * the conversion of the OCP Microscaling Formats (MX) specification v1.0 to the BF16 w_hat of
+ * Eq. 3, with the sharing rule of Section 3.2: the scaling block is the sampling group, i.e. all
+ * 32-element row vectors of a group (a 32 x 32 block, a 1 x G group, a row) carry the same
+ * scale, which keeps a square block consistent under transposition.
+ *   scale byte (E8M0)  max(E - emax, 0), E = biased exponent of max_group |w_hat|: the shared
+ *                      exponent floor(log2 max) - emax clamped below at -127 (emax = 8 / 4)
+ *   element            w_hat / 2^(byte - 127), round to nearest even onto the element grid
+ *                      (subnormals included), clamped to the largest normal (448 / 28); the
+ *                      sign of zero is kept
+ * Buffer layout (one device allocation per tensor, 32-byte aligned, see gws_mx_layout):
+ *   [0, codes_bytes)            element codes in logical row-major order.  E4M3: one byte each.
+ *                               E3M2: a little-endian bit stream, element k at bits [6k, 6k+5]
+ *                               (4 elements in 3 bytes, a 32-element vector in 24).
+ *   [scales_offset, total)      one scale byte per 32 elements, [rows, cols/32] row-major;
+ *                               scales_offset = codes_bytes rounded up to 256.
+ * Supported tensors (anything else: GWS_ERR_UNSUPPORTED, nothing launched): dense (ld == cols),
+ * cols a multiple of 32, 32-byte aligned pointers, elem_offset as for the fast kernels, and
+ * groups of 1 x {32, 64, 128, 256}, whole rows up to 32768 elements, or 32 x 32 blocks with rows
+ * a multiple of 32.
+ */
+typedef enum gws_mx_format { GWS_MX_FP8_E4M3 = 0, GWS_MX_FP6_E3M2 = 1 } gws_mx_format;
+
+/* Sizes of the MX buffer of a tensor; any of the three outputs may be NULL.  Host arithmetic only. */
+int gws_mx_layout(const gws_desc* desc, int format, size_t* codes_bytes, size_t* scales_offset, size_t* total_bytes);
+
+/* BF16 w_hat (device, read only) -> MX buffer (device, written).  seed / step are not used. */
+int gws_mx_quantize(const gws_desc* desc, int format, const void* w_hat, void* mx_out, void* stream);
+
+/* gws_sample_fwd with the result written as MX instead of BF16, in one pass over W: exactly
+ * gws_mx_quantize applied to the w_hat gws_sample_fwd would have written.  scale_out as there. */
+int gws_sample_fwd_mx(const gws_desc* desc, int format, const void* w, const float* bt, void* mx_out,
+                      float* scale_out, void* stream);
+
 /* ---- many tensors per launch ---------------------------------------------------------------
  * One linear layer of a 1B-parameter model is a few microseconds of HBM time, so a training
  * step samples all layers with as few launches as possible: tensors that run on the same kernel
@@ -244,6 +281,11 @@ int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream
  * between ranks) instead of written; `bt` is not used.  GWS_ERR_NULL if the plan has no forward side
  * or a tensor was prepared without a scale array. */
 int gws_sample_fwd_scaled_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
+
+/* gws_sample_fwd_mx for every tensor of a plan whose `w_hat` pointers are MX buffers (gws_mx_layout)
+ * instead of BF16 tensors.  GWS_ERR_UNSUPPORTED, with nothing launched, if any tensor of the plan is
+ * outside what the MX calls support. */
+int gws_sample_fwd_mx_multi(const gws_multi_plan* plan, int format, uint64_t step, void* stream);
 
 /* ---- bit-width parametrisation and seeds (Section 3.6, "Bitwidth" and "Managing seed") ---------------
  *

@@ -66,6 +66,10 @@ _SIGNATURES = {
     "gws_sample_bwd": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gws_scale_from_absmax": (c_int, [c_int64, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gws_sample_fwd_scaled": (c_int, [POINTER(Desc), c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gws_mx_layout": (c_int, [POINTER(Desc), c_int, POINTER(c_size_t), POINTER(c_size_t), POINTER(c_size_t)]),
+    "gws_mx_quantize": (c_int, [POINTER(Desc), c_int, c_void_p, c_void_p, c_void_p]),
+    "gws_sample_fwd_mx": (c_int, [POINTER(Desc), c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gws_sample_fwd_mx_multi": (c_int, [POINTER(_MultiPlan), c_int, c_uint64, c_void_p]),
     "gws_workspace_bytes": (c_size_t, [c_int]),
     "gws_multi_prepare": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, c_void_p, c_size_t,
                                   POINTER(_MultiPlan), c_void_p]),
@@ -209,6 +213,44 @@ def sample_fwd_scaled(desc: Desc, w: torch.Tensor, scale: torch.Tensor, w_hat: O
     return w_hat
 
 
+MX_FP8_E4M3, MX_FP6_E3M2 = 0, 1
+
+
+def mx_layout(desc: Desc, fmt: int):
+    """(codes_bytes, scales_offset, total_bytes) of the MX buffer of a tensor."""
+    a, b, c = c_size_t(), c_size_t(), c_size_t()
+    _check(load_library().gws_mx_layout(ctypes.byref(desc), fmt, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)))
+    return int(a.value), int(b.value), int(c.value)
+
+
+def _mx_buffer(desc: Desc, fmt: int, mx_out: Optional[torch.Tensor], device) -> torch.Tensor:
+    total = mx_layout(desc, fmt)[2]
+    if mx_out is None:
+        return torch.empty(total, dtype=torch.uint8, device=device)
+    if mx_out.dtype != torch.uint8 or mx_out.numel() < total or not mx_out.is_contiguous():
+        raise ValueError("gws: mx_out must be a contiguous uint8 tensor of at least %d bytes" % total)
+    return mx_out
+
+
+def mx_quantize(desc: Desc, fmt: int, w_hat: torch.Tensor, mx_out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """BF16 w_hat -> MX buffer (uint8; layout of ``mx_layout``)."""
+    _require_cuda(w_hat, mx_out)
+    mx_out = _mx_buffer(desc, fmt, mx_out, w_hat.device)
+    _check(load_library().gws_mx_quantize(ctypes.byref(desc), fmt, _ptr(w_hat), _ptr(mx_out), _stream(stream)))
+    return mx_out
+
+
+def sample_fwd_mx(desc: Desc, fmt: int, w: torch.Tensor, bt: torch.Tensor, mx_out: Optional[torch.Tensor] = None,
+                  scale_out: Optional[torch.Tensor] = None, want_scale: bool = True, stream=None):
+    """Forward sampling with w_hat written as MX.  Returns (mx_out, scale_out)."""
+    _require_cuda(w, bt, mx_out, scale_out)
+    mx_out = _mx_buffer(desc, fmt, mx_out, w.device)
+    if scale_out is None and want_scale:
+        scale_out = torch.empty(n_groups(desc), dtype=torch.float32, device=w.device)
+    _check(load_library().gws_sample_fwd_mx(ctypes.byref(desc), fmt, _ptr(w), _ptr(bt), _ptr(mx_out), _ptr(scale_out), _stream(stream)))
+    return mx_out, scale_out
+
+
 def sample_bwd(desc: Desc, grad_w_hat: torch.Tensor, scale: torch.Tensor, grad_w: Optional[torch.Tensor] = None,
                grad_bt: Optional[torch.Tensor] = None, stream=None):
     """Returns (grad_w, grad_bt); grad_w is ``grad_w_hat`` itself when no copy was requested."""
@@ -291,6 +333,10 @@ class MultiPlan:
 
     def sample_bwd_multi(self, step: int, stream=None) -> None:
         _check(load_library().gws_sample_bwd_multi(ctypes.byref(self.plan), step, _stream(stream)))
+
+    def sample_fwd_mx_multi(self, fmt: int, step: int, stream=None) -> None:
+        """Forward with MX output; the plan's ``w_hat`` tensors are MX buffers (uint8, ``mx_layout``)."""
+        _check(load_library().gws_sample_fwd_mx_multi(ctypes.byref(self.plan), fmt, step, _stream(stream)))
 
     def sample_fwd_scaled_multi(self, step: int, stream=None) -> None:
         """Forward with the factors already in the plan's ``scale`` arrays (read, not written)."""

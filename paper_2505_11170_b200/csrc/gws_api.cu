@@ -129,6 +129,22 @@ Entry make_entry(const gws_desc* d, int cls, const void* in, void* out, const fl
   return e;
 }
 
+// ---- layout of an MX buffer ----------------------------------------------------------------------------
+// Element codes first (E4M3: one byte per element; E3M2: 6 bits per element), then, from the next multiple of
+// 256 bytes, one E8M0 scale byte per 32 elements.
+size_t mx_codes_bytes(int64_t n_elements, int format) {
+  return format == gws::kMxE4M3 ? static_cast<size_t>(n_elements) : static_cast<size_t>(n_elements) / 4u * 3u;
+}
+size_t mx_scales_offset(int64_t n_elements, int format) { return (mx_codes_bytes(n_elements, format) + 255u) & ~static_cast<size_t>(255u); }
+size_t mx_total_bytes(int64_t n_elements, int format) { return mx_scales_offset(n_elements, format) + static_cast<size_t>(n_elements) / 32u; }
+
+// The `pad` field of a record: where the scale bytes start inside the output buffer, in units of 16 bytes (MX modes only).
+template <int MODE>
+uint32_t mx_scales_off16(const Entry& e) {
+  if (!(gws::mode_is_mx_fwd(MODE) || gws::mode_is_mx_quant(MODE))) return 0u;
+  return static_cast<uint32_t>(mx_scales_offset(e.rows * e.cols, gws::mode_mx_format(MODE)) / 16u);
+}
+
 // ---- flat-group launches: tensor records by value in the kernel parameters ---------------------------
 
 gws::FlatRec to_flat_rec(const Entry& e) {
@@ -328,6 +344,7 @@ int launch_square_batch(const Entry* const* entries, int count, uint32_t lo, uin
     r.cpr = static_cast<uint32_t>(e.cols / 32);
     r.k0 = e.seed_lo;
     r.k1 = e.seed_hi;
+    r.pad = mx_scales_off16<MODE>(e);
     bands[k] = static_cast<uint32_t>(e.rows / 32);
   }
   const int64_t tiles = gws::fill_square_batch<CAP>(b, recs, bands, count, lo, hi);
@@ -348,6 +365,46 @@ int launch_squares(const std::vector<const Entry*>& entries, uint64_t step, cuda
     if (st != GWS_OK) return st;
   }
   return GWS_OK;
+}
+
+// ---- MX output (element codes + scale bytes instead of BF16) -----------------------------------------------
+//
+// Only the kernels that work on 64-byte chunks write MX (a chunk is one 32-element MX vector): flat groups of 32
+// to 256 elements, whole rows of a multiple of 32 elements up to 32768, whole 32 x 32 blocks; dense, 32-byte
+// aligned.  Everything else is GWS_ERR_UNSUPPORTED, decided before anything is launched.
+bool mx_entry_ok(int cls, const Entry& e) {
+  if (e.cols % 32 != 0 || e.ld != e.cols || !aligned(e.in, 32) || !aligned(e.out, 32)) return false;
+  if (cls == gws::kFlat) return e.lanes_log2 >= 2u;
+  if (cls == gws::kRowWarp || cls == gws::kRowCta) return row_chunk_eligible(e);
+  return square_eligible(e);
+}
+
+// `count` entries of one kernel class, all of them passing mx_entry_ok.
+template <int MODE>
+int launch_mx(int cls, const Entry* entries, int count, uint64_t step, cudaStream_t stream) {
+  const uint32_t lo = static_cast<uint32_t>(step), hi = static_cast<uint32_t>(step >> 32);
+  if (cls == gws::kFlat) {
+    std::vector<gws::FlatRec> recs;
+    for (int k = 0; k < count; ++k) {
+      gws::FlatRec r = to_flat_rec(entries[k]);
+      r.pad = mx_scales_off16<MODE>(entries[k]);
+      recs.push_back(r);
+    }
+    return launch_flat_variant<MODE, gws::kWide32>(recs, lo, hi, stream);
+  }
+  if (cls == gws::kRowWarp || cls == gws::kRowCta) {
+    std::vector<gws::RowRec> shared_rows, block_rows;
+    for (int k = 0; k < count; ++k) {
+      gws::RowRec r = to_row_rec(entries[k]);
+      r.pad = mx_scales_off16<MODE>(entries[k]);
+      (r.tpr_log2 == 8u ? block_rows : shared_rows).push_back(r);
+    }
+    const int st = launch_row_chunks<MODE, false>(shared_rows, lo, hi, stream);
+    return st != GWS_OK ? st : launch_row_chunks<MODE, true>(block_rows, lo, hi, stream);
+  }
+  std::vector<const Entry*> squares;
+  for (int k = 0; k < count; ++k) squares.push_back(&entries[k]);
+  return launch_squares<MODE>(squares, step, stream);
 }
 
 // One tensor on the vector kernels (row classes) or the general kernel.  The general kernel alone also
@@ -459,6 +516,51 @@ int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scal
   const int cls = classify(desc, aligned(w, 16) && aligned(w_hat, 16));
   const Entry e = make_entry(desc, cls, w, w_hat, nullptr, const_cast<float*>(scale));   // this mode only reads it
   return launch<gws::kFwdScaled>(cls, e, nullptr, 0, tiles_of(desc, cls), desc->step, static_cast<cudaStream_t>(stream));
+}
+
+int gws_mx_layout(const gws_desc* desc, int format, size_t* codes_bytes, size_t* scales_offset, size_t* total_bytes) {
+  const int st = validate_desc(desc);
+  if (st != GWS_OK) return st;
+  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2) return GWS_ERR_UNSUPPORTED;
+  if (desc->cols % 32 != 0) return GWS_ERR_UNSUPPORTED;
+  const int64_t n = desc->rows * desc->cols;
+  if (codes_bytes) *codes_bytes = mx_codes_bytes(n, format);
+  if (scales_offset) *scales_offset = mx_scales_offset(n, format);
+  if (total_bytes) *total_bytes = mx_total_bytes(n, format);
+  return GWS_OK;
+}
+
+int gws_mx_quantize(const gws_desc* desc, int format, const void* w_hat, void* mx_out, void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2) return GWS_ERR_UNSUPPORTED;
+  if (w_hat == nullptr || mx_out == nullptr) return GWS_ERR_NULL;
+  if (!aligned(w_hat, 2)) return GWS_ERR_ALIGN;
+  if (desc->cols % 32 != 0) return GWS_ERR_UNSUPPORTED;
+  if (overlaps(w_hat, span_bytes(desc), mx_out, mx_total_bytes(desc->rows * desc->cols, format))) return GWS_ERR_ALIAS;
+  const int cls = classify(desc, aligned(w_hat, 16) && aligned(mx_out, 16));
+  const Entry e = make_entry(desc, cls, w_hat, mx_out, nullptr, nullptr);
+  if (!mx_entry_ok(cls, e)) return GWS_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  return format == GWS_MX_FP8_E4M3 ? launch_mx<gws::kQuantMx8>(cls, &e, 1, desc->step, s)
+                                   : launch_mx<gws::kQuantMx6>(cls, &e, 1, desc->step, s);
+}
+
+int gws_sample_fwd_mx(const gws_desc* desc, int format, const void* w, const float* bt, void* mx_out, float* scale_out,
+                      void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2) return GWS_ERR_UNSUPPORTED;
+  if (w == nullptr || bt == nullptr || mx_out == nullptr) return GWS_ERR_NULL;
+  if (!aligned(w, 2) || !aligned(bt, 4) || !aligned(scale_out, 4)) return GWS_ERR_ALIGN;
+  if (desc->cols % 32 != 0) return GWS_ERR_UNSUPPORTED;
+  if (overlaps(w, span_bytes(desc), mx_out, mx_total_bytes(desc->rows * desc->cols, format))) return GWS_ERR_ALIAS;
+  const int cls = classify(desc, aligned(w, 16) && aligned(mx_out, 16));
+  const Entry e = make_entry(desc, cls, w, mx_out, bt, scale_out);
+  if (!mx_entry_ok(cls, e)) return GWS_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  return format == GWS_MX_FP8_E4M3 ? launch_mx<gws::kFwdMx8>(cls, &e, 1, desc->step, s)
+                                   : launch_mx<gws::kFwdMx6>(cls, &e, 1, desc->step, s);
 }
 
 int gws_sample_bwd(const gws_desc* desc, const void* grad_w_hat, const float* scale, void* grad_w, float* grad_bt,
@@ -705,7 +807,33 @@ static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
   return GWS_OK;
 }
 
+// Forward pass of a plan with MX output: the w_hat pointers the plan was prepared with are MX buffers.
+template <int MODE>
+static int run_multi_mx(const gws_multi_plan* plan, uint64_t step, void* stream) {
+  if (plan == nullptr) return GWS_ERR_NULL;
+  if (plan->workspace == nullptr || plan->host_tables == nullptr) return GWS_ERR_WORKSPACE;
+  if (!plan->has_fwd) return GWS_ERR_NULL;
+  auto host_table = [&](int cls) {
+    return reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) + plan->fwd_offset[cls]);
+  };
+  for (int cls = 0; cls < 4; ++cls)
+    for (int i = 0; i < plan->count[cls]; ++i)
+      if (!mx_entry_ok(cls, host_table(cls)[i])) return GWS_ERR_UNSUPPORTED;
+  for (int cls = 0; cls < 4; ++cls) {
+    if (plan->count[cls] == 0) continue;
+    const int st = launch_mx<MODE>(cls, host_table(cls), plan->count[cls], step, static_cast<cudaStream_t>(stream));
+    if (st != GWS_OK) return st;
+  }
+  return GWS_OK;
+}
+
 extern "C" {
+
+int gws_sample_fwd_mx_multi(const gws_multi_plan* plan, int format, uint64_t step, void* stream) {
+  if (format == GWS_MX_FP8_E4M3) return run_multi_mx<gws::kFwdMx8>(plan, step, stream);
+  if (format == GWS_MX_FP6_E3M2) return run_multi_mx<gws::kFwdMx6>(plan, step, stream);
+  return GWS_ERR_UNSUPPORTED;
+}
 
 int gws_multi_launch_count(const gws_multi_plan* plan, int backward) {
   if (plan == nullptr) return GWS_ERR_NULL;

@@ -37,7 +37,15 @@ namespace gws {
 
 // kFwdScaled: forward with the per-group factor s_g supplied (in `gin`) instead of derived from this tensor's own
 // maxima: the add and cast of Eq. 3 for a tensor whose groups reach into memory this call does not see.
-enum Mode { kAbsmax = 0, kFwd = 1, kBwd = 2, kFwdScaled = 3 };
+enum Mode { kAbsmax = 0, kFwd = 1, kBwd = 2, kFwdScaled = 3, kFwdMx8 = 4, kFwdMx6 = 5, kQuantMx8 = 6, kQuantMx6 = 7 };
+// kFwdMx*: the forward pass with w_hat written as MX floating point (E4M3 or E3M2 elements, one E8M0 scale per 32
+// elements) instead of BF16; kQuantMx*: that conversion alone, from a BF16 w_hat in `in`.
+enum MxFormat { kMxE4M3 = 0, kMxE3M2 = 1 };
+__host__ __device__ constexpr bool mode_is_mx_fwd(int m) { return m == kFwdMx8 || m == kFwdMx6; }
+__host__ __device__ constexpr bool mode_is_mx_quant(int m) { return m == kQuantMx8 || m == kQuantMx6; }
+__host__ __device__ constexpr bool mode_is_fwd(int m) { return m == kFwd || mode_is_mx_fwd(m); }            // takes maxima of w, writes scale_out
+__host__ __device__ constexpr int mode_mx_format(int m) { return (m == kFwdMx8 || m == kQuantMx8) ? kMxE4M3 : kMxE3M2; }
+__host__ __device__ constexpr bool mode_reads_group_input(int m) { return m != kAbsmax && !mode_is_mx_quant(m); }
 enum KernelClass { kFlat = 0, kRowWarp = 1, kRowCta = 2, kGeneral = 3 };
 
 // Full description of one tensor: the record of the multi-tensor tables and the parameter of the
@@ -45,6 +53,8 @@ enum KernelClass { kFlat = 0, kRowWarp = 1, kRowCta = 2, kGeneral = 3 };
 //   absmax: in = w,           gout = absmax
 //   fwd:    in = w,           out = w_hat,           gin = bt,    gout = scale_out or null
 //   scaled: in = w,           out = w_hat,           gout = scale (read only): the forward record serves both forms
+//   fwd mx: as fwd, out = the MX buffer (element codes, then the scale bytes at the offset the record states)
+//   quant:  in = w_hat (BF16), out = the MX buffer
 //   bwd:    in = grad_w_hat,  out = grad_w or null,  gin = scale, gout = grad_bt
 struct __align__(16) Entry {
   const void* in;
@@ -134,6 +144,16 @@ __device__ __forceinline__ void st_vec32(void* base, uint64_t byte_off, const ui
   asm volatile("st.global.v8.u32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]), "r"(x[4]),
                "r"(x[5]), "r"(x[6]), "r"(x[7])
                : "memory");
+}
+__device__ __forceinline__ void st_vec8(void* base, uint64_t byte_off, uint32_t a, uint32_t b) {
+  char* p = reinterpret_cast<char*>(base) + byte_off;
+  GWS_CHECK(p, 8, 2, );
+  *reinterpret_cast<uint2*>(p) = make_uint2(a, b);
+}
+__device__ __forceinline__ void st_u8(void* base, uint64_t byte_off, uint32_t x) {
+  uint8_t* p = reinterpret_cast<uint8_t*>(base) + byte_off;
+  GWS_CHECK(p, 1, 7, );
+  *p = static_cast<uint8_t>(x);
 }
 __device__ __forceinline__ float ld_f32(const float* base, uint64_t i) {
   GWS_CHECK(base + i, 4, 3, 0.0f);
@@ -233,7 +253,7 @@ __device__ __forceinline__ uint4 sample_vec_t(const uint4& w, const Words4& r, c
 __device__ __forceinline__ uint4 sample_vec(const uint4& w, const Words4& r, const Scale& k) {
   return k.tiny ? sample_vec_t<true>(w, r, k) : sample_vec_t<false>(w, r, k);
 }
-// One 64-byte chunk whose first vector has the (low) Philox counter word v0.
+// One 64-byte chunk whose first vector has the (low) Philox counter word v0.  y may be x (word j depends on word j alone).
 template <bool TINY>
 __device__ __forceinline__ void sample_chunk_t(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
                                                const Scale& sc, uint32_t* y) {
@@ -275,6 +295,56 @@ __device__ __forceinline__ void dot_vec(const uint4& g, const Words4& r, DotAcc&
 // dL/db_t of a group from its scale and the sum of g * 2R.
 __device__ __forceinline__ float grad_bt_of(float scale, float sum_g_2r) {
   return __fmul_rn(__fmul_rn(-kLn2, scale), __fmul_rn(sum_g_2r, 0.5f));
+}
+
+// ---- w_hat as MX floating point ------------------------------------------------------------------------
+//
+// OCP Microscaling conversion of the BF16 w_hat with one scale per sampling group (Section 3.2: vectors of a
+// square block share their scale): scale byte = max(E - emax, 0), E the biased exponent of the group's largest
+// |w_hat| (so the shared exponent floor(log2 max) - emax is clamped at -127), elements = w_hat * 2^(127 - byte)
+// rounded to nearest even onto the element grid and clamped to its largest normal, which is what
+// cvt.rn.satfinite does.  The multiplication by a power of two is exact.
+// Buffer: element codes from byte 0 in chunk order (E4M3: 32 bytes per 32-element chunk; E3M2: 24, code k of the
+// chunk at bits [6k, 6k+5] of a little-endian bit stream), scale bytes from byte 16 * scales_off16, one per chunk.
+template <int FMT>
+__device__ __forceinline__ uint32_t cvt_mx_x2(float upper, float lower) {
+  uint16_t d;
+  if (FMT == kMxE4M3) asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(upper), "f"(lower));
+  else asm("cvt.rn.satfinite.e3m2x2.f32 %0, %1, %2;" : "=h"(d) : "f"(upper), "f"(lower));
+  return d;
+}
+template <int FMT>
+__device__ __forceinline__ void mx_write(void* out, uint32_t scales_off16, uint32_t chunk, const uint32_t* y, float amax) {
+  constexpr int kEmax = FMT == kMxE4M3 ? 8 : 4;
+  const int biased = static_cast<int>(__float_as_uint(amax) >> 23);       // amax >= 0
+  const uint32_t byte = static_cast<uint32_t>(max(biased - kEmax, 0));
+  const uint32_t mult_bits = (254u - byte) << 23;                          // 2^(127 - byte)
+  const float mult = __uint_as_float(mult_bits);
+  uint32_t q[16];                                                          // two codes each, element 2j in the low byte
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float lo = __fmul_rn(__uint_as_float(y[j] << 16), mult);
+    const float hi = fma_bf16(hi16(y[j]), hi16(mult_bits), -0.0f);         // + (-0): keeps the sign of a zero product
+    q[j] = cvt_mx_x2<FMT>(hi, lo);
+  }
+  if (FMT == kMxE4M3) {
+    uint32_t w[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) w[k] = q[2 * k] | (q[2 * k + 1] << 16);
+    st_vec32(out, static_cast<uint64_t>(chunk) * 32u, w);
+  } else {
+    uint32_t v[8];                                                         // 24 bits: four codes
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const uint32_t a = q[2 * k], b = q[2 * k + 1];
+      v[k] = (a & 0x3Fu) | ((a >> 2) & 0xFC0u) | ((b & 0x3Fu) << 12) | (((b >> 2) & 0xFC0u) << 12);
+    }
+    const uint64_t at = static_cast<uint64_t>(chunk) * 24u;
+    st_vec8(out, at, v[0] | (v[1] << 24), (v[1] >> 8) | (v[2] << 16));
+    st_vec8(out, at + 8u, (v[2] >> 16) | (v[3] << 8), v[4] | (v[5] << 24));
+    st_vec8(out, at + 16u, (v[5] >> 8) | (v[6] << 16), (v[6] >> 16) | (v[7] << 8));
+  }
+  st_u8(out, static_cast<uint64_t>(scales_off16) * 16u + chunk, byte);
 }
 
 __device__ __forceinline__ Words4 philox_vec(const Entry& e, uint64_t vec_in_tensor, uint32_t step_lo, uint32_t step_hi) {
@@ -340,7 +410,7 @@ struct FlatRec {
   int32_t tile_begin;       // first tile of this tensor inside its launch
   uint32_t k0, k1;          // seed
   PhiloxPre pre;            // the step- and seed-dependent constants of the first two Philox rounds
-  uint32_t pad;
+  uint32_t pad;             // MX modes: byte offset of the scale bytes inside `out`, in units of 16
 };
 static_assert(sizeof(FlatRec) == 80, "FlatRec layout");
 constexpr int kFlatHint = 128;
@@ -391,6 +461,9 @@ __device__ __forceinline__ void store_chunk(void* base, uint64_t chunk, uint32_t
   }
 }
 __device__ __forceinline__ uint32_t absmax_words4(const uint32_t* x) { return maxabs2(maxabs2(x[0], x[1]), maxabs2(x[2], x[3])); }
+__device__ __forceinline__ uint32_t absmax_chunk(const uint32_t* x) {
+  return maxabs2(maxabs2(absmax_words4(x), absmax_words4(x + 4)), maxabs2(absmax_words4(x + 8), absmax_words4(x + 12)));
+}
 
 // Groups of at least one chunk: `lanes` = chunks per group (1, 2, 4 or 8 neighbouring lanes).
 // A thread handles CPT chunks, 256 chunks apart, all loaded before the first is used.
@@ -408,7 +481,7 @@ __device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t first_chunk
     ok[i] = chunk0 < n_chunks;
     chunk[i] = ok[i] ? chunk0 : n_chunks - 1u;   // keeps the warp whole for the shuffles
     c[i] = load_chunk<USE32>(e.in, chunk[i], 4);
-    gv[i] = (MODE != kAbsmax) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, chunk[i] >> lanes_log2) : 0.0f;
+    gv[i] = mode_reads_group_input(MODE) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, chunk[i] >> lanes_log2) : 0.0f;
   }
 #pragma unroll
   for (int i = 0; i < CPT; ++i) {
@@ -434,21 +507,28 @@ __device__ __forceinline__ void flat_wide(const FlatRec& e, uint32_t first_chunk
       if (ok[i]) store_chunk<USE32>(e.out, chunk[i], 4, y);
       continue;
     }
-    uint32_t m = maxabs2(maxabs2(absmax_words4(c[i].x), absmax_words4(c[i].x + 4)),
-                         maxabs2(absmax_words4(c[i].x + 8), absmax_words4(c[i].x + 12)));
+    uint32_t m = absmax_chunk(c[i].x);
     for (uint32_t o = 1; o < lanes; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     const float a = absmax_finish(m);
     if (MODE == kAbsmax) {
       if (writer) st_f32(e.gout, g, a);
       continue;
     }
+    if (mode_is_mx_quant(MODE)) {   // the chunk is w_hat itself
+      if (ok[i]) mx_write<mode_mx_format(MODE)>(e.out, e.pad, chunk[i], c[i].x, a);
+      continue;
+    }
     const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv[i])));
     Chunk y;
     sample_chunk(c[i].x, v0, e.k0, e.k1, e.pre, sc, y.x);
-    if (ok[i]) {
+    if (mode_is_mx_fwd(MODE)) {
+      uint32_t my = absmax_chunk(y.x);
+      for (uint32_t o = 1; o < lanes; o <<= 1) my = maxabs2(my, __shfl_xor_sync(0xFFFFFFFFu, my, o));
+      if (ok[i]) mx_write<mode_mx_format(MODE)>(e.out, e.pad, chunk[i], y.x, absmax_finish(my));
+    } else if (ok[i]) {
       store_chunk<USE32>(e.out, chunk[i], 4, y);
-      if (writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
     }
+    if (writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
   }
 }
 
@@ -601,7 +681,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
     ok[i] = q[i] < cpr;
     if (ok[i]) {
       c[i] = load_chunk<true>(e.in, row_chunk0 + q[i], 4);
-      gv[i] = (MODE != kAbsmax) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, band * cpr + q[i]) : 0.0f;
+      gv[i] = mode_reads_group_input(MODE) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, band * cpr + q[i]) : 0.0f;
     }
   }
 #pragma unroll
@@ -630,8 +710,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
       store_chunk<true>(e.out, chunk, 4, y);
       continue;
     }
-    uint32_t m = maxabs2(maxabs2(absmax_words4(c[i].x), absmax_words4(c[i].x + 4)),
-                         maxabs2(absmax_words4(c[i].x + 8), absmax_words4(c[i].x + 12)));
+    uint32_t m = absmax_chunk(c[i].x);
 #pragma unroll
     for (uint32_t o = 1; o < 32u; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     const float a = absmax_finish(m);
@@ -639,10 +718,21 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
       if (lane == 0u) st_f32(e.gout, g, a);
       continue;
     }
+    if (mode_is_mx_quant(MODE)) {
+      mx_write<mode_mx_format(MODE)>(e.out, e.pad, chunk, c[i].x, a);
+      continue;
+    }
     const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv[i])));
     Chunk y;
     sample_chunk(c[i].x, v0, e.k0, e.k1, e.pre, sc, y.x);
-    store_chunk<true>(e.out, chunk, 4, y);
+    if (mode_is_mx_fwd(MODE)) {
+      uint32_t my = absmax_chunk(y.x);
+#pragma unroll
+      for (uint32_t o = 1; o < 32u; o <<= 1) my = maxabs2(my, __shfl_xor_sync(0xFFFFFFFFu, my, o));
+      mx_write<mode_mx_format(MODE)>(e.out, e.pad, chunk, y.x, absmax_finish(my));
+    } else {
+      store_chunk<true>(e.out, chunk, 4, y);
+    }
     if (lane == 0u && e.gout != nullptr) st_f32(e.gout, g, sc.s);
   }
 }
@@ -703,6 +793,22 @@ struct RowBatch {
 constexpr int kRowCapSmall = 4, kRowCapLarge = 168;
 constexpr int kRowThreads = 256, kRowMaxCpt = 4;
 
+// Maximum over a row of the per-thread packed maxima: shuffles inside the `span` lanes that share the row, then (BLOCK)
+// one shared-memory step.  AGAIN: red_u may still be read from an earlier use in this block.
+template <bool BLOCK, bool AGAIN>
+__device__ __forceinline__ uint32_t row_maxabs(uint32_t m, uint32_t span, uint32_t lane, uint32_t warp, uint32_t* red_u) {
+  for (uint32_t o = 1; o < span; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if (BLOCK) {
+    if (AGAIN) __syncthreads();
+    if (lane == 0) red_u[warp] = m;
+    __syncthreads();
+    m = red_u[0];
+#pragma unroll
+    for (int w = 1; w < kRowThreads / 32; ++w) m = maxabs2(m, red_u[w]);
+  }
+  return m;
+}
+
 // MAXCPT (1..4): the chunks a thread holds in this launch; sizes the register arrays.
 template <int MODE, bool BLOCK, int CAP, int MAXCPT>
 __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ RowBatch<CAP> b) {
@@ -734,7 +840,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
       for (int i = 0; i < 16; ++i) c[k].x[i] = 0u;
     }
   }
-  const float gv = (MODE != kAbsmax) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, row) : 0.0f;
+  const float gv = mode_reads_group_input(MODE) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, row) : 0.0f;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const uint32_t span = BLOCK ? 32u : tpr;   // lanes of this warp that share the row
 
@@ -769,34 +875,46 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
   if (MODE != kFwdScaled) {
     uint32_t m = 0u;
 #pragma unroll
-    for (int k = 0; k < MAXCPT; ++k)
-      m = maxabs2(m, maxabs2(maxabs2(absmax_words4(c[k].x), absmax_words4(c[k].x + 4)),
-                             maxabs2(absmax_words4(c[k].x + 8), absmax_words4(c[k].x + 12))));
-    for (uint32_t o = 1; o < span; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    if (BLOCK) {
-      if (lane == 0) red_u[warp] = m;
-      __syncthreads();
-      m = red_u[0];
-#pragma unroll
-      for (int w = 1; w < kRowThreads / 32; ++w) m = maxabs2(m, red_u[w]);
-    }
-    a = absmax_finish(m);
+    for (int k = 0; k < MAXCPT; ++k) m = maxabs2(m, absmax_chunk(c[k].x));
+    a = absmax_finish(row_maxabs<BLOCK, false>(m, span, lane, warp, red_u));
   }
   if (MODE == kAbsmax) {
     if (okr && t == 0u) st_f32(e.gout, row, a);
     return;
   }
-  const Scale sc = make_scale(MODE == kFwdScaled ? gv : __fmul_rn(a, pow2_one_minus(gv)));
+  if (mode_is_mx_quant(MODE)) {   // the chunks are w_hat itself
 #pragma unroll
-  for (int k = 0; k < MAXCPT; ++k) {
-    if (!ok[k]) continue;
-    const uint32_t chunk = row_chunk0 + static_cast<uint32_t>(k) * tpr + t;
-    const uint32_t v0 = e.vec_lo + chunk * 4u;
-    Chunk y;
-    sample_chunk(c[k].x, v0, e.k0, e.k1, e.pre, sc, y.x);
-    if (okr) store_chunk<true>(e.out, chunk, 4, y);
+    for (int k = 0; k < MAXCPT; ++k)
+      if (ok[k] && okr) mx_write<mode_mx_format(MODE)>(e.out, e.pad, row_chunk0 + static_cast<uint32_t>(k) * tpr + t, c[k].x, a);
+    return;
   }
-  if (MODE == kFwd && okr && t == 0u && e.gout != nullptr) st_f32(e.gout, row, sc.s);
+  const Scale sc = make_scale(MODE == kFwdScaled ? gv : __fmul_rn(a, pow2_one_minus(gv)));
+  if (mode_is_mx_fwd(MODE)) {
+    // w_hat replaces w in the registers; its row maximum is known only after every chunk has been sampled
+    uint32_t my = 0u;
+#pragma unroll
+    for (int k = 0; k < MAXCPT; ++k) {
+      if (!ok[k]) continue;
+      const uint32_t chunk = row_chunk0 + static_cast<uint32_t>(k) * tpr + t;
+      sample_chunk(c[k].x, e.vec_lo + chunk * 4u, e.k0, e.k1, e.pre, sc, c[k].x);
+      my = maxabs2(my, absmax_chunk(c[k].x));
+    }
+    const float ay = absmax_finish(row_maxabs<BLOCK, true>(my, span, lane, warp, red_u));
+#pragma unroll
+    for (int k = 0; k < MAXCPT; ++k)
+      if (ok[k] && okr) mx_write<mode_mx_format(MODE)>(e.out, e.pad, row_chunk0 + static_cast<uint32_t>(k) * tpr + t, c[k].x, ay);
+  } else {
+#pragma unroll
+    for (int k = 0; k < MAXCPT; ++k) {
+      if (!ok[k]) continue;
+      const uint32_t chunk = row_chunk0 + static_cast<uint32_t>(k) * tpr + t;
+      const uint32_t v0 = e.vec_lo + chunk * 4u;
+      Chunk y;
+      sample_chunk(c[k].x, v0, e.k0, e.k1, e.pre, sc, y.x);
+      if (okr) store_chunk<true>(e.out, chunk, 4, y);
+    }
+  }
+  if (mode_is_fwd(MODE) && okr && t == 0u && e.gout != nullptr) st_f32(e.gout, row, sc.s);
 }
 
 // Host side: as fill_flat_batch.  Tiles: rows per block for shared rows (256 / threads per row), one row per block else.
