@@ -380,7 +380,22 @@ def main():
         sh_elems = sum(p_.n_elements for p_ in sh_plans)
         sh_fwd_ms = timed(lambda k: sh.forward_finish(k, sh.forward_local(k)), 20)
         sh_bwd_ms = timed(lambda k: sh.backward_finish(sh.backward_local(k)), 20)
+        # forward pass with w_hat written as MX floating point instead of BF16 (Table C.1's datatypes for w_hat)
+        fwd_mx = {}
+        for name, fmt, code_bytes in (("fp8_e4m3", gws.MX_FP8_E4M3, 1.0), ("fp6_e3m2", gws.MX_FP6_E3M2, 0.75)):
+            MX = [torch.empty(gws.mx_layout(d, fmt)[2], dtype=torch.uint8, device=dev) for d in descs]
+            mx_plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=MX, scale=SC)
+            ms = timed(lambda k: mx_plan.sample_fwd_mx_multi(fmt, k), 20)
+            per_elem = 2 + code_bytes + 1 / 32 + 8 / 128
+            fwd_mx[name] = {"ms_per_launch": ms, "bytes_per_element": per_elem, "GB/s": n_elem * per_elem / (ms * 1e-3) / 1e9,
+                            "gelem_per_s": n_elem / (ms * 1e-3) / 1e9}
+            # the conversion alone, from the BF16 w_hat of the last forward pass (one launch per tensor)
+            q_ms = timed(lambda k: [gws.mx_quantize(descs[i], fmt, WH[i], mx_out=MX[i]) for i in range(len(specs))], 5)
+            fwd_mx[name]["quantize_only"] = {"ms": q_ms, "launches": len(specs),
+                                             "GB/s": n_elem * (2 + code_bytes + 1 / 32) / (q_ms * 1e-3) / 1e9}
+            del mx_plan, MX
         extras = {
+            "fwd_mx_output": fwd_mx,
             "sharded_rank_local_work": {"world": shard_world, "rank": shard_rank, "elements": sh_elems, "end_pieces": sh.n_pieces,
                                         "fwd_ms": sh_fwd_ms, "bwd_ms": sh_bwd_ms, "launches_per_forward": sh.launches_per_forward,
                                         "fwd_GB/s": sh_elems * FWD_BYTES_PER_ELEM / (sh_fwd_ms * 1e-3) / 1e9,
