@@ -24,7 +24,7 @@ import os
 binding.load_library(_build.CHECK_LIB_PATH if os.path.exists(_build.CHECK_LIB_PATH) else _build.build(self_check=True))
 assert binding.selfcheck_enabled()
 dev = "cuda"
-arena = torch.zeros(96 << 20, dtype=torch.uint8, device=dev)
+arena = torch.zeros(128 << 20, dtype=torch.uint8, device=dev)
 cursor = [0]
 def carve(nbytes, dtype):
     start = (cursor[0] + 255) // 256 * 256
@@ -46,14 +46,23 @@ def run_all(window_inputs_only):
         ins.append((d, w, g, bt, ng))
     split = cursor[0]
     for d, w, g, bt, ng in ins:
+        mx_ok = d.cols %% 32 == 0 and (d.group_rows, d.group_cols) in ((1, 128), (1, 0), (32, 32)) and d.rows %% d.group_rows == 0 \
+            and d.cols <= 32768
+        mx = [carve(binding.mx_layout(d, f)[2], torch.uint8) for f in (0, 1)] if mx_ok else None
         outs.append((carve(w.numel() * 2, torch.bfloat16).view_as(w), carve(ng * 4, torch.float32), carve(ng * 4, torch.float32),
-                     carve(ng * 4, torch.float32), carve(w.numel() * 2, torch.bfloat16).view_as(w)))
+                     carve(ng * 4, torch.float32), carve(w.numel() * 2, torch.bfloat16).view_as(w), mx))
     window = arena[:split] if window_inputs_only else arena[:cursor[0]]
     binding.selfcheck_set_window(window)
-    for (d, w, g, bt, ng), (w_hat, sc, gbt, am, gw) in zip(ins, outs):
+    for (d, w, g, bt, ng), (w_hat, sc, gbt, am, gw, mx) in zip(ins, outs):
         binding.sample_fwd(d, w, bt, w_hat, sc)
         binding.sample_bwd(d, g, sc, gw, gbt)
         binding.group_absmax(d, w, am)
+        binding.scale_from_absmax(am, bt, scale=am)
+        binding.sample_fwd_scaled(d, w, am, w_hat)
+        if mx is not None:
+            for f in (0, 1):
+                binding.sample_fwd_mx(d, f, w, bt, mx_out=mx[f], scale_out=sc)
+                binding.mx_quantize(d, f, w_hat, mx_out=mx[f])
     torch.cuda.synchronize()
     return binding.selfcheck_report()
 report["inside"] = run_all(False)
