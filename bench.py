@@ -384,7 +384,7 @@ def main():
         fwd_mx = {}
         for name, fmt, code_bytes in (("fp8_e4m3", gws.MX_FP8_E4M3, 1.0), ("fp6_e3m2", gws.MX_FP6_E3M2, 0.75)):
             MX = [torch.empty(gws.mx_layout(d, fmt)[2], dtype=torch.uint8, device=dev) for d in descs]
-            mx_plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=MX, scale=SC)
+            mx_plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=MX, scale=SC, mx_format=fmt)
             ms = timed(lambda k: mx_plan.sample_fwd_mx_multi(fmt, k), 20)
             per_elem = 2 + code_bytes + 1 / 32 + 8 / 128
             fwd_mx[name] = {"ms_per_launch": ms, "bytes_per_element": per_elem, "GB/s": n_elem * per_elem / (ms * 1e-3) / 1e9,

@@ -215,6 +215,8 @@ typedef struct gws_multi_ptrs {
   const void* const* grad_w_hat;
   void* const* grad_w; /* array may be NULL, and so may each entry: identity, no copy */
   float* const* grad_bt;
+  int32_t w_hat_kind;  /* what the w_hat pointers are: 0 = BF16 tensors; 1 + gws_mx_format = MX buffers
+                          (gws_mx_layout), to be written by gws_sample_fwd_mx_multi only */
 } gws_multi_ptrs;
 
 /* Caller-owned, filled by gws_multi_prepare, read by the *_multi calls.  Plain data. */
@@ -227,6 +229,8 @@ typedef struct gws_multi_plan {
   int64_t tiles[4];     /* size of each class in its table's units: 1024-vector tiles, 8-row tiles, rows, blocks  */
   int64_t fwd_offset[4], bwd_offset[4]; /* byte offsets of the class tables inside both workspaces          */
   int64_t total_elements;
+  int32_t w_hat_kind;   /* copied from gws_multi_ptrs: a forward call for the other kind of output is refused */
+  int32_t reserved;
 } gws_multi_plan;
 
 /* Bytes gws_multi_prepare needs for n tensors, both of device workspace (256-byte aligned base) and
@@ -282,9 +286,11 @@ int gws_sample_bwd_multi(const gws_multi_plan* plan, uint64_t step, void* stream
  * or a tensor was prepared without a scale array. */
 int gws_sample_fwd_scaled_multi(const gws_multi_plan* plan, uint64_t step, void* stream);
 
-/* gws_sample_fwd_mx for every tensor of a plan whose `w_hat` pointers are MX buffers (gws_mx_layout)
- * instead of BF16 tensors.  GWS_ERR_UNSUPPORTED, with nothing launched, if any tensor of the plan is
- * outside what the MX calls support. */
+/* gws_sample_fwd_mx for every tensor of a plan prepared with w_hat_kind = 1 + format, i.e. whose
+ * `w_hat` pointers are MX buffers (gws_mx_layout) instead of BF16 tensors.  GWS_ERR_UNSUPPORTED, with
+ * nothing launched, if the plan was prepared for another kind of output or any tensor of it is outside
+ * what the MX calls support; gws_sample_fwd_multi and gws_sample_fwd_scaled_multi refuse such a plan
+ * the same way (they would write 2 bytes per element). */
 int gws_sample_fwd_mx_multi(const gws_multi_plan* plan, int format, uint64_t step, void* stream);
 
 /* ---- bit-width parametrisation and seeds (Section 3.6, "Bitwidth" and "Managing seed") ---------------

@@ -46,13 +46,13 @@ class Desc(Structure):
 class _MultiPtrs(Structure):
     _fields_ = [("w", POINTER(c_void_p)), ("bt", POINTER(c_void_p)), ("w_hat", POINTER(c_void_p)),
                 ("scale", POINTER(c_void_p)), ("grad_w_hat", POINTER(c_void_p)), ("grad_w", POINTER(c_void_p)),
-                ("grad_bt", POINTER(c_void_p))]
+                ("grad_bt", POINTER(c_void_p)), ("w_hat_kind", c_int32)]
 
 
 class _MultiPlan(Structure):
     _fields_ = [("workspace", c_void_p), ("host_tables", c_void_p), ("n_tensors", c_int32), ("has_fwd", c_int32), ("has_bwd", c_int32),
                 ("count", c_int32 * 4), ("tiles", c_int64 * 4), ("fwd_offset", c_int64 * 4), ("bwd_offset", c_int64 * 4),
-                ("total_elements", c_int64)]
+                ("total_elements", c_int64), ("w_hat_kind", c_int32), ("reserved", c_int32)]
 
 
 _lib: Optional[ctypes.CDLL] = None
@@ -291,7 +291,8 @@ class MultiPlan:
     """``gws_multi_prepare`` + the two ``*_multi`` launches for a fixed set of tensors."""
 
     def __init__(self, descs: Sequence[Desc], w=None, bt=None, w_hat=None, scale=None, grad_w_hat=None, grad_w=None,
-                 grad_bt=None, stream=None):
+                 grad_bt=None, stream=None, mx_format: Optional[int] = None):
+        """``mx_format``: the ``w_hat`` tensors are MX buffers (uint8, ``mx_layout``) of that format, not BF16."""
         lib = load_library()
         n = len(descs)
         anyt = next(t for group in (w, grad_w_hat) if group is not None for t in group if t is not None)
@@ -300,7 +301,7 @@ class MultiPlan:
         self._descs = (Desc * n)(*descs)
         arrays = [_ptr_array(g, n) for g in self._keep]
         cast = lambda a: ctypes.cast(a, POINTER(c_void_p)) if a is not None else None
-        self._ptrs = _MultiPtrs(*[cast(a) for a in arrays])
+        self._ptrs = _MultiPtrs(*[cast(a) for a in arrays], 0 if mx_format is None else 1 + mx_format)
         nbytes = int(lib.gws_workspace_bytes(n))
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=anyt.device)
         self.plan = _MultiPlan()

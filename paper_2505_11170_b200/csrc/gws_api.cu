@@ -645,6 +645,9 @@ static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs
   if (has_fwd && (ptrs->bt == nullptr || ptrs->w_hat == nullptr)) return GWS_ERR_NULL;
   if (has_bwd && (ptrs->scale == nullptr || ptrs->grad_bt == nullptr)) return GWS_ERR_NULL;
   if (workspace == nullptr || !aligned(workspace, 256) || workspace_bytes < gws_workspace_bytes(n)) return GWS_ERR_WORKSPACE;
+  const int kind = ptrs->w_hat_kind;
+  if (kind != 0 && kind != 1 + GWS_MX_FP8_E4M3 && kind != 1 + GWS_MX_FP6_E3M2) return GWS_ERR_UNSUPPORTED;
+  if (kind != 0 && !has_fwd) return GWS_ERR_NULL;
 
   ClassTables t;
   int64_t total = 0;
@@ -661,7 +664,9 @@ static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs
       const float* bt = ptrs->bt[i];
       if (w == nullptr || w_hat == nullptr || bt == nullptr) return GWS_ERR_NULL;
       if (!aligned(w, 2) || !aligned(w_hat, 2) || !aligned(bt, 4) || !aligned(scale, 4)) return GWS_ERR_ALIGN;
-      if (overlaps(w, span_bytes(d), w_hat, span_bytes(d))) return GWS_ERR_ALIAS;
+      if (kind != 0 && d->cols % 32 != 0) return GWS_ERR_UNSUPPORTED;
+      const size_t out_bytes = kind == 0 ? span_bytes(d) : mx_total_bytes(d->rows * d->cols, kind - 1);
+      if (overlaps(w, span_bytes(d), w_hat, out_bytes)) return GWS_ERR_ALIAS;
       vec_ok = vec_ok && aligned(w, 16) && aligned(w_hat, 16);
     }
     void* gw = nullptr;
@@ -697,6 +702,7 @@ static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs
   plan.has_fwd = has_fwd ? 1 : 0;
   plan.has_bwd = has_bwd ? 1 : 0;
   plan.total_elements = total;
+  plan.w_hat_kind = kind;
   image.clear();
   auto place = [&](std::vector<Entry>& v, int cls, int64_t* where) -> int {
     int64_t running = 0;
@@ -770,6 +776,7 @@ static int run_multi(const gws_multi_plan* plan, uint64_t step, void* stream) {
   if (plan == nullptr) return GWS_ERR_NULL;
   if (plan->workspace == nullptr || plan->host_tables == nullptr) return GWS_ERR_WORKSPACE;
   if (backward ? !plan->has_bwd : !plan->has_fwd) return GWS_ERR_NULL;
+  if (!backward && plan->w_hat_kind != 0) return GWS_ERR_UNSUPPORTED;   // the outputs are MX buffers: too small for BF16
   const Entry none{};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   auto host_table = [&](int cls) {
@@ -813,6 +820,7 @@ static int run_multi_mx(const gws_multi_plan* plan, uint64_t step, void* stream)
   if (plan == nullptr) return GWS_ERR_NULL;
   if (plan->workspace == nullptr || plan->host_tables == nullptr) return GWS_ERR_WORKSPACE;
   if (!plan->has_fwd) return GWS_ERR_NULL;
+  if (plan->w_hat_kind != 1 + gws::mode_mx_format(MODE)) return GWS_ERR_UNSUPPORTED;
   auto host_table = [&](int cls) {
     return reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) + plan->fwd_offset[cls]);
   };

@@ -22,7 +22,7 @@
 //             run of chunks; groups up to a chunk live inside the thread.
 //   k_row     group = one row (a multiple of 32 elements, up to 32768): 1..32 lanes or one block
 //             share a row, whose chunks stay in registers between the max and the add.
-//   k_square  group = the paper's 32 x 32 block: a warp per block, lane = row.
+//   k_square  group = the paper's 32 x 32 block: a warp per pair of neighbouring blocks, 16 lanes per block.
 //   k_row_warp / k_row_cta   whole rows the chunk kernel does not take (16-byte vectors), one tensor
 //             per launch;  k_general  every other shape: one block per group, scalar accesses,
 //             tensor record read from a device table in multi-tensor plans.
@@ -150,6 +150,11 @@ __device__ __forceinline__ void st_vec8(void* base, uint64_t byte_off, uint32_t 
   GWS_CHECK(p, 8, 2, );
   *reinterpret_cast<uint2*>(p) = make_uint2(a, b);
 }
+__device__ __forceinline__ void st_u32(void* base, uint64_t byte_off, uint32_t x) {
+  char* p = reinterpret_cast<char*>(base) + byte_off;
+  GWS_CHECK(p, 4, 2, );
+  *reinterpret_cast<uint32_t*>(p) = x;
+}
 __device__ __forceinline__ void st_u8(void* base, uint64_t byte_off, uint32_t x) {
   uint8_t* p = reinterpret_cast<uint8_t*>(base) + byte_off;
   GWS_CHECK(p, 1, 7, );
@@ -266,6 +271,19 @@ __device__ __forceinline__ void sample_chunk_t(const uint32_t* x, uint32_t v0, u
     for (int j = 0; j < 4; ++j) y[4 * k + j] = sample_pair_t<TINY>(x[4 * k + j], p[j], sc);
   }
 }
+// Half a chunk: 16 elements, two Philox vectors.
+template <bool TINY>
+__device__ __forceinline__ void sample_half_t(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
+                                              const Scale& sc, uint32_t* y) {
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const Words4 r = philox4x32_10_pre(v0 + k, k0, k1, pre);
+    uint32_t p[4];
+    decode8(r, p);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) y[4 * k + j] = sample_pair_t<TINY>(x[4 * k + j], p[j], sc);
+  }
+}
 __device__ __forceinline__ void sample_chunk(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
                                              const Scale& sc, uint32_t* y) {
   if (sc.tiny) sample_chunk_t<true>(x, v0, k0, k1, pre, sc, y);
@@ -313,38 +331,77 @@ __device__ __forceinline__ uint32_t cvt_mx_x2(float upper, float lower) {
   else asm("cvt.rn.satfinite.e3m2x2.f32 %0, %1, %2;" : "=h"(d) : "f"(upper), "f"(lower));
   return d;
 }
+// Scale byte of a group whose largest |w_hat| is `amax`, and the bits of the multiplier 2^(127 - byte).
 template <int FMT>
-__device__ __forceinline__ void mx_write(void* out, uint32_t scales_off16, uint32_t chunk, const uint32_t* y, float amax) {
+__device__ __forceinline__ uint32_t mx_scale_byte(float amax) {
   constexpr int kEmax = FMT == kMxE4M3 ? 8 : 4;
-  const int biased = static_cast<int>(__float_as_uint(amax) >> 23);       // amax >= 0
-  const uint32_t byte = static_cast<uint32_t>(max(biased - kEmax, 0));
-  const uint32_t mult_bits = (254u - byte) << 23;                          // 2^(127 - byte)
+  return static_cast<uint32_t>(max(static_cast<int>(__float_as_uint(amax) >> 23) - kEmax, 0));   // amax >= 0: no sign bit
+}
+__device__ __forceinline__ uint32_t mx_mult_bits(uint32_t byte) { return (254u - byte) << 23; }
+
+// Codes of 16 elements (8 packed BF16 pairs): E4M3 -> 4 words, E3M2 -> 3 words (four 6-bit codes per 3 bytes).
+template <int FMT>
+__device__ __forceinline__ void mx_encode_half(const uint32_t* y, uint32_t mult_bits, uint32_t* out) {
   const float mult = __uint_as_float(mult_bits);
-  uint32_t q[16];                                                          // two codes each, element 2j in the low byte
+  uint32_t q[8];                                                           // two codes each, element 2j in the low byte
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
+  for (int j = 0; j < 8; ++j) {
     const float lo = __fmul_rn(__uint_as_float(y[j] << 16), mult);
     const float hi = fma_bf16(hi16(y[j]), hi16(mult_bits), -0.0f);         // + (-0): keeps the sign of a zero product
     q[j] = cvt_mx_x2<FMT>(hi, lo);
   }
   if (FMT == kMxE4M3) {
-    uint32_t w[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) w[k] = q[2 * k] | (q[2 * k + 1] << 16);
-    st_vec32(out, static_cast<uint64_t>(chunk) * 32u, w);
+    for (int k = 0; k < 4; ++k) out[k] = q[2 * k] | (q[2 * k + 1] << 16);
   } else {
-    uint32_t v[8];                                                         // 24 bits: four codes
+    uint32_t v[4];                                                         // 24 bits: four codes
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < 4; ++k) {
       const uint32_t a = q[2 * k], b = q[2 * k + 1];
       v[k] = (a & 0x3Fu) | ((a >> 2) & 0xFC0u) | ((b & 0x3Fu) << 12) | (((b >> 2) & 0xFC0u) << 12);
     }
+    out[0] = v[0] | (v[1] << 24);
+    out[1] = (v[1] >> 8) | (v[2] << 16);
+    out[2] = (v[2] >> 16) | (v[3] << 8);
+  }
+}
+// One whole 32-element vector (chunk) held by one thread.
+template <int FMT>
+__device__ __forceinline__ void mx_write(void* out, uint32_t scales_off16, uint32_t chunk, const uint32_t* y, float amax) {
+  const uint32_t byte = mx_scale_byte<FMT>(amax), mult_bits = mx_mult_bits(byte);
+  if (FMT == kMxE4M3) {
+    uint32_t w[8];
+    mx_encode_half<FMT>(y, mult_bits, w);
+    mx_encode_half<FMT>(y + 8, mult_bits, w + 4);
+    st_vec32(out, static_cast<uint64_t>(chunk) * 32u, w);
+  } else {
+    uint32_t w[6];
+    mx_encode_half<FMT>(y, mult_bits, w);
+    mx_encode_half<FMT>(y + 8, mult_bits, w + 3);
     const uint64_t at = static_cast<uint64_t>(chunk) * 24u;
-    st_vec8(out, at, v[0] | (v[1] << 24), (v[1] >> 8) | (v[2] << 16));
-    st_vec8(out, at + 8u, (v[2] >> 16) | (v[3] << 8), v[4] | (v[5] << 24));
-    st_vec8(out, at + 16u, (v[5] >> 8) | (v[6] << 16), (v[6] >> 16) | (v[7] << 8));
+    st_vec8(out, at, w[0], w[1]);
+    st_vec8(out, at + 8u, w[2], w[3]);
+    st_vec8(out, at + 16u, w[4], w[5]);
   }
   st_u8(out, static_cast<uint64_t>(scales_off16) * 16u + chunk, byte);
+}
+// Half `h` (16 elements) of the vector `chunk`; the thread with the first half also writes the scale byte.
+template <int FMT>
+__device__ __forceinline__ void mx_write_half(void* out, uint32_t scales_off16, uint32_t chunk, uint32_t h, const uint32_t* y, float amax) {
+  const uint32_t byte = mx_scale_byte<FMT>(amax), mult_bits = mx_mult_bits(byte);
+  if (FMT == kMxE4M3) {
+    uint32_t w[4];
+    mx_encode_half<FMT>(y, mult_bits, w);
+    st_vec(out, static_cast<uint64_t>(chunk) * 2u + h, make_uint4(w[0], w[1], w[2], w[3]));
+  } else {
+    uint32_t w[3];
+    mx_encode_half<FMT>(y, mult_bits, w);
+    const uint64_t at = static_cast<uint64_t>(chunk) * 24u + h * 12u;
+    st_u32(out, at, w[0]);
+    st_u32(out, at + 4u, w[1]);
+    st_u32(out, at + 8u, w[2]);
+  }
+  if (h == 0u) st_u8(out, static_cast<uint64_t>(scales_off16) * 16u + chunk, byte);
 }
 
 __device__ __forceinline__ Words4 philox_vec(const Entry& e, uint64_t vec_in_tensor, uint32_t step_lo, uint32_t step_hi) {
@@ -629,11 +686,12 @@ inline int64_t fill_flat_batch(FlatBatch<CAP>& b, const FlatRec* recs, int count
 
 // ---- the paper's square blocks: 32 x 32 elements (Eq. 3, b_l = 32) -------------------------------------
 //
-// A 32 x 32 block is one 64-byte chunk in each of 32 consecutive rows: a warp takes one block, lane =
-// row, so the block maximum and the gradient sum are full-warp shuffle reductions and every lane still
-// moves 64 contiguous bytes.  The 8 warps of a thread block take 8 neighbouring blocks of the same 32
-// rows (512 contiguous bytes per row), CPT of them each.  Tensors with whole blocks only (rows and
-// cols multiples of 32), dense and 32-byte aligned; the general kernel covers the rest.
+// A 32 x 32 block is 64 bytes in each of 32 consecutive rows.  A warp takes two neighbouring blocks (128
+// contiguous bytes per row) and reads 8 rows per access, four lanes per row, so an access touches 8 cache
+// lines; with a lane per row it touched 32, and the L1 data pipe, not HBM, set the pace.  The 16 lanes of a
+// block reduce its maximum and its gradient sum with four shuffle steps.  The 8 warps of a thread block
+// take 16 neighbouring blocks of the same 32 rows (1 KiB contiguous per row).  Tensors with whole blocks
+// only (rows and cols multiples of 32), dense and 32-byte aligned; the general kernel covers the rest.
 struct SquareRec {
   const void* in;
   void* out;
@@ -660,7 +718,6 @@ constexpr int kSquareCpt = 2;
 
 template <int MODE, int CAP>
 __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__ SquareBatch<CAP> b) {
-  constexpr int CPT = kSquareCpt;
   const int32_t tile = static_cast<int32_t>(blockIdx.x);
   int idx = b.hint[tile >> b.hint_shift];
   while (idx + 1 < b.n && b.e[idx + 1].tile_begin <= tile) ++idx;
@@ -669,72 +726,98 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
   const uint32_t band = local / e.tiles_per_band, in_band = local - band * e.tiles_per_band;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const uint32_t cpr = e.cpr;
-  const uint32_t row_chunk0 = (band * 32u + lane) * cpr;
-
-  uint32_t q[CPT];
-  bool ok[CPT];       // uniform over the warp
-  Chunk c[CPT];
-  float gv[CPT];
+  // A warp takes two neighbouring blocks: 128 contiguous bytes of each of 32 rows.  One access covers 8 rows: lanes
+  // 4r..4r+3 read the four 32-byte pieces of row r, so the warp touches 8 cache lines instead of 32.  A lane holds
+  // one piece (16 elements: half of a block's row) of rows 8k + (lane >> 2), k = 0..3, all in the block `blk`.
+  const uint32_t blk = in_band * (8u * kSquareCpt) + warp * 2u + ((lane & 3u) >> 1);
+  const uint32_t half = lane & 1u;
+  const bool ok = blk < cpr;                      // the same for the 16 lanes that share a block
+  const uint32_t g = band * cpr + blk;
+  const bool writer = ok && (lane & ~2u) == 0u;   // lanes 0 and 2: first piece of each block
+  uint32_t piece[4];                              // index of the 32-byte piece in the tensor
+  uint32_t x[4][8];
 #pragma unroll
-  for (int i = 0; i < CPT; ++i) {
-    q[i] = in_band * (8u * CPT) + static_cast<uint32_t>(i) * 8u + warp;
-    ok[i] = q[i] < cpr;
-    if (ok[i]) {
-      c[i] = load_chunk<true>(e.in, row_chunk0 + q[i], 4);
-      gv[i] = mode_reads_group_input(MODE) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, band * cpr + q[i]) : 0.0f;
-    }
-  }
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t row = band * 32u + 8u * static_cast<uint32_t>(k) + (lane >> 2);
+    piece[k] = (row * cpr + blk) * 2u + half;
+    if (ok) {
+      const Vec32 v = ld_vec32(e.in, static_cast<uint64_t>(piece[k]) * 32u);
 #pragma unroll
-  for (int i = 0; i < CPT; ++i) {
-    if (!ok[i]) continue;
-    const uint32_t g = band * cpr + q[i];
-    const uint32_t chunk = row_chunk0 + q[i];
-    const uint32_t v0 = e.vec_lo + chunk * 4u;
-    if (MODE == kBwd) {
-      DotAcc dot;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const Words4 r = philox4x32_10_pre(v0 + k, e.k0, e.k1, e.pre);
-        dot_vec(make_uint4(c[i].x[4 * k], c[i].x[4 * k + 1], c[i].x[4 * k + 2], c[i].x[4 * k + 3]), r, dot);
-      }
-      float acc = dot.total();
-#pragma unroll
-      for (uint32_t o = 1; o < 32u; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-      if (lane == 0u) st_f32(e.gout, g, grad_bt_of(gv[i], acc));
-      if (e.out != nullptr) store_chunk<true>(e.out, chunk, 4, c[i]);
-      continue;
-    }
-    if (MODE == kFwdScaled) {
-      Chunk y;
-      sample_chunk(c[i].x, v0, e.k0, e.k1, e.pre, make_scale(gv[i]), y.x);
-      store_chunk<true>(e.out, chunk, 4, y);
-      continue;
-    }
-    uint32_t m = absmax_chunk(c[i].x);
-#pragma unroll
-    for (uint32_t o = 1; o < 32u; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    const float a = absmax_finish(m);
-    if (MODE == kAbsmax) {
-      if (lane == 0u) st_f32(e.gout, g, a);
-      continue;
-    }
-    if (mode_is_mx_quant(MODE)) {
-      mx_write<mode_mx_format(MODE)>(e.out, e.pad, chunk, c[i].x, a);
-      continue;
-    }
-    const Scale sc = make_scale(__fmul_rn(a, pow2_one_minus(gv[i])));
-    Chunk y;
-    sample_chunk(c[i].x, v0, e.k0, e.k1, e.pre, sc, y.x);
-    if (mode_is_mx_fwd(MODE)) {
-      uint32_t my = absmax_chunk(y.x);
-#pragma unroll
-      for (uint32_t o = 1; o < 32u; o <<= 1) my = maxabs2(my, __shfl_xor_sync(0xFFFFFFFFu, my, o));
-      mx_write<mode_mx_format(MODE)>(e.out, e.pad, chunk, y.x, absmax_finish(my));
+      for (int i = 0; i < 8; ++i) x[k][i] = v.v[i];
     } else {
-      store_chunk<true>(e.out, chunk, 4, y);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[k][i] = 0u;
     }
-    if (lane == 0u && e.gout != nullptr) st_f32(e.gout, g, sc.s);
   }
+  const float gv = (ok && mode_reads_group_input(MODE)) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, g) : 0.0f;
+  // shuffles over the 16 lanes of a block: they differ in bit 0 (half) and bits 2..4 (row)
+  auto block_max = [](uint32_t m) {
+    m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+#pragma unroll
+    for (uint32_t o = 4; o < 32u; o <<= 1) m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    return m;
+  };
+
+  if (MODE == kBwd) {
+    DotAcc dot;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t v0 = e.vec_lo + piece[k] * 2u;
+#pragma unroll
+      for (int v = 0; v < 2; ++v) {
+        const Words4 r = philox4x32_10_pre(v0 + v, e.k0, e.k1, e.pre);
+        dot_vec(make_uint4(x[k][4 * v], x[k][4 * v + 1], x[k][4 * v + 2], x[k][4 * v + 3]), r, dot);   // zero pieces add nothing
+      }
+      if (ok && e.out != nullptr) st_vec32(e.out, static_cast<uint64_t>(piece[k]) * 32u, x[k]);
+    }
+    float acc = dot.total();
+    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
+#pragma unroll
+    for (uint32_t o = 4; o < 32u; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if (writer) st_f32(e.gout, g, grad_bt_of(gv, acc));
+    return;
+  }
+
+  float a = 0.0f;
+  if (MODE != kFwdScaled) {
+    uint32_t m = 0u;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) m = maxabs2(m, maxabs2(absmax_words4(x[k]), absmax_words4(x[k] + 4)));
+    a = absmax_finish(block_max(m));
+  }
+  if (MODE == kAbsmax) {
+    if (writer) st_f32(e.gout, g, a);
+    return;
+  }
+  if (mode_is_mx_quant(MODE)) {   // the pieces are w_hat itself
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (ok) mx_write_half<mode_mx_format(MODE)>(e.out, e.pad, piece[k] >> 1, half, x[k], a);
+    return;
+  }
+  const Scale sc = make_scale(MODE == kFwdScaled ? gv : __fmul_rn(a, pow2_one_minus(gv)));
+  if (mode_is_mx_fwd(MODE)) {
+    uint32_t my = 0u;               // w_hat replaces w in the registers until the block maximum is known
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (sc.tiny) sample_half_t<true>(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, x[k]);
+      else sample_half_t<false>(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, x[k]);
+      my = maxabs2(my, maxabs2(absmax_words4(x[k]), absmax_words4(x[k] + 4)));
+    }
+    const float ay = absmax_finish(block_max(my));
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (ok) mx_write_half<mode_mx_format(MODE)>(e.out, e.pad, piece[k] >> 1, half, x[k], ay);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      uint32_t y[8];
+      if (sc.tiny) sample_half_t<true>(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, y);
+      else sample_half_t<false>(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, y);
+      if (ok) st_vec32(e.out, static_cast<uint64_t>(piece[k]) * 32u, y);
+    }
+  }
+  if (mode_is_fwd(MODE) && writer && e.gout != nullptr) st_f32(e.gout, g, sc.s);
 }
 
 // Host side: `bands[k]` = rows / 32 of record k.  Returns the number of tiles.

@@ -1,0 +1,118 @@
+"""Throughput of the sampling pass on the other workload shapes of the paper (one JSON line each).
+
+    python -m paper_2505_11170_b200.throughput [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [--reps N] [--blocks B]
+
+gpt2         all GPT2-124M linear weights, one group per row (and the same set with groups of 128)
+gpt2_single  one GPT2-124M MLP weight, both orientations
+stress       4096^2, 8192^2, 28672 x 8192 with groups of 32, 128 and whole rows
+square       Llama2-1B-shaped blocks with the paper's 32 x 32 groups (Eq. 3, b_l = 32)
+llama        the Llama2-1B-shaped set with groups of 128 (the benchmark's workload; --blocks limits it)
+mx           the same set with w_hat written as MX FP8 / FP6 instead of BF16
+
+Every timed pass is one multi-tensor launch set over the whole workload, timed with CUDA events on the launching
+stream after three warm-up passes; a 256 MiB buffer is written between passes so that no pass finds its inputs in L2.
+Bytes are the algorithmic ones (read W, write w_hat, read b_t, write scale; read grad, read scale, write grad_bt).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import torch
+
+from . import binding as gws
+from . import synthetic as syn
+from .binding import Desc
+
+_ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _peak_gbs() -> float:
+    try:
+        with open(os.path.join(_ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"])
+    except (OSError, KeyError, ValueError):
+        return 6650.0
+
+
+def run(name: str, specs, reps: int, dev, mx_format=None) -> dict:
+    n = syn.total_elements(specs)
+    descs = [Desc.make(s.rows, s.cols, s.group_rows, s.group_cols, seed=syn.layer_seed(0, i)) for i, s in enumerate(specs)]
+    W = [syn.weights(s, i, device=dev) for i, s in enumerate(specs)]
+    BT = [syn.bitwidths(s, i, device=dev) for i, s in enumerate(specs)]
+    G = [syn.upstream_grad(s, i, device=dev) for i, s in enumerate(specs)]
+    if mx_format is None:
+        WH = [torch.empty_like(t) for t in W]
+        out_bytes = 2.0
+    else:
+        WH = [torch.empty(gws.mx_layout(d, mx_format)[2], dtype=torch.uint8, device=dev) for d in descs]
+        out_bytes = (1.0 if mx_format == gws.MX_FP8_E4M3 else 0.75) + 1.0 / 32.0
+    SC = [torch.empty(s.n_groups, device=dev) for s in specs]
+    GBT = [torch.empty(s.n_groups, device=dev) for s in specs]
+    fwd_plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=WH, scale=SC, mx_format=mx_format)
+    bwd_plan = gws.MultiPlan(descs, scale=SC, grad_w_hat=G, grad_bt=GBT)
+    forward = (lambda k: fwd_plan.sample_fwd_multi(k)) if mx_format is None else (lambda k: fwd_plan.sample_fwd_mx_multi(mx_format, k))
+    n_groups = sum(s.n_groups for s in specs)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    t_fwd = t_bwd = 0.0
+    for k in range(3 + reps):
+        flush.zero_()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        forward(k)
+        e[1].record()
+        bwd_plan.sample_bwd_multi(k)
+        e[2].record()
+        torch.cuda.synchronize()
+        if k >= 3:
+            t_fwd += e[0].elapsed_time(e[1])
+            t_bwd += e[1].elapsed_time(e[2])
+    t_fwd, t_bwd = t_fwd / reps, t_bwd / reps
+    fwd_bytes = n * (2.0 + out_bytes) + n_groups * 8
+    bwd_bytes = n * 2.0 + n_groups * 8
+    peak = _peak_gbs()
+    line = {"workload": name, "elements": n, "tensors": len(specs), "output": "bf16" if mx_format is None else ("mx_fp8_e4m3", "mx_fp6_e3m2")[mx_format],
+            "fwd_us": t_fwd * 1e3, "fwd_GB/s": fwd_bytes / t_fwd / 1e6, "fwd_frac_of_measured_hbm": fwd_bytes / t_fwd / 1e6 / peak,
+            "bwd_us": t_bwd * 1e3, "bwd_GB/s": bwd_bytes / t_bwd / 1e6, "bwd_frac_of_measured_hbm": bwd_bytes / t_bwd / 1e6 / peak,
+            "launches_fwd": fwd_plan.launches_per_pass, "launches_bwd": bwd_plan.launches_per_pass, "reps": reps, "l2": "flushed between passes"}
+    print(json.dumps(line), flush=True)
+    return line
+
+
+def main(argv=None) -> None:
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("which", nargs="*", default=["gpt2", "stress"])
+    ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--blocks", type=int, default=22, help="transformer blocks of the Llama-shaped sets")
+    args = ap.parse_args(argv)
+    if not torch.cuda.is_available():
+        raise SystemExit("a CUDA device is needed: the sampling pass has no CPU path")
+    gws.load_library()
+    dev = torch.device("cuda", 0)
+    for w in args.which:
+        if w == "gpt2":
+            run("gpt2_124m all linear weights, row groups", syn.gpt2_124m_all(), args.reps, dev)
+            run("gpt2_124m all linear weights, groups of 128", syn.gpt2_124m_all(128), args.reps, dev)
+        elif w == "gpt2_single":
+            run("gpt2_124m fc 3072x768, row groups", syn.gpt2_124m_single(), args.reps, dev)
+            run("gpt2_124m fc 768x3072 (literal orientation), row groups", syn.gpt2_124m_single(True), args.reps, dev)
+        elif w == "stress":
+            for rows, cols in syn.STRESS_SHAPES:
+                for g in syn.STRESS_GROUPS:
+                    run(f"{rows}x{cols}, groups of {g or 'one row'}", [syn.stress_case(rows, cols, g)], args.reps, dev)
+        elif w == "square":
+            specs = [syn.TensorSpec(s.name, s.rows, s.cols, 32, 32) for s in syn.llama2_1b(n_blocks=min(args.blocks, 4))]
+            run(f"llama2_1b blocks 0-{min(args.blocks, 4) - 1}, 32x32 groups", specs, args.reps, dev)
+        elif w == "llama":
+            run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev)
+        elif w == "mx":
+            for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2):
+                run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev, mx_format=fmt)
+        else:
+            raise SystemExit(f"unknown workload {w!r}")
+
+
+if __name__ == "__main__":
+    main(sys.argv[1:])

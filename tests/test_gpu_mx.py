@@ -94,12 +94,21 @@ def test_many_tensors_share_launches(fmt_gpu, fmt_orc):
     BT = [torch.randint(3, 7, (gws.n_groups(d),), generator=torch.Generator().manual_seed(k)).float().to(DEV) for k, d in enumerate(descs)]
     OUT = [torch.zeros(gws.mx_layout(d, fmt_gpu)[2], dtype=torch.uint8, device=DEV) for d in descs]
     SC = [torch.empty(gws.n_groups(d), device=DEV) for d in descs]
-    plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=OUT, scale=SC)
+    plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=OUT, scale=SC, mx_format=fmt_gpu)
     before = gws.launch_count()
     plan.sample_fwd_mx_multi(fmt_gpu, 9)
     launches = gws.launch_count() - before
     torch.cuda.synchronize()
     assert launches <= 5                    # flat, rows shared by a warp (by chunks per thread), block rows, squares
+    # a plan is prepared for one kind of output; every other forward call on it is refused before anything is launched
+    lib = gws.load_library()
+    before = gws.launch_count()
+    assert lib.gws_sample_fwd_multi(ctypes.byref(plan.plan), 9, None) == binding.ERR_UNSUPPORTED
+    assert lib.gws_sample_fwd_scaled_multi(ctypes.byref(plan.plan), 9, None) == binding.ERR_UNSUPPORTED
+    assert lib.gws_sample_fwd_mx_multi(ctypes.byref(plan.plan), 1 - fmt_gpu, 9, None) == binding.ERR_UNSUPPORTED
+    bf16_plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=[torch.empty_like(t) for t in W], scale=SC)
+    assert lib.gws_sample_fwd_mx_multi(ctypes.byref(bf16_plan.plan), fmt_gpu, 9, None) == binding.ERR_UNSUPPORTED
+    assert gws.launch_count() == before
     for k, (r, c, gr, gc) in enumerate(shapes):
         want_hat, want_scale = orc.sample_fwd(bits_of(W[k]), BT[k].cpu().numpy(), r, c, gr, gc, seed=100 + k, step=9)
         want_codes, want_scales = _want(want_hat, r, c, gr, gc, fmt_orc)
