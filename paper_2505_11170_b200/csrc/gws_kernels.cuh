@@ -729,27 +729,23 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
   // A warp takes two neighbouring blocks: 128 contiguous bytes of each of 32 rows.  One access covers 8 rows: lanes
   // 4r..4r+3 read the four 32-byte pieces of row r, so the warp touches 8 cache lines instead of 32.  A lane holds
   // one piece (16 elements: half of a block's row) of rows 8k + (lane >> 2), k = 0..3, all in the block `blk`.
-  const uint32_t blk = in_band * (8u * kSquareCpt) + warp * 2u + ((lane & 3u) >> 1);
+  const uint32_t blk0 = in_band * (8u * kSquareCpt) + warp * 2u + ((lane & 3u) >> 1);
   const uint32_t half = lane & 1u;
-  const bool ok = blk < cpr;                      // the same for the 16 lanes that share a block
+  const bool ok = blk0 < cpr;                     // the same for the 16 lanes that share a block
+  const uint32_t blk = ok ? blk0 : cpr - 1u;      // lanes past the last block redo it and store nothing
   const uint32_t g = band * cpr + blk;
   const bool writer = ok && (lane & ~2u) == 0u;   // lanes 0 and 2: first piece of each block
+  const uint32_t piece0 = ((band * 32u + (lane >> 2)) * cpr + blk) * 2u + half, piece_step = 16u * cpr;   // 8 rows on
   uint32_t piece[4];                              // index of the 32-byte piece in the tensor
   uint32_t x[4][8];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    const uint32_t row = band * 32u + 8u * static_cast<uint32_t>(k) + (lane >> 2);
-    piece[k] = (row * cpr + blk) * 2u + half;
-    if (ok) {
-      const Vec32 v = ld_vec32(e.in, static_cast<uint64_t>(piece[k]) * 32u);
+    piece[k] = piece0 + static_cast<uint32_t>(k) * piece_step;
+    const Vec32 v = ld_vec32(e.in, static_cast<uint64_t>(piece[k]) * 32u);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) x[k][i] = v.v[i];
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) x[k][i] = 0u;
-    }
+    for (int i = 0; i < 8; ++i) x[k][i] = v.v[i];
   }
-  const float gv = (ok && mode_reads_group_input(MODE)) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, g) : 0.0f;
+  const float gv = mode_reads_group_input(MODE) ? ld_f32(MODE == kFwdScaled ? e.gout : e.gin, g) : 0.0f;
   // shuffles over the 16 lanes of a block: they differ in bit 0 (half) and bits 2..4 (row)
   auto block_max = [](uint32_t m) {
     m = maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
@@ -766,7 +762,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
 #pragma unroll
       for (int v = 0; v < 2; ++v) {
         const Words4 r = philox4x32_10_pre(v0 + v, e.k0, e.k1, e.pre);
-        dot_vec(make_uint4(x[k][4 * v], x[k][4 * v + 1], x[k][4 * v + 2], x[k][4 * v + 3]), r, dot);   // zero pieces add nothing
+        dot_vec(make_uint4(x[k][4 * v], x[k][4 * v + 1], x[k][4 * v + 2], x[k][4 * v + 3]), r, dot);
       }
       if (ok && e.out != nullptr) st_vec32(e.out, static_cast<uint64_t>(piece[k]) * 32u, x[k]);
     }
