@@ -165,3 +165,76 @@ def test_config5_sample_then_gemm_unfused():
             # BF16 output rounding (2^-8 relative, with margin) plus FP32 accumulation error relative to sum |x||w|
             budget = 2.0 ** -8 * abs(want) + 1e-5 * float(np.abs(x[m].double().cpu().numpy()) @ np.abs(wn)) + 1e-30
             assert abs(got - want) <= budget, (m, n, got, want)
+
+
+@pytest.mark.parametrize("fmt_gpu,fmt_orc", [(gws.MX_FP8_E4M3, orc.MX_E4M3), (gws.MX_FP6_E3M2, orc.MX_E3M2)])
+def test_config3_with_mx_output_on_row_slices(fmt_gpu, fmt_orc):
+    # the whole Llama2-1B-shaped set in one launch with w_hat written as MX; the oracle on a slice of every tensor
+    specs = syn.llama2_1b()
+    descs = [Desc.make(s.rows, s.cols, 1, s.group_cols, seed=syn.layer_seed(0, i)) for i, s in enumerate(specs)]
+    W = [syn.weights(s, i, device=DEV) for i, s in enumerate(specs)]
+    BT = [syn.bitwidths(s, i, device=DEV) for i, s in enumerate(specs)]
+    SC = [torch.empty(s.n_groups, device=DEV) for s in specs]
+    MX = [torch.empty(gws.mx_layout(d, fmt_gpu)[2], dtype=torch.uint8, device=DEV) for d in descs]
+    plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=MX, scale=SC, mx_format=fmt_gpu)
+    assert plan.launches_per_pass == 1
+    step = 4
+    plan.sample_fwd_mx_multi(fmt_gpu, step)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(11)
+    code_bytes_per_row = lambda cols: cols if fmt_orc == orc.MX_E4M3 else cols * 3 // 4
+    for i, s in enumerate(specs):
+        nrows = 4
+        r0 = int(rng.integers(0, s.rows - nrows)) if i % 7 else s.rows - nrows      # the last rows of some tensors
+        gpr = s.cols // s.group_cols
+        hat, _ = orc.sample_fwd(bits_of(W[i][r0:r0 + nrows]), BT[i][r0 * gpr:(r0 + nrows) * gpr].cpu().numpy(), nrows, s.cols, 1,
+                                s.group_cols, seed=descs[i].seed, step=step, elem_offset=r0 * s.cols)
+        codes, scales = orc.mx_emit(hat, nrows, s.cols, 1, s.group_cols, fmt_orc)
+        want_codes = codes if fmt_orc == orc.MX_E4M3 else orc.mx_pack6(codes)
+        codes_bytes, scales_off, _ = gws.mx_layout(descs[i], fmt_gpu)
+        cb = code_bytes_per_row(s.cols)
+        got_codes = MX[i][r0 * cb:(r0 + nrows) * cb].cpu().numpy()
+        got_scales = MX[i][scales_off + r0 * s.cols // 32:scales_off + (r0 + nrows) * s.cols // 32].cpu().numpy()
+        assert np.array_equal(got_codes, want_codes), (s.name, r0)
+        assert np.array_equal(got_scales, scales), (s.name, r0)
+
+
+def test_config3_cut_into_six_flat_shards_carries_the_bits_of_the_uncut_set():
+    # one rank's share of every tensor (6 does not divide them: every shard has a partial group at each end), the other
+    # ranks' partial results for those groups supplied from the uncut tensors; forward and backward of the rank
+    from paper_2505_11170_b200.sharding import ShardedSetSampler, plan_flat_shard
+    specs = syn.llama2_1b(n_blocks=4)
+    world, rank, step = 6, 2, 7
+    descs, W, BT, G, WH, SC, GBT = _device_set(specs)
+    full = gws.MultiPlan(descs, w=W, bt=BT, w_hat=WH, scale=SC, grad_w_hat=G, grad_bt=GBT)
+    full.sample_fwd_multi(step)
+    full.sample_bwd_multi(step)
+    plans = [plan_flat_shard(s.numel, s.group_cols, rank, world) for s in specs]
+    cut = lambda t, p: t.view(-1)[p.begin:p.end]
+    grp = lambda t, p: t[p.first_group:p.first_group + p.n_local_groups]
+    w_hat = [torch.full((p.n_elements,), float("nan"), dtype=torch.bfloat16, device=DEV) for p in plans]
+    sh = ShardedSetSampler(plans, [d.seed for d in descs], [cut(W[i], p) for i, p in enumerate(plans)],
+                           [grp(BT[i], p) for i, p in enumerate(plans)], w_hat, [cut(G[i], p) for i, p in enumerate(plans)])
+    assert sh.n_pieces == sum(len(p.pieces) for p in plans) >= len(specs) and sh.launches_per_forward <= 8
+    # forward: what the MAX all-reduce would deliver is the uncut tensor's factor of each shared group
+    buf = sh.forward_local(step)
+    reduced = buf.clone()
+    n_slots = world + 1
+    for t, p in enumerate(plans):
+        for piece in p.pieces:
+            reduced[t * n_slots + piece.read_slot] = SC[t][p.first_group + piece.local_group]
+    assert (reduced >= buf).all()                                  # a part's factor never exceeds the group's
+    sh.forward_finish(step, reduced)
+    # backward: the SUM all-reduce delivers the uncut group's gradient; this rank's share must not exceed it in magnitude
+    # by more than rounding, and what it keeps for whole groups must match outright
+    buf = sh.backward_local(step)
+    reduced = buf.clone()
+    for t, p in enumerate(plans):
+        for piece in p.pieces:
+            reduced[t * n_slots + piece.read_slot] = GBT[t][p.first_group + piece.local_group]
+    sh.backward_finish(reduced)
+    torch.cuda.synchronize()
+    for t, p in enumerate(plans):
+        assert torch.equal(w_hat[t].view(torch.int16), cut(WH[t], p).view(torch.int16)), specs[t].name
+        assert torch.equal(sh.scale[t].view(torch.int32), grp(SC[t], p).view(torch.int32)), specs[t].name
+        assert torch.equal(sh.grad_bt[t].view(torch.int32), grp(GBT[t], p).view(torch.int32)), specs[t].name
