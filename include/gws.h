@@ -72,7 +72,9 @@ typedef enum gws_status {
   GWS_ERR_WORKSPACE = -6, /* workspace NULL, misaligned (256 B) or too small                   */
   GWS_ERR_CUDA = -7,      /* a CUDA runtime call failed; see gws_last_cuda_error()             */
   GWS_ERR_LIMIT = -8,     /* size beyond a documented maximum                                  */
-  GWS_ERR_UNSUPPORTED = -9 /* the call needs a different build of the library                  */
+  GWS_ERR_UNSUPPORTED = -9 /* the call needs a different build of the library, or the tensor is
+                              outside what the call supports (MX output), or the plan was
+                              prepared for another kind of output                              */
 } gws_status;
 
 /* One tensor and its noise stream. */
@@ -196,6 +198,30 @@ int gws_mx_quantize(const gws_desc* desc, int format, const void* w_hat, void* m
  * gws_mx_quantize applied to the w_hat gws_sample_fwd would have written.  scale_out as there. */
 int gws_sample_fwd_mx(const gws_desc* desc, int format, const void* w, const float* bt, void* mx_out,
                       float* scale_out, void* stream);
+
+/* ---- sampling fused into the GEMM that consumes w_hat --------------------------------------------
+ * Section 3.5 ("Separate kernels") keeps the sampling kernels and the GEMM apart; this entry point is
+ * the variant the paper decided against, so that the decision can be measured on this GPU:
+ *     Y[m, n] = X[m, k] * W_hat[n, k]^T,   W_hat = Eq. 3 + BF16 cast of W, sampled tile by tile in the
+ * prologue of a tcgen05 / TMA GEMM (FP32 accumulation in tensor memory, Y rounded to BF16 once) and
+ * never written to global memory unless w_hat_out is given.  W_hat has the bits gws_sample_fwd gives.
+ *   wdesc           W: rows = n (a multiple of 128), cols = k (a multiple of 128), dense, groups 1 x 128
+ *   m               rows of X and Y, a multiple of rows_per_block
+ *   x               device, BF16 [m, k] row-major, 16-byte aligned, read only (through a TMA tensor map)
+ *   w, bt           as for gws_sample_fwd; w 32-byte aligned
+ *   y               device, BF16 [m, n] row-major, written
+ *   w_hat_out       device, BF16 [n, k] or NULL: the sampled weights (written by one block per tile)
+ *   scale_out       device, FP32 [n * k / 128] or NULL
+ *   status          device, one int or NULL: set to 1 if a block gave up waiting for a copy or for the
+ *                   tensor core (about a second); its part of Y is then not written.  Never set otherwise.
+ *   rows_per_block  128, 256 or 512: rows of X per thread block; every sampled tile of W is used for that
+ *                   many rows, so a larger value repeats less sampling work (512 takes all tensor memory
+ *                   and 161 KiB of shared memory of an SM).
+ * Other shapes: GWS_ERR_UNSUPPORTED.  gws_gemm_last_error() describes a GWS_ERR_CUDA of this call.
+ */
+int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y,
+                   void* w_hat_out, float* scale_out, int* status, int rows_per_block, void* stream);
+const char* gws_gemm_last_error(void);
 
 /* ---- many tensors per launch ---------------------------------------------------------------
  * One linear layer of a 1B-parameter model is a few microseconds of HBM time, so a training

@@ -10,7 +10,8 @@ CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libgws.so")
 SOURCES = [os.path.join(CSRC, "gws_api.cu")]
-HEADERS = [os.path.join(CSRC, "gws_kernels.cuh"), os.path.join(CSRC, "gws_math.cuh"), os.path.join(INCLUDE, "gws.h")]
+HEADERS = [os.path.join(CSRC, "gws_kernels.cuh"), os.path.join(CSRC, "gws_math.cuh"), os.path.join(CSRC, "gws_gemm.cuh"),
+           os.path.join(INCLUDE, "gws.h")]
 
 # -fmad=false: the add-then-cast path must round the multiply and the add separately.
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-fmad=false",

@@ -70,6 +70,8 @@ _SIGNATURES = {
     "gws_mx_quantize": (c_int, [POINTER(Desc), c_int, c_void_p, c_void_p, c_void_p]),
     "gws_sample_fwd_mx": (c_int, [POINTER(Desc), c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gws_sample_fwd_mx_multi": (c_int, [POINTER(_MultiPlan), c_int, c_uint64, c_void_p]),
+    "gws_gemm_fused": (c_int, [POINTER(Desc), c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
+    "gws_gemm_last_error": (c_char_p, []),
     "gws_workspace_bytes": (c_size_t, [c_int]),
     "gws_multi_prepare": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, c_void_p, c_size_t,
                                   POINTER(_MultiPlan), c_void_p]),
@@ -249,6 +251,23 @@ def sample_fwd_mx(desc: Desc, fmt: int, w: torch.Tensor, bt: torch.Tensor, mx_ou
         scale_out = torch.empty(n_groups(desc), dtype=torch.float32, device=w.device)
     _check(load_library().gws_sample_fwd_mx(ctypes.byref(desc), fmt, _ptr(w), _ptr(bt), _ptr(mx_out), _ptr(scale_out), _stream(stream)))
     return mx_out, scale_out
+
+
+def gemm_fused(wdesc: Desc, x: torch.Tensor, w: torch.Tensor, bt: torch.Tensor, y: Optional[torch.Tensor] = None,
+               w_hat_out: Optional[torch.Tensor] = None, scale_out: Optional[torch.Tensor] = None,
+               status: Optional[torch.Tensor] = None, rows_per_block: int = 512, stream=None) -> torch.Tensor:
+    """Y = X @ W_hat^T with W_hat sampled inside the GEMM (never stored unless ``w_hat_out`` is given).  Returns Y."""
+    _require_cuda(x, w, bt, y, w_hat_out, scale_out, status)
+    if x.dim() != 2 or x.shape[1] != wdesc.cols or not x.is_contiguous() or x.dtype != torch.bfloat16:
+        raise ValueError("gws: x must be a contiguous BF16 [m, k] tensor with k = cols of W")
+    if y is None:
+        y = torch.empty((x.shape[0], wdesc.rows), dtype=torch.bfloat16, device=x.device)
+    lib = load_library()
+    st = lib.gws_gemm_fused(ctypes.byref(wdesc), x.shape[0], _ptr(x), _ptr(w), _ptr(bt), _ptr(y), _ptr(w_hat_out), _ptr(scale_out),
+                            _ptr(status), rows_per_block, _stream(stream))
+    if st != OK:
+        raise GwsError(st, lib.gws_gemm_last_error().decode() if st == ERR_CUDA else "")
+    return y
 
 
 def sample_bwd(desc: Desc, grad_w_hat: torch.Tensor, scale: torch.Tensor, grad_w: Optional[torch.Tensor] = None,

@@ -1098,7 +1098,7 @@ const char* gws_status_string(int status) {
     case GWS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case GWS_ERR_CUDA: return "CUDA runtime error (see gws_last_cuda_error)";
     case GWS_ERR_LIMIT: return "size beyond a documented maximum";
-    case GWS_ERR_UNSUPPORTED: return "not available in this build of the library";
+    case GWS_ERR_UNSUPPORTED: return "not supported: by this build of the library, or for this shape or kind of output";
     default: return "unknown status";
   }
 }
@@ -1108,3 +1108,5 @@ const char* gws_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
 uint64_t gws_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"
+
+#include "gws_gemm.cuh"   // gws_gemm_fused: the tcgen05 GEMM with sampling in its prologue

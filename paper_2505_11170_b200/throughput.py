@@ -1,6 +1,6 @@
 """Throughput of the sampling pass on the other workload shapes of the paper (one JSON line each).
 
-    python -m paper_2505_11170_b200.throughput [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [--reps N] [--blocks B]
+    python -m paper_2505_11170_b200.throughput [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [--reps N] [--blocks B]
 
 gpt2         all GPT2-124M linear weights, one group per row (and the same set with groups of 128)
 gpt2_single  one GPT2-124M MLP weight, both orientations
@@ -8,6 +8,7 @@ stress       4096^2, 8192^2, 28672 x 8192 with groups of 32, 128 and whole rows
 square       Llama2-1B-shaped blocks with the paper's 32 x 32 groups (Eq. 3, b_l = 32)
 llama        the Llama2-1B-shaped set with groups of 128 (the benchmark's workload; --blocks limits it)
 mx           the same set with w_hat written as MX FP8 / FP6 instead of BF16
+gemm         sampling fused into a tcgen05 GEMM against sampling + library GEMM against the plain library GEMM
 
 Every timed pass is one multi-tensor launch set over the whole workload, timed with CUDA events on the launching
 stream after three warm-up passes; a 256 MiB buffer is written between passes so that no pass finds its inputs in L2.
@@ -81,6 +82,50 @@ def run(name: str, specs, reps: int, dev, mx_format=None) -> dict:
     return line
 
 
+def run_gemm(reps: int, dev) -> dict:
+    """Llama2-1B-shaped up-projection: X [8 x 2048 tokens, 2048] times w_hat^T (W 5632 x 2048, groups of 128, 6 bits):
+    sampling fused into the GEMM, against sampling followed by the library GEMM, against the library GEMM on W alone."""
+    m, n, k = 16384, 5632, 2048
+    spec = syn.TensorSpec("up", n, k, 1, 128)
+    w = syn.weights(spec, 0, device=dev)
+    bt = syn.bitwidths(spec, 0, fixed=6.0, device=dev)
+    x = torch.randn(m, k, generator=torch.Generator(device=dev).manual_seed(3 * 1000003), device=dev).to(torch.bfloat16)
+    d = Desc.make(n, k, 1, 128, seed=syn.layer_seed(0, 0))
+    y = torch.empty(m, n, dtype=torch.bfloat16, device=dev)
+    w_hat = torch.empty_like(w)
+    scale = torch.empty(spec.n_groups, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(fn):
+        total = 0.0
+        for i in range(3 + reps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn(i)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                total += a.elapsed_time(b)
+        return total / reps * 1e3
+
+    def unfused(i):
+        gws.sample_fwd(d.with_step(i), w, bt, w_hat, scale)
+        torch.matmul(x, w_hat.t(), out=y)
+
+    line = {"workload": "up-projection 16384 x 2048 by 5632 x 2048 (groups of 128, 6 bits)", "flops": 2.0 * m * n * k, "reps": reps,
+            "plain_gemm_us": timed(lambda i: torch.matmul(x, w.t(), out=y)), "sample_then_gemm_us": timed(unfused)}
+    for rpb in (128, 256, 512):
+        line[f"fused_{rpb}_rows_per_block_us"] = timed(lambda i: gws.gemm_fused(d.with_step(i), x, w, bt, y=y, status=status, rows_per_block=rpb))
+    line["status"] = int(status.item())
+    line["fused_TFLOP/s"] = line["flops"] / (line["fused_512_rows_per_block_us"] * 1e-6) / 1e12
+    line["overhead_unfused_pct"] = 100.0 * (line["sample_then_gemm_us"] / line["plain_gemm_us"] - 1.0)
+    line["overhead_fused_pct"] = 100.0 * (line["fused_512_rows_per_block_us"] / line["plain_gemm_us"] - 1.0)
+    print(json.dumps(line), flush=True)
+    return line
+
+
 def main(argv=None) -> None:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("which", nargs="*", default=["gpt2", "stress"])
@@ -107,6 +152,8 @@ def main(argv=None) -> None:
             run(f"llama2_1b blocks 0-{min(args.blocks, 4) - 1}, 32x32 groups", specs, args.reps, dev)
         elif w == "llama":
             run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev)
+        elif w == "gemm":
+            run_gemm(args.reps, dev)
         elif w == "mx":
             for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2):
                 run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev, mx_format=fmt)
