@@ -2,7 +2,7 @@
 // cast) tile by tile in the prologue of a tcgen05 GEMM, never written to global memory.  Section 3.5 of the paper keeps
 // sampling and GEMM apart; this is the variant it decided against, built to be measured.
 //
-// One thread block (128 threads) computes MT x 128 rows by 128 columns of Y.  Per step along K (128 elements = one
+// One thread block (512 threads) computes MT x 128 rows by 128 columns of Y.  Per step along K (128 elements = one
 // sampling group per row of W):
 //   * one thread starts the TMA loads of the X tiles (MT x 128 rows x 128 K, 128-byte swizzle) onto an mbarrier;
 //   * all threads sample the W tile (128 rows of W x 128 K; four lanes per row, exactly the arithmetic of the flat-group
@@ -23,7 +23,7 @@
 namespace {
 
 constexpr int kTileM = 128, kTileN = 128, kTileK = 128;
-constexpr int kGemmThreads = 128;
+constexpr int kGemmThreads = 512;   // one 64-byte chunk of the W tile per thread and step
 constexpr uint32_t kAtomBytes = 128u * 128u;        // 128 rows x 128 bytes (64 BF16 along K): one swizzle atom column
 constexpr uint32_t kTileBytes = 2u * kAtomBytes;    // 128 rows x 128 K
 constexpr long long kWaitCycles = 2000000000LL;     // about a second
@@ -147,10 +147,10 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
           tma_load_2d(smem_x + mt * kTileBytes + atom * kAtomBytes, &x_map, &bar_x, static_cast<int32_t>(kt * kTileK + atom * 64),
                       static_cast<int32_t>(m0 + mt * kTileM));
     }
-    // sample the W tile: four lanes per row (one 128-element group), 32 rows per pass
+    // sample the W tile: four lanes per row (one 128-element group)
 #pragma unroll 1
-    for (uint32_t pass = 0; pass < 4; ++pass) {
-      const uint32_t r = pass * 32u + (tid >> 2);
+    for (uint32_t pass = 0; pass < 512u / kGemmThreads; ++pass) {
+      const uint32_t r = pass * (kGemmThreads / 4u) + (tid >> 2);
       const uint32_t row = n0 + r;
       const uint32_t chunk = (row * a.k + kt * kTileK) / 32u + quarter;
       const gws::Chunk c = gws::load_chunk<true>(a.w, chunk, 4);
@@ -195,22 +195,22 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
   if (!failed) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     uint16_t* y = reinterpret_cast<uint16_t*>(a.y);
+    // a warp reads the quarter (warp % 4) of the 128 accumulator rows; the warps of a quarter share its column blocks
+    const uint32_t quarter_rows = (warp & 3u) * 32u;
 #pragma unroll 1
-    for (int mt = 0; mt < MT; ++mt) {
-      const uint64_t row = static_cast<uint64_t>(m0) + mt * kTileM + warp * 32u + lane;
-#pragma unroll 1
-      for (uint32_t cb = 0; cb < kTileN / 32; ++cb) {
-        uint32_t acc[32];
-        tmem_ld32(tmem_base + ((warp * 32u) << 16) + mt * kTileN + cb * 32u, acc);
-        uint4* out = reinterpret_cast<uint4*>(y + row * a.n + n0 + cb * 32u);
+    for (uint32_t idx = warp >> 2; idx < MT * (kTileN / 32); idx += kGemmThreads / 128) {
+      const uint32_t mt = idx / (kTileN / 32), cb = idx % (kTileN / 32);
+      const uint64_t row = static_cast<uint64_t>(m0) + mt * kTileM + quarter_rows + lane;
+      uint32_t acc[32];
+      tmem_ld32(tmem_base + (quarter_rows << 16) + mt * kTileN + cb * 32u, acc);
+      uint4* out = reinterpret_cast<uint4*>(y + row * a.n + n0 + cb * 32u);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint32_t p[4];
+      for (int q = 0; q < 4; ++q) {
+        uint32_t p[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            p[e] = gws::pack_bf16_rne(__uint_as_float(acc[8 * q + 2 * e]), __uint_as_float(acc[8 * q + 2 * e + 1]));
-          out[q] = make_uint4(p[0], p[1], p[2], p[3]);
-        }
+        for (int e = 0; e < 4; ++e)
+          p[e] = gws::pack_bf16_rne(__uint_as_float(acc[8 * q + 2 * e]), __uint_as_float(acc[8 * q + 2 * e + 1]));
+        out[q] = make_uint4(p[0], p[1], p[2], p[3]);
       }
     }
   } else if (tid == 0 && a.status != nullptr) {
