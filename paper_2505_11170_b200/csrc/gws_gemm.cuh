@@ -133,6 +133,12 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
   const uint32_t tmem_base = tmem_slot;
 
   const uint32_t quarter = tid & 3u;                    // which 32 elements of the 128-element group
+  static_assert(kGemmThreads == 512, "one chunk of the W tile per thread and step");
+  const uint32_t r = tid >> 2, row = n0 + r;
+  const uint32_t chunk0 = (row * a.k) / 32u + quarter;  // this thread's chunk of step 0; step kt: + 4 * kt
+  // the chunk and bit-width of the next step are fetched before the current step's arithmetic starts
+  gws::Chunk c_next = gws::load_chunk<true>(a.w, chunk0, 4);
+  float bt_next = gws::ld_f32(a.bt, row * k_tiles);
   for (uint32_t kt = 0; kt < k_tiles; ++kt) {
     // the tensor core must have finished reading the previous step's tiles before they are overwritten
     if (kt > 0 && !mbar_wait(&bar_mma, (kt - 1u) & 1u)) failed = 1;
@@ -148,17 +154,19 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
                       static_cast<int32_t>(m0 + mt * kTileM));
     }
     // sample the W tile: four lanes per row (one 128-element group)
-#pragma unroll 1
-    for (uint32_t pass = 0; pass < 512u / kGemmThreads; ++pass) {
-      const uint32_t r = pass * (kGemmThreads / 4u) + (tid >> 2);
-      const uint32_t row = n0 + r;
-      const uint32_t chunk = (row * a.k + kt * kTileK) / 32u + quarter;
-      const gws::Chunk c = gws::load_chunk<true>(a.w, chunk, 4);
+    {
+      const uint32_t chunk = chunk0 + 4u * kt;
+      const gws::Chunk c = c_next;
+      const float bits = bt_next;
+      if (kt + 1u < k_tiles) {
+        c_next = gws::load_chunk<true>(a.w, chunk + 4u, 4);
+        bt_next = gws::ld_f32(a.bt, row * k_tiles + kt + 1u);
+      }
       uint32_t m = gws::absmax_chunk(c.x);
       m = gws::maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
       m = gws::maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
       const uint32_t g = row * k_tiles + kt;
-      const gws::Scale sc = gws::make_scale(__fmul_rn(gws::absmax_finish(m), gws::pow2_one_minus(gws::ld_f32(a.bt, g))));
+      const gws::Scale sc = gws::make_scale(__fmul_rn(gws::absmax_finish(m), gws::pow2_one_minus(bits)));
       gws::Chunk y;
       gws::sample_chunk(c.x, a.vec_lo + chunk * 4u, a.k0, a.k1, a.pre, sc, y.x);
       uint8_t* dst = smem_w + (quarter >> 1) * kAtomBytes + (r >> 3) * 1024u + (r & 7u) * 128u;
