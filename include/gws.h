@@ -222,6 +222,9 @@ int gws_sample_fwd_mx(const gws_desc* desc, int format, const void* w, const flo
 int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y,
                    void* w_hat_out, float* scale_out, int* status, int rows_per_block, void* stream);
 const char* gws_gemm_last_error(void);
+/* Diagnostic: runs the fused GEMM's bounded wait on an mbarrier that nothing completes (one thread, about a
+ * second).  status2: device, two ints, written: [0] = 1 (the wait gave up, as it must), [1] = SM cycles waited / 1024. */
+int gws_gemm_wait_probe(int* status2, void* stream);
 
 /* ---- many tensors per launch ---------------------------------------------------------------
  * One linear layer of a 1B-parameter model is a few microseconds of HBM time, so a training

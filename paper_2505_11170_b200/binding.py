@@ -72,6 +72,7 @@ _SIGNATURES = {
     "gws_sample_fwd_mx_multi": (c_int, [POINTER(_MultiPlan), c_int, c_uint64, c_void_p]),
     "gws_gemm_fused": (c_int, [POINTER(Desc), c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
     "gws_gemm_last_error": (c_char_p, []),
+    "gws_gemm_wait_probe": (c_int, [c_void_p, c_void_p]),
     "gws_workspace_bytes": (c_size_t, [c_int]),
     "gws_multi_prepare": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_void_p, c_size_t, c_void_p, c_size_t,
                                   POINTER(_MultiPlan), c_void_p]),

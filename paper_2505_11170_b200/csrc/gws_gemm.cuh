@@ -229,6 +229,20 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
 }
 
+// The bounded wait on its own: one thread waits on an mbarrier that nothing will ever complete, gives up after
+// kWaitCycles and reports it the way the GEMM does.  status[0] = 1: gave up; status[1] = SM cycles waited / 1024.
+__global__ void k_wait_probe(int* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const long long t0 = clock64();
+    const bool completed = mbar_wait(&bar, 0);
+    status[0] = completed ? 0 : 1;
+    status[1] = static_cast<int>(((clock64() - t0) >> 10) & 0x7FFFFFFF);
+  }
+}
+
 using EncodeTiled = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
@@ -251,6 +265,15 @@ int launch_gemm(const CUtensorMap& map, const GemmArgs& args, int64_t m, cudaStr
 extern "C" {
 
 const char* gws_gemm_last_error(void) { return g_gemm_error.c_str(); }
+
+int gws_gemm_wait_probe(int* status2, void* stream) {
+  if (status2 == nullptr) return GWS_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(status2) % 4) != 0) return GWS_ERR_ALIGN;
+  k_wait_probe<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status2);
+  const cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) { g_gemm_error = std::string("wait probe launch: ") + cudaGetErrorString(err); return GWS_ERR_CUDA; }
+  return GWS_OK;
+}
 
 int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y, void* w_hat_out,
                    float* scale_out, int* status, int rows_per_block, void* stream) {

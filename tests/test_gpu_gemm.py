@@ -103,3 +103,19 @@ def test_fused_gemm_refuses_other_shapes_before_any_launch():
     assert call(Desc.make(128, 128, 1, 128), 128, 128, w=p + (1 << 19) + 16) == binding.ERR_ALIGN
     assert call(Desc.make(128, 128, 1, 128), 0, 128) == binding.OK                         # nothing to do
     assert lib.gws_gemm_fused(ctypes.byref(Desc.make(128, 128, 1, 128)), 128, None, p, fp, p, None, None, None, 128, None) == binding.ERR_NULL
+
+
+def test_a_wait_that_nothing_completes_gives_up_and_reports_it():
+    # the GEMM's waits (on the copy of X, on the tensor core) are bounded: the same wait on a barrier that no one
+    # will ever complete must return after about a second with the failure recorded, the context still usable
+    lib = gws.load_library()
+    status = torch.full((2,), -1, dtype=torch.int32, device=DEV)
+    assert lib.gws_gemm_wait_probe(status.data_ptr(), None) == binding.OK
+    torch.cuda.synchronize()
+    gave_up, cycles = status.cpu().tolist()
+    assert gave_up == 1
+    assert cycles >= 2_000_000_000 // 1024                          # it waited its whole limit first (cycles / 1024)
+    y = gws.gemm_fused(Desc.make(128, 128, 1, 128), torch.zeros(128, 128, dtype=torch.bfloat16, device=DEV),
+                       torch.zeros(128, 128, dtype=torch.bfloat16, device=DEV), torch.full((128,), 4.0, device=DEV), rows_per_block=128)
+    torch.cuda.synchronize()
+    assert (y == 0).all()                                           # the device still works
