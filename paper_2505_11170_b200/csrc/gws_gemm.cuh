@@ -139,6 +139,8 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
   // the chunk and bit-width of the next step are fetched before the current step's arithmetic starts
   gws::Chunk c_next = gws::load_chunk<true>(a.w, chunk0, 4);
   float bt_next = gws::ld_f32(a.bt, row * k_tiles);
+  bool copy_pending = false;       // thread 0: a copy of X has been started and not yet seen to land
+  uint32_t copy_parity = 0;
   for (uint32_t kt = 0; kt < k_tiles; ++kt) {
     // the tensor core must have finished reading the previous step's tiles before they are overwritten
     if (kt > 0 && !mbar_wait(&bar_mma, (kt - 1u) & 1u)) failed = 1;
@@ -152,6 +154,8 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
         for (int atom = 0; atom < 2; ++atom)
           tma_load_2d(smem_x + mt * kTileBytes + atom * kAtomBytes, &x_map, &bar_x, static_cast<int32_t>(kt * kTileK + atom * 64),
                       static_cast<int32_t>(m0 + mt * kTileM));
+      copy_pending = true;
+      copy_parity = kt & 1u;
     }
     // sample the W tile: four lanes per row (one 128-element group)
     {
@@ -185,6 +189,7 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
       if (!mbar_wait(&bar_x, kt & 1u)) {
         failed = 1;
       } else {
+        copy_pending = false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
@@ -221,8 +226,10 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_consta
         out[q] = make_uint4(p[0], p[1], p[2], p[3]);
       }
     }
-  } else if (tid == 0 && a.status != nullptr) {
-    atomicExch(a.status, 1);
+  } else if (tid == 0) {
+    if (a.status != nullptr) atomicExch(a.status, 1);
+    // a copy that may still be in flight gets one more bounded wait before the shared memory is given up
+    if (copy_pending) (void)mbar_wait(&bar_x, copy_parity);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
