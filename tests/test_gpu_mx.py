@@ -140,3 +140,20 @@ def test_unsupported_shapes_are_refused_before_any_launch():
     assert gws.mx_layout(Desc.make(64, 96), 0) == (6144, 6144, 6144 + 192)
     assert gws.mx_layout(Desc.make(64, 96), 1) == (4608, 4608, 4608 + 192)
     assert gws.mx_layout(Desc.make(2, 32), 1) == (48, 256, 258)
+
+
+def test_nan_and_inf_never_fault():
+    # unspecified values, but the call must complete and leave the device usable
+    w = _weights(64, 256, 3)
+    w.view(-1)[5] = float("nan")
+    w.view(-1)[300] = float("inf")
+    w.view(-1)[9000] = float("-inf")
+    d = Desc.make(64, 256, 1, 128, seed=1, step=1)
+    bt = torch.full((gws.n_groups(d),), 5.0, device=DEV)
+    for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2):
+        gws.sample_fwd_mx(d, fmt, w.to(DEV), bt)
+        gws.mx_quantize(d, fmt, w.to(DEV))
+    gws.sample_fwd_scaled(d, w.to(DEV), torch.full((gws.n_groups(d),), float("nan"), device=DEV))
+    torch.cuda.synchronize()
+    ok, _ = gws.sample_fwd(d, _weights(64, 256, 4).to(DEV), bt)
+    assert not torch.isnan(ok.float()).any()
