@@ -308,9 +308,9 @@ def main():
         hSC = [torch.empty_like(x).pin_memory() for x in hBT]
         hGBT = [torch.empty_like(x).pin_memory() for x in hBT]
 
-        # Tensors go round-robin over three streams, so the upload of one overlaps the download of another (the two
-        # copy directions use different engines).  Tensors that share pinned buffers share a stream, which orders them.
-        side = [torch.cuda.Stream(device=dev) for _ in range(3)]
+        # One stream per set of pinned buffers: the upload of one tensor overlaps the download of another (the two copy
+        # directions use different engines), and tensors that share pinned buffers share a stream, which orders them.
+        side = [torch.cuda.Stream(device=dev) for _ in range(len(block))]
 
         def host_step(k):
             for st in side:
@@ -336,7 +336,7 @@ def main():
         e2e = {"value": whole_job_throughput(bytes_per_step, world, e2e_ms) / 1e9, "unit": "GB/s",
                "h2d_bytes_per_step": int(n_elem * 4 + n_groups * 4), "d2h_bytes_per_step": int(n_elem * 2 + n_groups * 8),
                "ms_per_step": float(e2e_ms), "steps": e2e_steps,
-               "note": "gws_sample_step_host per tensor on three streams; pinned host buffers of one transformer block reused "
+               "note": "gws_sample_step_host per tensor on seven streams; pinned host buffers of one transformer block reused "
                        "for all 22; bound by the host link (6.9 GB cross it per step)"}
 
     # ---- side measurements (one GPU only; not part of `value`) ----
