@@ -144,7 +144,6 @@ class ShardedSampler:
         self.plan = plan
         self.seed = seed
         self.process_group = process_group
-        self._partial: Optional[torch.Tensor] = None
 
     # -- descriptors -------------------------------------------------------------------------------------------
     def _body_desc(self, step: int) -> Desc:
