@@ -375,7 +375,10 @@ void gwso_sample_bwd(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows,
 //     is kept.
 // Element formats: E4M3 = 1 sign, 4 exponent (bias 7), 3 mantissa bits, largest normal 448 = 1.75 * 2^8
 // (emax 8; the code S.1111.111 is NaN and never produced from finite input); E3M2 = 1 sign, 3 exponent
-// (bias 3), 2 mantissa bits, largest normal 28 = 1.75 * 2^4 (emax 4), no NaN or infinity.
+// (bias 3), 2 mantissa bits, largest normal 28 = 1.75 * 2^4 (emax 4), no NaN or infinity.  Format 2 is
+// Table C.1's FP8_e3m4, which the paper names without defining and which is not an OCP element type; it is
+// read by analogy with E3M2: 1 sign, 3 exponent (bias 3), 4 mantissa bits, every code finite, largest
+// normal 31 = 1.9375 * 2^4 (emax 4).
 
 struct MxElement {
   int exponent_bits, mantissa_bits, bias, emax;
@@ -384,6 +387,7 @@ struct MxElement {
 
 static MxElement mx_element(int format) {
   if (format == 0) return MxElement{4, 3, 7, 8, 448.0};
+  if (format == 2) return MxElement{3, 4, 3, 4, 31.0};
   return MxElement{3, 2, 3, 4, 28.0};
 }
 

@@ -275,7 +275,7 @@ def layer_seed(user_seed: int, layer: int) -> int:
 
 # ---- w_hat in an MX floating-point format (Section 3.1, Table C.1) ---------------------------------------
 
-MX_E4M3, MX_E3M2 = 0, 1
+MX_E4M3, MX_E3M2, MX_E3M4 = 0, 1, 2
 
 
 def mx_decode(fmt: int, code: int) -> float:

@@ -10,9 +10,10 @@ import torch
 from oracle import gws_oracle as orc
 from util import bits_of, f32_of_bits
 
-E4M3, E3M2 = orc.MX_E4M3, orc.MX_E3M2
+E4M3, E3M2, E3M4 = orc.MX_E4M3, orc.MX_E3M2, orc.MX_E3M4
 FORMATS = {E4M3: dict(width=8, mbits=3, bias=7, emax=8, max=448.0, finite=[c for c in range(256) if c & 0x7F != 0x7F]),
-           E3M2: dict(width=6, mbits=2, bias=3, emax=4, max=28.0, finite=list(range(64)))}
+           E3M2: dict(width=6, mbits=2, bias=3, emax=4, max=28.0, finite=list(range(64))),
+           E3M4: dict(width=8, mbits=4, bias=3, emax=4, max=31.0, finite=list(range(256)))}
 
 
 def test_element_grids_match_their_definition():
@@ -21,6 +22,8 @@ def test_element_grids_match_their_definition():
     assert orc.mx_decode(E4M3, 0xFE) == -448.0 and math.isnan(orc.mx_decode(E4M3, 0x7F))
     assert orc.mx_decode(E3M2, 0x1F) == 28.0 and orc.mx_decode(E3M2, 0x0C) == 1.0
     assert orc.mx_decode(E3M2, 0x04) == 0.25 and orc.mx_decode(E3M2, 0x01) == 0.0625 and orc.mx_decode(E3M2, 0x3F) == -28.0
+    assert orc.mx_decode(E3M4, 0x7F) == 31.0 and orc.mx_decode(E3M4, 0x30) == 1.0 and orc.mx_decode(E3M4, 0x10) == 0.25
+    assert orc.mx_decode(E3M4, 0x01) == 2.0 ** -6 and orc.mx_decode(E3M4, 0xFF) == -31.0
     for fmt, f in FORMATS.items():
         half = 1 << (f["width"] - 1)
         pos = [orc.mx_decode(fmt, c) for c in f["finite"] if c < half]
@@ -43,7 +46,7 @@ def _nearest_even_code(fmt, x):
     return best | (half if math.copysign(1.0, x) < 0 else 0)
 
 
-@pytest.mark.parametrize("fmt", [E4M3, E3M2])
+@pytest.mark.parametrize("fmt", [E4M3, E3M2, E3M4])
 def test_rounding_is_nearest_even_with_clamping(fmt):
     f = FORMATS[fmt]
     half = 1 << (f["width"] - 1)
@@ -74,7 +77,7 @@ def _w_hat(rows, cols, seed, sigma=0.02):
     return bits_of(t.to(torch.bfloat16))
 
 
-@pytest.mark.parametrize("fmt", [E4M3, E3M2])
+@pytest.mark.parametrize("fmt", [E4M3, E3M2, E3M4])
 @pytest.mark.parametrize("rows,cols,gr,gc", [(4, 128, 1, 32), (3, 256, 1, 128), (5, 96, 1, 0), (64, 64, 32, 32)])
 def test_emission_properties(fmt, rows, cols, gr, gc):
     f = FORMATS[fmt]
@@ -114,7 +117,7 @@ def test_square_blocks_commute_with_transposition():
     n = 96
     w = _w_hat(n, n, 5)
     wt = np.ascontiguousarray(w.reshape(n, n).T).ravel()
-    for fmt in (E4M3, E3M2):
+    for fmt in (E4M3, E3M2, E3M4):
         c, s = orc.mx_emit(w, n, n, 32, 32, fmt)
         ct, st = orc.mx_emit(wt, n, n, 32, 32, fmt)
         assert np.array_equal(c.reshape(n, n).T, ct.reshape(n, n))
