@@ -176,7 +176,10 @@ int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scal
  *                      (subnormals included), clamped to the largest normal (448 / 28); the
  *                      sign of zero is kept
  * Buffer layout (one device allocation per tensor, 32-byte aligned, see gws_mx_layout):
- *   [0, codes_bytes)            element codes in logical row-major order.  E4M3: one byte each.
+ * GWS_MX_FP8_E3M4 is Table C.1's FP8_e3m4, which the paper names without defining and which is not
+ * an OCP element type: it is read by analogy with E3M2 (bias 3, every code finite, largest normal 31,
+ * emax 4) and converted in integer arithmetic (the GPU has no instruction for it).
+ *   [0, codes_bytes)            element codes in logical row-major order.  E4M3 / E3M4: one byte each.
  *                               E3M2: a little-endian bit stream, element k at bits [6k, 6k+5]
  *                               (4 elements in 3 bytes, a 32-element vector in 24).
  *   [scales_offset, total)      one scale byte per 32 elements, [rows, cols/32] row-major;
@@ -186,7 +189,7 @@ int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scal
  * groups of 1 x {32, 64, 128, 256}, whole rows up to 32768 elements, or 32 x 32 blocks with rows
  * a multiple of 32.
  */
-typedef enum gws_mx_format { GWS_MX_FP8_E4M3 = 0, GWS_MX_FP6_E3M2 = 1 } gws_mx_format;
+typedef enum gws_mx_format { GWS_MX_FP8_E4M3 = 0, GWS_MX_FP6_E3M2 = 1, GWS_MX_FP8_E3M4 = 2 } gws_mx_format;
 
 /* Sizes of the MX buffer of a tensor; any of the three outputs may be NULL.  Host arithmetic only. */
 int gws_mx_layout(const gws_desc* desc, int format, size_t* codes_bytes, size_t* scales_offset, size_t* total_bytes);

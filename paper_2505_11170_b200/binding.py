@@ -216,7 +216,7 @@ def sample_fwd_scaled(desc: Desc, w: torch.Tensor, scale: torch.Tensor, w_hat: O
     return w_hat
 
 
-MX_FP8_E4M3, MX_FP6_E3M2 = 0, 1
+MX_FP8_E4M3, MX_FP6_E3M2, MX_FP8_E3M4 = 0, 1, 2
 
 
 def mx_layout(desc: Desc, fmt: int):

@@ -133,7 +133,7 @@ Entry make_entry(const gws_desc* d, int cls, const void* in, void* out, const fl
 // Element codes first (E4M3: one byte per element; E3M2: 6 bits per element), then, from the next multiple of
 // 256 bytes, one E8M0 scale byte per 32 elements.
 size_t mx_codes_bytes(int64_t n_elements, int format) {
-  return format == gws::kMxE4M3 ? static_cast<size_t>(n_elements) : static_cast<size_t>(n_elements) / 4u * 3u;
+  return format == gws::kMxE3M2 ? static_cast<size_t>(n_elements) / 4u * 3u : static_cast<size_t>(n_elements);
 }
 size_t mx_scales_offset(int64_t n_elements, int format) { return (mx_codes_bytes(n_elements, format) + 255u) & ~static_cast<size_t>(255u); }
 size_t mx_total_bytes(int64_t n_elements, int format) { return mx_scales_offset(n_elements, format) + static_cast<size_t>(n_elements) / 32u; }
@@ -521,7 +521,7 @@ int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scal
 int gws_mx_layout(const gws_desc* desc, int format, size_t* codes_bytes, size_t* scales_offset, size_t* total_bytes) {
   const int st = validate_desc(desc);
   if (st != GWS_OK) return st;
-  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2) return GWS_ERR_UNSUPPORTED;
+  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2 && format != GWS_MX_FP8_E3M4) return GWS_ERR_UNSUPPORTED;
   if (desc->cols % 32 != 0) return GWS_ERR_UNSUPPORTED;
   const int64_t n = desc->rows * desc->cols;
   if (codes_bytes) *codes_bytes = mx_codes_bytes(n, format);
@@ -533,7 +533,7 @@ int gws_mx_layout(const gws_desc* desc, int format, size_t* codes_bytes, size_t*
 int gws_mx_quantize(const gws_desc* desc, int format, const void* w_hat, void* mx_out, void* stream) {
   const int st = precheck(desc);
   if (st != GWS_OK) return st < 0 ? st : GWS_OK;
-  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2) return GWS_ERR_UNSUPPORTED;
+  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2 && format != GWS_MX_FP8_E3M4) return GWS_ERR_UNSUPPORTED;
   if (w_hat == nullptr || mx_out == nullptr) return GWS_ERR_NULL;
   if (!aligned(w_hat, 2)) return GWS_ERR_ALIGN;
   if (desc->cols % 32 != 0) return GWS_ERR_UNSUPPORTED;
@@ -542,15 +542,16 @@ int gws_mx_quantize(const gws_desc* desc, int format, const void* w_hat, void* m
   const Entry e = make_entry(desc, cls, w_hat, mx_out, nullptr, nullptr);
   if (!mx_entry_ok(cls, e)) return GWS_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  return format == GWS_MX_FP8_E4M3 ? launch_mx<gws::kQuantMx8>(cls, &e, 1, desc->step, s)
-                                   : launch_mx<gws::kQuantMx6>(cls, &e, 1, desc->step, s);
+  if (format == GWS_MX_FP8_E4M3) return launch_mx<gws::kQuantMx8>(cls, &e, 1, desc->step, s);
+  if (format == GWS_MX_FP8_E3M4) return launch_mx<gws::kQuantMx8b>(cls, &e, 1, desc->step, s);
+  return launch_mx<gws::kQuantMx6>(cls, &e, 1, desc->step, s);
 }
 
 int gws_sample_fwd_mx(const gws_desc* desc, int format, const void* w, const float* bt, void* mx_out, float* scale_out,
                       void* stream) {
   const int st = precheck(desc);
   if (st != GWS_OK) return st < 0 ? st : GWS_OK;
-  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2) return GWS_ERR_UNSUPPORTED;
+  if (format != GWS_MX_FP8_E4M3 && format != GWS_MX_FP6_E3M2 && format != GWS_MX_FP8_E3M4) return GWS_ERR_UNSUPPORTED;
   if (w == nullptr || bt == nullptr || mx_out == nullptr) return GWS_ERR_NULL;
   if (!aligned(w, 2) || !aligned(bt, 4) || !aligned(scale_out, 4)) return GWS_ERR_ALIGN;
   if (desc->cols % 32 != 0) return GWS_ERR_UNSUPPORTED;
@@ -559,8 +560,9 @@ int gws_sample_fwd_mx(const gws_desc* desc, int format, const void* w, const flo
   const Entry e = make_entry(desc, cls, w, mx_out, bt, scale_out);
   if (!mx_entry_ok(cls, e)) return GWS_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  return format == GWS_MX_FP8_E4M3 ? launch_mx<gws::kFwdMx8>(cls, &e, 1, desc->step, s)
-                                   : launch_mx<gws::kFwdMx6>(cls, &e, 1, desc->step, s);
+  if (format == GWS_MX_FP8_E4M3) return launch_mx<gws::kFwdMx8>(cls, &e, 1, desc->step, s);
+  if (format == GWS_MX_FP8_E3M4) return launch_mx<gws::kFwdMx8b>(cls, &e, 1, desc->step, s);
+  return launch_mx<gws::kFwdMx6>(cls, &e, 1, desc->step, s);
 }
 
 int gws_sample_bwd(const gws_desc* desc, const void* grad_w_hat, const float* scale, void* grad_w, float* grad_bt,
@@ -646,7 +648,7 @@ static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs
   if (has_bwd && (ptrs->scale == nullptr || ptrs->grad_bt == nullptr)) return GWS_ERR_NULL;
   if (workspace == nullptr || !aligned(workspace, 256) || workspace_bytes < gws_workspace_bytes(n)) return GWS_ERR_WORKSPACE;
   const int kind = ptrs->w_hat_kind;
-  if (kind != 0 && kind != 1 + GWS_MX_FP8_E4M3 && kind != 1 + GWS_MX_FP6_E3M2) return GWS_ERR_UNSUPPORTED;
+  if (kind < 0 || kind > 1 + GWS_MX_FP8_E3M4) return GWS_ERR_UNSUPPORTED;
   if (kind != 0 && !has_fwd) return GWS_ERR_NULL;
 
   ClassTables t;
@@ -840,6 +842,7 @@ extern "C" {
 int gws_sample_fwd_mx_multi(const gws_multi_plan* plan, int format, uint64_t step, void* stream) {
   if (format == GWS_MX_FP8_E4M3) return run_multi_mx<gws::kFwdMx8>(plan, step, stream);
   if (format == GWS_MX_FP6_E3M2) return run_multi_mx<gws::kFwdMx6>(plan, step, stream);
+  if (format == GWS_MX_FP8_E3M4) return run_multi_mx<gws::kFwdMx8b>(plan, step, stream);
   return GWS_ERR_UNSUPPORTED;
 }
 

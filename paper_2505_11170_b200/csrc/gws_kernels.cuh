@@ -37,14 +37,16 @@ namespace gws {
 
 // kFwdScaled: forward with the per-group factor s_g supplied (in `gin`) instead of derived from this tensor's own
 // maxima: the add and cast of Eq. 3 for a tensor whose groups reach into memory this call does not see.
-enum Mode { kAbsmax = 0, kFwd = 1, kBwd = 2, kFwdScaled = 3, kFwdMx8 = 4, kFwdMx6 = 5, kQuantMx8 = 6, kQuantMx6 = 7 };
+enum Mode { kAbsmax = 0, kFwd = 1, kBwd = 2, kFwdScaled = 3, kFwdMx8 = 4, kFwdMx6 = 5, kQuantMx8 = 6, kQuantMx6 = 7, kFwdMx8b = 8, kQuantMx8b = 9 };
 // kFwdMx*: the forward pass with w_hat written as MX floating point (E4M3 or E3M2 elements, one E8M0 scale per 32
 // elements) instead of BF16; kQuantMx*: that conversion alone, from a BF16 w_hat in `in`.
-enum MxFormat { kMxE4M3 = 0, kMxE3M2 = 1 };
-__host__ __device__ constexpr bool mode_is_mx_fwd(int m) { return m == kFwdMx8 || m == kFwdMx6; }
-__host__ __device__ constexpr bool mode_is_mx_quant(int m) { return m == kQuantMx8 || m == kQuantMx6; }
+enum MxFormat { kMxE4M3 = 0, kMxE3M2 = 1, kMxE3M4 = 2 };   // Mx8 = E4M3, Mx6 = E3M2, Mx8b = E3M4
+__host__ __device__ constexpr bool mode_is_mx_fwd(int m) { return m == kFwdMx8 || m == kFwdMx6 || m == kFwdMx8b; }
+__host__ __device__ constexpr bool mode_is_mx_quant(int m) { return m == kQuantMx8 || m == kQuantMx6 || m == kQuantMx8b; }
 __host__ __device__ constexpr bool mode_is_fwd(int m) { return m == kFwd || mode_is_mx_fwd(m); }            // takes maxima of w, writes scale_out
-__host__ __device__ constexpr int mode_mx_format(int m) { return (m == kFwdMx8 || m == kQuantMx8) ? kMxE4M3 : kMxE3M2; }
+__host__ __device__ constexpr int mode_mx_format(int m) {
+  return (m == kFwdMx8 || m == kQuantMx8) ? kMxE4M3 : ((m == kFwdMx8b || m == kQuantMx8b) ? kMxE3M4 : kMxE3M2);
+}
 __host__ __device__ constexpr bool mode_reads_group_input(int m) { return m != kAbsmax && !mode_is_mx_quant(m); }
 enum KernelClass { kFlat = 0, kRowWarp = 1, kRowCta = 2, kGeneral = 3 };
 
@@ -324,8 +326,26 @@ __device__ __forceinline__ float grad_bt_of(float scale, float sum_g_2r) {
 // cvt.rn.satfinite does.  The multiplication by a power of two is exact.
 // Buffer: element codes from byte 0 in chunk order (E4M3: 32 bytes per 32-element chunk; E3M2: 24, code k of the
 // chunk at bits [6k, 6k+5] of a little-endian bit stream), scale bytes from byte 16 * scales_off16, one per chunk.
+// E3M4 (1-3-4, bias 3, every code finite, largest normal 31) has no conversion instruction: round to nearest even in
+// integer arithmetic.  Below the smallest normal (2^-2) the codes are multiples of 2^-6: adding 2^17 makes the FP32
+// adder round to that spacing.  From there up the mantissa is cut at bit 19 with the usual round-to-even increment,
+// a carry moves into the exponent, and anything beyond the last code is clamped to it.
+__device__ __forceinline__ uint32_t cvt_e3m4(float x) {
+  const uint32_t bits = __float_as_uint(x), sign = (bits >> 24) & 0x80u;
+  const float a = fabsf(x);
+  uint32_t mag;
+  if (a < 0.25f) {
+    mag = __float_as_uint(__fadd_rn(a, 0x1p17f)) - __float_as_uint(0x1p17f);
+  } else {
+    uint32_t ab = bits & 0x7FFFFFFFu;
+    ab += 0x3FFFFu + ((ab >> 19) & 1u);
+    mag = min((ab >> 19) - ((127u - 3u) << 4), 0x7Fu);
+  }
+  return sign | mag;
+}
 template <int FMT>
 __device__ __forceinline__ uint32_t cvt_mx_x2(float upper, float lower) {
+  if (FMT == kMxE3M4) return (cvt_e3m4(upper) << 8) | cvt_e3m4(lower);
   uint16_t d;
   if (FMT == kMxE4M3) asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(upper), "f"(lower));
   else asm("cvt.rn.satfinite.e3m2x2.f32 %0, %1, %2;" : "=h"(d) : "f"(upper), "f"(lower));
@@ -334,12 +354,12 @@ __device__ __forceinline__ uint32_t cvt_mx_x2(float upper, float lower) {
 // Scale byte of a group whose largest |w_hat| is `amax`, and the bits of the multiplier 2^(127 - byte).
 template <int FMT>
 __device__ __forceinline__ uint32_t mx_scale_byte(float amax) {
-  constexpr int kEmax = FMT == kMxE4M3 ? 8 : 4;
+  constexpr int kEmax = FMT == kMxE4M3 ? 8 : 4;   // E3M2 and E3M4: 4
   return static_cast<uint32_t>(max(static_cast<int>(__float_as_uint(amax) >> 23) - kEmax, 0));   // amax >= 0: no sign bit
 }
 __device__ __forceinline__ uint32_t mx_mult_bits(uint32_t byte) { return (254u - byte) << 23; }
 
-// Codes of 16 elements (8 packed BF16 pairs): E4M3 -> 4 words, E3M2 -> 3 words (four 6-bit codes per 3 bytes).
+// Codes of 16 elements (8 packed BF16 pairs): E4M3 / E3M4 -> 4 words, E3M2 -> 3 words (four 6-bit codes per 3 bytes).
 template <int FMT>
 __device__ __forceinline__ void mx_encode_half(const uint32_t* y, uint32_t mult_bits, uint32_t* out) {
   const float mult = __uint_as_float(mult_bits);
@@ -350,7 +370,7 @@ __device__ __forceinline__ void mx_encode_half(const uint32_t* y, uint32_t mult_
     const float hi = fma_bf16(hi16(y[j]), hi16(mult_bits), -0.0f);         // + (-0): keeps the sign of a zero product
     q[j] = cvt_mx_x2<FMT>(hi, lo);
   }
-  if (FMT == kMxE4M3) {
+  if (FMT != kMxE3M2) {   // one byte per code
 #pragma unroll
     for (int k = 0; k < 4; ++k) out[k] = q[2 * k] | (q[2 * k + 1] << 16);
   } else {
@@ -369,7 +389,7 @@ __device__ __forceinline__ void mx_encode_half(const uint32_t* y, uint32_t mult_
 template <int FMT>
 __device__ __forceinline__ void mx_write(void* out, uint32_t scales_off16, uint32_t chunk, const uint32_t* y, float amax) {
   const uint32_t byte = mx_scale_byte<FMT>(amax), mult_bits = mx_mult_bits(byte);
-  if (FMT == kMxE4M3) {
+  if (FMT != kMxE3M2) {
     uint32_t w[8];
     mx_encode_half<FMT>(y, mult_bits, w);
     mx_encode_half<FMT>(y + 8, mult_bits, w + 4);
@@ -389,7 +409,7 @@ __device__ __forceinline__ void mx_write(void* out, uint32_t scales_off16, uint3
 template <int FMT>
 __device__ __forceinline__ void mx_write_half(void* out, uint32_t scales_off16, uint32_t chunk, uint32_t h, const uint32_t* y, float amax) {
   const uint32_t byte = mx_scale_byte<FMT>(amax), mult_bits = mx_mult_bits(byte);
-  if (FMT == kMxE4M3) {
+  if (FMT != kMxE3M2) {
     uint32_t w[4];
     mx_encode_half<FMT>(y, mult_bits, w);
     st_vec(out, static_cast<uint64_t>(chunk) * 2u + h, make_uint4(w[0], w[1], w[2], w[3]));

@@ -49,7 +49,7 @@ def run(name: str, specs, reps: int, dev, mx_format=None) -> dict:
         out_bytes = 2.0
     else:
         WH = [torch.empty(gws.mx_layout(d, mx_format)[2], dtype=torch.uint8, device=dev) for d in descs]
-        out_bytes = (1.0 if mx_format == gws.MX_FP8_E4M3 else 0.75) + 1.0 / 32.0
+        out_bytes = (0.75 if mx_format == gws.MX_FP6_E3M2 else 1.0) + 1.0 / 32.0
     SC = [torch.empty(s.n_groups, device=dev) for s in specs]
     GBT = [torch.empty(s.n_groups, device=dev) for s in specs]
     fwd_plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=WH, scale=SC, mx_format=mx_format)
@@ -74,7 +74,7 @@ def run(name: str, specs, reps: int, dev, mx_format=None) -> dict:
     fwd_bytes = n * (2.0 + out_bytes) + n_groups * 8
     bwd_bytes = n * 2.0 + n_groups * 8
     peak = _peak_gbs()
-    line = {"workload": name, "elements": n, "tensors": len(specs), "output": "bf16" if mx_format is None else ("mx_fp8_e4m3", "mx_fp6_e3m2")[mx_format],
+    line = {"workload": name, "elements": n, "tensors": len(specs), "output": "bf16" if mx_format is None else ("mx_fp8_e4m3", "mx_fp6_e3m2", "mx_fp8_e3m4")[mx_format],
             "fwd_us": t_fwd * 1e3, "fwd_GB/s": fwd_bytes / t_fwd / 1e6, "fwd_frac_of_measured_hbm": fwd_bytes / t_fwd / 1e6 / peak,
             "bwd_us": t_bwd * 1e3, "bwd_GB/s": bwd_bytes / t_bwd / 1e6, "bwd_frac_of_measured_hbm": bwd_bytes / t_bwd / 1e6 / peak,
             "launches_fwd": fwd_plan.launches_per_pass, "launches_bwd": bwd_plan.launches_per_pass, "reps": reps, "l2": "flushed between passes"}
@@ -155,7 +155,7 @@ def main(argv=None) -> None:
         elif w == "gemm":
             run_gemm(args.reps, dev)
         elif w == "mx":
-            for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2):
+            for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2, gws.MX_FP8_E3M4):
                 run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev, mx_format=fmt)
         else:
             raise SystemExit(f"unknown workload {w!r}")

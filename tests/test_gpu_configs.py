@@ -167,7 +167,7 @@ def test_config5_sample_then_gemm_unfused():
             assert abs(got - want) <= budget, (m, n, got, want)
 
 
-@pytest.mark.parametrize("fmt_gpu,fmt_orc", [(gws.MX_FP8_E4M3, orc.MX_E4M3), (gws.MX_FP6_E3M2, orc.MX_E3M2)])
+@pytest.mark.parametrize("fmt_gpu,fmt_orc", [(gws.MX_FP8_E4M3, orc.MX_E4M3), (gws.MX_FP6_E3M2, orc.MX_E3M2), (gws.MX_FP8_E3M4, orc.MX_E3M4)])
 def test_config3_with_mx_output_on_row_slices(fmt_gpu, fmt_orc):
     # the whole Llama2-1B-shaped set in one launch with w_hat written as MX; the oracle on a slice of every tensor
     specs = syn.llama2_1b()
@@ -182,7 +182,7 @@ def test_config3_with_mx_output_on_row_slices(fmt_gpu, fmt_orc):
     plan.sample_fwd_mx_multi(fmt_gpu, step)
     torch.cuda.synchronize()
     rng = np.random.default_rng(11)
-    code_bytes_per_row = lambda cols: cols if fmt_orc == orc.MX_E4M3 else cols * 3 // 4
+    code_bytes_per_row = lambda cols: cols * 3 // 4 if fmt_orc == orc.MX_E3M2 else cols
     for i, s in enumerate(specs):
         nrows = 4
         r0 = int(rng.integers(0, s.rows - nrows)) if i % 7 else s.rows - nrows      # the last rows of some tensors
@@ -190,7 +190,7 @@ def test_config3_with_mx_output_on_row_slices(fmt_gpu, fmt_orc):
         hat, _ = orc.sample_fwd(bits_of(W[i][r0:r0 + nrows]), BT[i][r0 * gpr:(r0 + nrows) * gpr].cpu().numpy(), nrows, s.cols, 1,
                                 s.group_cols, seed=descs[i].seed, step=step, elem_offset=r0 * s.cols)
         codes, scales = orc.mx_emit(hat, nrows, s.cols, 1, s.group_cols, fmt_orc)
-        want_codes = codes if fmt_orc == orc.MX_E4M3 else orc.mx_pack6(codes)
+        want_codes = orc.mx_pack6(codes) if fmt_orc == orc.MX_E3M2 else codes
         codes_bytes, scales_off, _ = gws.mx_layout(descs[i], fmt_gpu)
         cb = code_bytes_per_row(s.cols)
         got_codes = MX[i][r0 * cb:(r0 + nrows) * cb].cpu().numpy()

@@ -14,7 +14,7 @@ from util import bits_of
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-FORMATS = [(gws.MX_FP8_E4M3, orc.MX_E4M3), (gws.MX_FP6_E3M2, orc.MX_E3M2)]
+FORMATS = [(gws.MX_FP8_E4M3, orc.MX_E4M3), (gws.MX_FP6_E3M2, orc.MX_E3M2), (gws.MX_FP8_E3M4, orc.MX_E3M4)]
 
 # (rows, cols, group_rows, group_cols): flat groups (several tiles, a ragged last tile), rows shared by 1..32 threads and
 # rows that take a whole block, square blocks
@@ -44,7 +44,7 @@ def _unpack(buf, desc, fmt_gpu):
 
 def _want(w_hat_bits, rows, cols, gr, gc, fmt_orc):
     codes, scales = orc.mx_emit(w_hat_bits, rows, cols, gr, gc, fmt_orc)
-    return (codes if fmt_orc == orc.MX_E4M3 else orc.mx_pack6(codes)), scales
+    return (orc.mx_pack6(codes) if fmt_orc == orc.MX_E3M2 else codes), scales
 
 
 @pytest.mark.parametrize("fmt_gpu,fmt_orc", FORMATS)
@@ -105,7 +105,7 @@ def test_many_tensors_share_launches(fmt_gpu, fmt_orc):
     before = gws.launch_count()
     assert lib.gws_sample_fwd_multi(ctypes.byref(plan.plan), 9, None) == binding.ERR_UNSUPPORTED
     assert lib.gws_sample_fwd_scaled_multi(ctypes.byref(plan.plan), 9, None) == binding.ERR_UNSUPPORTED
-    assert lib.gws_sample_fwd_mx_multi(ctypes.byref(plan.plan), 1 - fmt_gpu, 9, None) == binding.ERR_UNSUPPORTED
+    assert lib.gws_sample_fwd_mx_multi(ctypes.byref(plan.plan), (fmt_gpu + 1) % 3, 9, None) == binding.ERR_UNSUPPORTED
     bf16_plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=[torch.empty_like(t) for t in W], scale=SC)
     assert lib.gws_sample_fwd_mx_multi(ctypes.byref(bf16_plan.plan), fmt_gpu, 9, None) == binding.ERR_UNSUPPORTED
     assert gws.launch_count() == before
@@ -150,7 +150,7 @@ def test_nan_and_inf_never_fault():
     w.view(-1)[9000] = float("-inf")
     d = Desc.make(64, 256, 1, 128, seed=1, step=1)
     bt = torch.full((gws.n_groups(d),), 5.0, device=DEV)
-    for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2):
+    for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2, gws.MX_FP8_E3M4):
         gws.sample_fwd_mx(d, fmt, w.to(DEV), bt)
         gws.mx_quantize(d, fmt, w.to(DEV))
     gws.sample_fwd_scaled(d, w.to(DEV), torch.full((gws.n_groups(d),), float("nan"), device=DEV))
