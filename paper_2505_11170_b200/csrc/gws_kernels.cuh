@@ -224,44 +224,54 @@ __device__ __forceinline__ uint16_t hi16(uint32_t x) { return static_cast<uint16
 // The per-group factor in the forms the forward pass needs.  The decode delivers 2R, so the
 // multiplier is s/2; halving is exact unless s is below 2^-125, where the product is formed as
 // (2R * 0.5) * s instead (both roundings then match R * s).
+// When s/2 has at most 8 significant bits (always for integer bit-widths: the group maximum is a BF16 number and
+// 2^(1-b) a power of two) it is itself a BF16 number, and w + 2R * (s/2) is one mixed-precision fma per element: the
+// product is exact, so the single rounding of the fma is the rounding of the separate add.
 struct Scale {
   float s, half;
-  bool tiny;
+  bool tiny, half_is_bf16;
 };
 __device__ __forceinline__ Scale make_scale(float s) {
   Scale k;
   k.s = s;
   k.half = __fmul_rn(s, 0.5f);
   k.tiny = s < 0x1p-120f;
+  k.half_is_bf16 = !k.tiny && (__float_as_uint(k.half) & 0xFFFFu) == 0u;
   return k;
 }
-template <bool TINY>
+// FORM: 0 = one multiply per element; 1 = tiny scale; 2 = s/2 is a BF16 number
+template <int FORM>
 __device__ __forceinline__ float noise_term(float two_r, const Scale& k) {
-  return TINY ? __fmul_rn(__fmul_rn(two_r, 0.5f), k.s) : __fmul_rn(two_r, k.half);
+  return FORM == 1 ? __fmul_rn(__fmul_rn(two_r, 0.5f), k.s) : __fmul_rn(two_r, k.half);
 }
 
 // Eq. 3 + cast for one pair word: 2 x ( bf16_rne( fl32(w + R*s) ) ).  R*s is exact, the add rounds
 // once in FP32 (a separate instruction: never contracted), the pack rounds to nearest even.
-template <bool TINY>
+template <int FORM>
 __device__ __forceinline__ uint32_t sample_pair_t(uint32_t w, uint32_t pair, const Scale& k) {
-  const float ql = noise_term<TINY>(__uint_as_float(pair << 16), k);
-  const float qh = noise_term<TINY>(__uint_as_float(pair & 0xFFFF0000u), k);
+  if (FORM == 2) {
+    const uint16_t hb = hi16(__float_as_uint(k.half));
+    return pack_bf16_rne(fma_bf16(static_cast<uint16_t>(pair & 0xFFFFu), hb, __uint_as_float(w << 16)),
+                         fma_bf16(hi16(pair), hb, __uint_as_float(w & 0xFFFF0000u)));
+  }
+  const float ql = noise_term<FORM>(__uint_as_float(pair << 16), k);
+  const float qh = noise_term<FORM>(__uint_as_float(pair & 0xFFFF0000u), k);
   return pack_bf16_rne(__fadd_rn(__uint_as_float(w << 16), ql), add_bf16(hi16(w), qh));
 }
-template <bool TINY>
+template <int FORM>
 __device__ __forceinline__ uint4 sample_vec_t(const uint4& w, const Words4& r, const Scale& k) {
   uint32_t p[4];
   decode8(r, p);
-  return make_uint4(sample_pair_t<TINY>(w.x, p[0], k), sample_pair_t<TINY>(w.y, p[1], k), sample_pair_t<TINY>(w.z, p[2], k),
-                    sample_pair_t<TINY>(w.w, p[3], k));
+  return make_uint4(sample_pair_t<FORM>(w.x, p[0], k), sample_pair_t<FORM>(w.y, p[1], k), sample_pair_t<FORM>(w.z, p[2], k),
+                    sample_pair_t<FORM>(w.w, p[3], k));
 }
-// The tiny-scale form is chosen once per vector / chunk (it is a property of the group), so the common
-// path carries one multiply per element.
+// The form is chosen once per vector / chunk (it is a property of the group), so the common path carries one
+// fma (or one multiply and one add) per element.
 __device__ __forceinline__ uint4 sample_vec(const uint4& w, const Words4& r, const Scale& k) {
-  return k.tiny ? sample_vec_t<true>(w, r, k) : sample_vec_t<false>(w, r, k);
+  return k.half_is_bf16 ? sample_vec_t<2>(w, r, k) : (k.tiny ? sample_vec_t<1>(w, r, k) : sample_vec_t<0>(w, r, k));
 }
 // One 64-byte chunk whose first vector has the (low) Philox counter word v0.  y may be x (word j depends on word j alone).
-template <bool TINY>
+template <int FORM>
 __device__ __forceinline__ void sample_chunk_t(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
                                                const Scale& sc, uint32_t* y) {
 #pragma unroll
@@ -270,11 +280,11 @@ __device__ __forceinline__ void sample_chunk_t(const uint32_t* x, uint32_t v0, u
     uint32_t p[4];
     decode8(r, p);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) y[4 * k + j] = sample_pair_t<TINY>(x[4 * k + j], p[j], sc);
+    for (int j = 0; j < 4; ++j) y[4 * k + j] = sample_pair_t<FORM>(x[4 * k + j], p[j], sc);
   }
 }
 // Half a chunk: 16 elements, two Philox vectors.
-template <bool TINY>
+template <int FORM>
 __device__ __forceinline__ void sample_half_t(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
                                               const Scale& sc, uint32_t* y) {
 #pragma unroll
@@ -283,13 +293,20 @@ __device__ __forceinline__ void sample_half_t(const uint32_t* x, uint32_t v0, ui
     uint32_t p[4];
     decode8(r, p);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) y[4 * k + j] = sample_pair_t<TINY>(x[4 * k + j], p[j], sc);
+    for (int j = 0; j < 4; ++j) y[4 * k + j] = sample_pair_t<FORM>(x[4 * k + j], p[j], sc);
   }
+}
+__device__ __forceinline__ void sample_half(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
+                                            const Scale& sc, uint32_t* y) {
+  if (sc.half_is_bf16) sample_half_t<2>(x, v0, k0, k1, pre, sc, y);
+  else if (sc.tiny) sample_half_t<1>(x, v0, k0, k1, pre, sc, y);
+  else sample_half_t<0>(x, v0, k0, k1, pre, sc, y);
 }
 __device__ __forceinline__ void sample_chunk(const uint32_t* x, uint32_t v0, uint32_t k0, uint32_t k1, const PhiloxPre& pre,
                                              const Scale& sc, uint32_t* y) {
-  if (sc.tiny) sample_chunk_t<true>(x, v0, k0, k1, pre, sc, y);
-  else sample_chunk_t<false>(x, v0, k0, k1, pre, sc, y);
+  if (sc.half_is_bf16) sample_chunk_t<2>(x, v0, k0, k1, pre, sc, y);
+  else if (sc.tiny) sample_chunk_t<1>(x, v0, k0, k1, pre, sc, y);
+  else sample_chunk_t<0>(x, v0, k0, k1, pre, sc, y);
 }
 
 // Running sum of float(g) * 2R: low and high BF16 halves of every pair go to their own accumulator
@@ -816,8 +833,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
     uint32_t my = 0u;               // w_hat replaces w in the registers until the block maximum is known
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      if (sc.tiny) sample_half_t<true>(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, x[k]);
-      else sample_half_t<false>(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, x[k]);
+      sample_half(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, x[k]);
       my = maxabs2(my, maxabs2(absmax_words4(x[k]), absmax_words4(x[k] + 4)));
     }
     const float ay = absmax_finish(block_max(my));
@@ -828,8 +844,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       uint32_t y[8];
-      if (sc.tiny) sample_half_t<true>(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, y);
-      else sample_half_t<false>(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, y);
+      sample_half(x[k], e.vec_lo + piece[k] * 2u, e.k0, e.k1, e.pre, sc, y);
       if (ok) st_vec32(e.out, static_cast<uint64_t>(piece[k]) * 32u, y);
     }
   }
