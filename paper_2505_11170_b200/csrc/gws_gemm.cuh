@@ -102,7 +102,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
 }
 
 template <int MT>
-__global__ void __launch_bounds__(kGemmThreads) k_gemm_fused(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ GemmArgs a) {
+__global__ void __launch_bounds__(kGemmThreads, MT == 4 ? 1 : 2) k_gemm_fused(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: the swizzle pattern is a function of the address bits 7..9
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023u) & ~static_cast<uintptr_t>(1023u));
