@@ -171,14 +171,14 @@ int gws_sample_fwd_scaled(const gws_desc* desc, const void* w, const float* scal
  * 32-element row vectors of a group (a 32 x 32 block, a 1 x G group, a row) carry the same
  * scale, which keeps a square block consistent under transposition.
  *   scale byte (E8M0)  max(E - emax, 0), E = biased exponent of max_group |w_hat|: the shared
- *                      exponent floor(log2 max) - emax clamped below at -127 (emax = 8 / 4)
+ *                      exponent floor(log2 max) - emax clamped below at -127 (emax = 8 for E4M3, else 4)
  *   element            w_hat / 2^(byte - 127), round to nearest even onto the element grid
- *                      (subnormals included), clamped to the largest normal (448 / 28); the
+ *                      (subnormals included), clamped to the largest normal (448 / 28 / 31); the
  *                      sign of zero is kept
- * Buffer layout (one device allocation per tensor, 32-byte aligned, see gws_mx_layout):
  * GWS_MX_FP8_E3M4 is Table C.1's FP8_e3m4, which the paper names without defining and which is not
  * an OCP element type: it is read by analogy with E3M2 (bias 3, every code finite, largest normal 31,
  * emax 4) and converted in integer arithmetic (the GPU has no instruction for it).
+ * Buffer layout (one device allocation per tensor, 32-byte aligned, see gws_mx_layout):
  *   [0, codes_bytes)            element codes in logical row-major order.  E4M3 / E3M4: one byte each.
  *                               E3M2: a little-endian bit stream, element k at bits [6k, 6k+5]
  *                               (4 elements in 3 bytes, a 32-element vector in 24).
