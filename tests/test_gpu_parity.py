@@ -403,3 +403,37 @@ def test_errors_surface_as_exceptions():
     assert e.value.status == -5
     with pytest.raises(ValueError):
         gws.sample_fwd(Desc.make(4, 64, 1, 32), w.cpu(), bt)
+
+
+def test_multi_tensor_launches_replay_from_a_cuda_graph():
+    # the launches of a plan carry their tensor records in the kernel parameters, so a captured graph replays them
+    # as they are: same step, same bits; nothing in the library synchronises or allocates during the capture
+    specs = [syn.TensorSpec("a", 64, 1024, 1, 128), syn.TensorSpec("b", 48, 768, 1, 0), syn.TensorSpec("c", 64, 96, 32, 32)]
+    descs = [Desc.make(s.rows, s.cols, s.group_rows, s.group_cols, seed=31 + i) for i, s in enumerate(specs)]
+    W = [syn.weights(s, i, device=DEV) for i, s in enumerate(specs)]
+    BT = [syn.bitwidths(s, i, device=DEV) for i, s in enumerate(specs)]
+    G = [syn.upstream_grad(s, i, device=DEV) for i, s in enumerate(specs)]
+    WH = [torch.zeros_like(t) for t in W]
+    SC = [torch.zeros(s.n_groups, device=DEV) for s in specs]
+    GBT = [torch.zeros(s.n_groups, device=DEV) for s in specs]
+    plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=WH, scale=SC, grad_w_hat=G, grad_bt=GBT)
+    plan.sample_fwd_multi(5)
+    plan.sample_bwd_multi(5)
+    torch.cuda.synchronize()
+    want = [t.clone() for t in WH + SC + GBT]
+    for t in WH + SC + GBT:
+        t.zero_()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            plan.sample_fwd_multi(5, stream=side)
+            plan.sample_bwd_multi(5, stream=side)
+    torch.cuda.synchronize()
+    assert all((t == 0).all() for t in WH)            # capture records, it does not run
+    graph.replay()
+    torch.cuda.synchronize()
+    for got, ref in zip(WH + SC + GBT, want):
+        assert torch.equal(got.view(torch.int16) if got.dtype == torch.bfloat16 else got.view(torch.int32),
+                           ref.view(torch.int16) if ref.dtype == torch.bfloat16 else ref.view(torch.int32))
