@@ -50,7 +50,10 @@
  *   - NaN / Inf in the inputs give unspecified values but never a fault.
  *
  * Every function returns 0 (GWS_OK) or a negative gws_status.  Arguments are validated on
- * the host before anything is launched; a failed call has enqueued nothing.
+ * the host before anything is launched: a call that fails validation has enqueued nothing.  The
+ * calls that issue several launches (the *_multi family, gws_sample_step_host) can also fail in
+ * the middle with GWS_ERR_CUDA or GWS_ERR_LIMIT, when the runtime rejects one launch; the launches
+ * before it are then already enqueued and their outputs should be treated as unspecified.
  */
 #ifndef GWS_H_
 #define GWS_H_
@@ -220,7 +223,9 @@ int gws_sample_fwd_mx(const gws_desc* desc, int format, const void* w, const flo
  *   rows_per_block  128, 256 or 512: rows of X per thread block; every sampled tile of W is used for that
  *                   many rows, so a larger value repeats less sampling work (512 takes all tensor memory
  *                   and 161 KiB of shared memory of an SM).
- * Other shapes: GWS_ERR_UNSUPPORTED.  gws_gemm_last_error() describes a GWS_ERR_CUDA of this call.
+ * Other shapes: GWS_ERR_UNSUPPORTED.  An output (y, w_hat_out, scale_out) that overlaps an input (x, w, bt) or
+ * another output: GWS_ERR_ALIAS (thread blocks re-read W and X while others write).
+ * gws_gemm_last_error() describes a GWS_ERR_CUDA of this call.
  */
 int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y,
                    void* w_hat_out, float* scale_out, int* status, int rows_per_block, void* stream);
@@ -363,8 +368,13 @@ uint64_t gws_layer_seed(uint64_t user_seed, uint64_t layer);
  * forward pass only, and allocates no device memory, frees none and calls no allocating library
  * routine.
  *   n, descs, ptrs   as for gws_multi_prepare; only w, bt, w_hat and scale of `ptrs` are used
- *                    (scale, and each of its entries, may be NULL).  n > GWS_STATIC_MAX_TENSORS
- *                    returns GWS_ERR_LIMIT and enqueues nothing.
+ *                    (scale, and each of its entries, may be NULL) and w_hat must be BF16 tensors
+ *                    (w_hat_kind = 0, anything else is GWS_ERR_UNSUPPORTED).  n > GWS_STATIC_MAX_TENSORS
+ *                    returns GWS_ERR_LIMIT.  Every error found while validating the arguments is
+ *                    returned before the array is touched and before anything is enqueued.
+ *   stream           must not be recording (cudaStreamBeginCapture): the call then returns
+ *                    GWS_ERR_UNSUPPORTED with nothing enqueued, because its table upload reads host
+ *                    memory that lives only for the duration of the call.
  *   step             gradient-update counter, as for gws_sample_fwd_multi
  * Results are bit-identical to gws_sample_fwd_multi.  Things to know:
  *   - The first call on each device looks up the array's device address (with that device current).
@@ -413,6 +423,9 @@ int64_t gws_noise_alu_probe_words(const gws_desc* desc);
 /* Host-side evaluation of the same inline decode / Philox code the kernels use (no GPU needed):
  * r8 receives R for the 8 fields of the 4 words; packed receives the nibble word. */
 void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed);
+/* The decode's raw output, four words holding the BF16 patterns of 2R for elements (2j, 2j+1), from the form the
+ * forward pass uses (a zero is always +0) and from the form the gradient sum of Eq. 4 uses (a zero may be -0). */
+void gws_host_decode8_pairs(const uint32_t* words4, uint32_t* pairs4, uint32_t* pairs4_signed_zero);
 void gws_host_philox(uint64_t seed, uint64_t step, uint64_t vec, uint32_t* out4);
 
 /* Self-checking build (compiled with -DGWS_SELF_CHECK; gws_selfcheck_enabled() returns 1): every

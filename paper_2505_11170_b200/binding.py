@@ -92,6 +92,7 @@ _SIGNATURES = {
     "gws_noise_alu_probe": (c_int, [POINTER(Desc), c_void_p, c_void_p]),
     "gws_noise_alu_probe_words": (c_int64, [POINTER(Desc)]),
     "gws_host_decode8": (None, [POINTER(c_uint32), POINTER(c_int8), POINTER(c_uint32)]),
+    "gws_host_decode8_pairs": (None, [POINTER(c_uint32), POINTER(c_uint32), POINTER(c_uint32)]),
     "gws_host_philox": (None, [c_uint64, c_uint64, c_uint64, POINTER(c_uint32)]),
     "gws_selfcheck_enabled": (c_int, []),
     "gws_selfcheck_set_window": (c_int, [c_void_p, c_size_t]),
@@ -454,6 +455,14 @@ def host_decode8(words4: Sequence[int]):
     p = c_uint32(0)
     load_library().gws_host_decode8(w, r, ctypes.byref(p))
     return list(r), int(p.value)
+
+
+def host_decode8_pairs(words4: Sequence[int]):
+    """The decode's four pair words (BF16 patterns of 2R) in its two forms: zero always +0, and zero of either sign."""
+    w = (c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in words4])
+    p, q = (c_uint32 * 4)(), (c_uint32 * 4)()
+    load_library().gws_host_decode8_pairs(w, p, q)
+    return list(p), list(q)
 
 
 def host_philox(seed: int, step: int, vec: int) -> List[int]:

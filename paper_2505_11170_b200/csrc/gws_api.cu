@@ -1009,6 +1009,15 @@ int gws_sample_fwd_multi_static(int n, const gws_desc* descs, const gws_multi_pt
   fwd_only.grad_w_hat = nullptr;
   fwd_only.grad_w = nullptr;
   fwd_only.grad_bt = nullptr;
+  if (ptrs->w_hat_kind != 0) return GWS_ERR_UNSUPPORTED;   // BF16 w_hat only; refused before anything is uploaded
+  // The table upload below reads host memory that dies with this call and the launches carry this call's step and
+  // pointers by value: a stream that is recording work for later replay would replay neither correctly.
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(static_cast<cudaStream_t>(stream), &capturing) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return GWS_ERR_UNSUPPORTED;
+  }
+  if (capturing != cudaStreamCaptureStatusNone) return GWS_ERR_UNSUPPORTED;
   void* table = nullptr;
   int st = static_tables_address(&table);
   if (st != GWS_OK) return st;
@@ -1082,6 +1091,18 @@ void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed) {
   gws::decode8(w, p);
   for (unsigned t = 0; t < 8; ++t) r8[t] = static_cast<int8_t>(gws::r_from_pairs(p, t));
   if (packed) *packed = gws::pack_nibbles(w);
+}
+
+void gws_host_decode8_pairs(const uint32_t* words4, uint32_t* pairs4, uint32_t* pairs4_signed_zero) {
+  gws::Words4 w;
+  for (int k = 0; k < 4; ++k) w.o[k] = words4[k];
+  uint32_t p[4], q[4];
+  gws::decode8(w, p);
+  gws::decode8_signed_zero(w, q);
+  for (int k = 0; k < 4; ++k) {
+    pairs4[k] = p[k];
+    pairs4_signed_zero[k] = q[k];
+  }
 }
 
 void gws_host_philox(uint64_t seed, uint64_t step, uint64_t vec, uint32_t* out4) {

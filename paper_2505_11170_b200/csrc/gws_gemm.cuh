@@ -299,6 +299,19 @@ int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* 
   if (misaligned(x, 16) || misaligned(w, 32) || misaligned(y, 16) || misaligned(bt, 4) || misaligned(w_hat_out, 32) || misaligned(scale_out, 4) ||
       misaligned(status, 4))
     return GWS_ERR_ALIGN;
+  // An output laid over an input would be overwritten while other thread blocks still read it (every block along M
+  // re-reads W, every block along N re-reads X): refused like in gws_sample_fwd.
+  const size_t x_bytes = static_cast<size_t>(m) * static_cast<size_t>(k) * 2u, w_bytes = static_cast<size_t>(n) * static_cast<size_t>(k) * 2u;
+  const size_t y_bytes = static_cast<size_t>(m) * static_cast<size_t>(n) * 2u, s_bytes = static_cast<size_t>(n) * static_cast<size_t>(k / kTileK) * 4u;
+  if (overlaps(y, y_bytes, x, x_bytes) || overlaps(y, y_bytes, w, w_bytes) || overlaps(y, y_bytes, bt, s_bytes)) return GWS_ERR_ALIAS;
+  if (w_hat_out != nullptr &&
+      (overlaps(w_hat_out, w_bytes, w, w_bytes) || overlaps(w_hat_out, w_bytes, x, x_bytes) || overlaps(w_hat_out, w_bytes, y, y_bytes) ||
+       overlaps(w_hat_out, w_bytes, bt, s_bytes)))
+    return GWS_ERR_ALIAS;
+  if (scale_out != nullptr &&
+      (overlaps(scale_out, s_bytes, w, w_bytes) || overlaps(scale_out, s_bytes, x, x_bytes) || overlaps(scale_out, s_bytes, y, y_bytes) ||
+       overlaps(scale_out, s_bytes, bt, s_bytes) || (w_hat_out != nullptr && overlaps(scale_out, s_bytes, w_hat_out, w_bytes))))
+    return GWS_ERR_ALIAS;
 
   static EncodeTiled encode = nullptr;
   if (encode == nullptr) {

@@ -323,7 +323,7 @@ __device__ __forceinline__ void dot_pair(uint32_t g, uint32_t pair, DotAcc& acc)
 }
 __device__ __forceinline__ void dot_vec(const uint4& g, const Words4& r, DotAcc& acc) {
   uint32_t p[4];
-  decode8(r, p);
+  decode8_signed_zero(r, p);   // g * (-0) adds a zero of either sign to the running sum: the sum is the same number
   dot_pair(g.x, p[0], acc);
   dot_pair(g.y, p[1], acc);
   dot_pair(g.z, p[2], acc);

@@ -139,6 +139,24 @@ GWS_HD void decode8(const Words4& r, uint32_t (&pair)[4]) {
   pair[3] = (z << 6) & kPairMask;
 }
 
+// The same decode for consumers that only multiply by the noise (the gradient sum of Eq. 4): a zero may come out as
+// -0, because the sign column is taken as it is instead of being cleared where |R| = 0.  Two operations fewer.
+GWS_HD void decode8_signed_zero(const Words4& r, uint32_t (&pair)[4]) {
+  const uint32_t o0 = r.o[0], o1 = r.o[1], o2 = r.o[2], o3 = r.o[3];
+  const uint32_t t1 = o1 & o2 & o3;
+  const uint32_t and7 = t1 & o0 & (t1 << 1);
+  const uint32_t top = o0 & (o1 | o2);
+  const uint32_t m2 = and7 & (top >> 8);
+  const uint32_t m1 = (o0 | o1) & (o0 << 8) & (o2 | o3);
+  const uint32_t any = m1 | (m2 << 7);
+  const uint32_t z1 = (any & ~kColsM) | (m2 & kColsM);
+  const uint32_t z = (o3 & kColsS) | (z1 & ~kColsS);
+  pair[0] = z & kPairMask;
+  pair[1] = (z << 2) & kPairMask;
+  pair[2] = (z << 4) & kPairMask;
+  pair[3] = (z << 6) & kPairMask;
+}
+
 // R of element t (0..7) from the pair words of its vector.
 GWS_HD int r_from_pairs(const uint32_t (&pair)[4], unsigned t) {
   const uint32_t h = (pair[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu;

@@ -24,11 +24,11 @@ class _SampledWeight(torch.autograd.Function):
     """(w, b_i) -> w_hat with the gradients of Eq. 4 and Eq. 11 / Eq. 12."""
 
     @staticmethod
-    def forward(ctx, w, bi, desc, b_init, b_target, lam):
+    def forward(ctx, w, bi, desc, b_init, b_target, lam, update):
         bt = binding.bitwidth(bi.detach(), b_init, b_target)
         w_hat, scale = binding.sample_fwd(desc, w.detach(), bt)
         ctx.save_for_backward(scale, bt)
-        ctx.desc, ctx.hyper = desc, (b_init, b_target, lam)
+        ctx.desc, ctx.hyper, ctx.update = desc, (b_init, b_target, lam), update
         return w_hat
 
     @staticmethod
@@ -37,8 +37,12 @@ class _SampledWeight(torch.autograd.Function):
         b_init, b_target, lam = ctx.hyper
         g = grad_w_hat.contiguous()
         _, grad_bt = binding.sample_bwd(ctx.desc, g, scale)                 # dL/dw is dL/dw_hat itself (Eq. 4)
-        grad_bi = binding.bitwidth_grad(grad_bt, bt, b_init, b_target, lam)
-        return g, grad_bi, None, None, None, None
+        # Eq. 12 adds its term once per gradient update, however many micro-batches are accumulated into b_i.grad:
+        # the first backward pass of an update carries it, the others are the plain chain rule.
+        first = ctx.update["lambda_term_due"]
+        ctx.update["lambda_term_due"] = False
+        grad_bi = binding.bitwidth_grad(grad_bt, bt, b_init, b_target, lam if first else 0.0)
+        return g, grad_bi, None, None, None, None, None
 
 
 class GaussWSLinear(torch.nn.Module):
@@ -47,7 +51,9 @@ class GaussWSLinear(torch.nn.Module):
     ``group`` is (group_rows, group_cols); the paper's choice is the 32 x 32 square block.  ``layer_index`` and
     ``user_seed`` give the layer its own noise stream (Section 3.6); call :meth:`advance` once per gradient update
     (not per micro-batch) so that forward and backward of one update see the same noise and the next update a new one.
-    ``lam`` > 0 adds this layer's term of Eq. 12 to the gradient of ``b_i``; :meth:`bitwidth_loss` returns its value.
+    ``lam`` > 0 adds this layer's term of Eq. 12 to the gradient of ``b_i``, once per update: the first backward pass
+    after construction or :meth:`advance` carries it, so accumulating k micro-batches does not multiply lambda by k;
+    :meth:`bitwidth_loss` returns the term's value.
     """
 
     def __init__(self, in_features: int, out_features: int, bias: bool = True, group=(32, 32), b_init: float = 6.0,
@@ -60,6 +66,7 @@ class GaussWSLinear(torch.nn.Module):
         self.bias = torch.nn.Parameter(torch.zeros(out_features, dtype=torch.bfloat16, device=device)) if bias else None
         self.seed = binding.layer_seed(user_seed, layer_index)
         self.step = 0
+        self._update = {"lambda_term_due": True}
         n_groups = binding.n_groups(self._desc())
         self.b_i = torch.nn.Parameter(torch.ones(n_groups, dtype=torch.float32, device=device))   # Eq. 11: starts at 1
 
@@ -69,9 +76,10 @@ class GaussWSLinear(torch.nn.Module):
     def advance(self) -> None:
         """One gradient update has been applied: the next forward pass draws new noise."""
         self.step += 1
+        self._update["lambda_term_due"] = True
 
     def sampled_weight(self) -> torch.Tensor:
-        return _SampledWeight.apply(self.weight, self.b_i, self._desc(), self.b_init, self.b_target, self.lam)
+        return _SampledWeight.apply(self.weight, self.b_i, self._desc(), self.b_init, self.b_target, self.lam, self._update)
 
     def bitwidth(self) -> torch.Tensor:
         return binding.bitwidth(self.b_i.detach(), self.b_init, self.b_target)

@@ -150,3 +150,46 @@ def test_inline_decode_matches_oracle_on_every_field_value(lib):
                 # neighbours are decoded from their own bits
                 for u in range(8):
                     assert r[u] == want[orc.field_of_element(words, u)]
+
+
+def test_gradient_decode_differs_from_the_forward_decode_only_in_the_sign_of_zero(lib):
+    # the backward kernels skip the step that clears the sign of a zero noise value (g * -0 adds nothing to the sum);
+    # everything else about the two decodes must agree, on random words and on words that make |R| = 2 likely
+    rng = np.random.default_rng(5)
+    cases = [rng.integers(0, 2**32, size=4, dtype=np.uint64) for _ in range(4000)]
+    cases += [rng.integers(0, 2**32, size=4, dtype=np.uint64) | rng.integers(0, 2**32, size=4, dtype=np.uint64) |
+              rng.integers(0, 2**32, size=4, dtype=np.uint64) for _ in range(4000)]
+    seen_minus_zero = seen_two = 0
+    for words in cases:
+        p, q = binding.host_decode8_pairs([int(x) for x in words])
+        r, _ = binding.host_decode8([int(x) for x in words])
+        for j in range(4):
+            for h in range(2):
+                a, b = (p[j] >> (16 * h)) & 0xFFFF, (q[j] >> (16 * h)) & 0xFFFF
+                assert a & 0x7FFF == b & 0x7FFF
+                if a & 0x7FFF:
+                    assert a == b
+                else:
+                    assert a == 0 and b in (0, 0x8000)
+                    seen_minus_zero += b == 0x8000
+                seen_two += (a & 0x7FFF) == 0x4080
+                assert {0: 0, 0x4000: 1, 0x4080: 2}[a & 0x7FFF] == abs(r[2 * j + h])
+    assert seen_minus_zero > 1000 and seen_two > 50
+
+
+def test_fused_gemm_refuses_outputs_that_overlap_inputs(lib):
+    # every thread block along M re-reads W and every block along N re-reads X, so an output laid over an input would
+    # silently corrupt Y (and the master weights); the check is host arithmetic on the pointers, nothing is launched
+    n, k, m = 128, 128, 128
+    d = Desc.make(n, k, 1, 128)
+    x, w, bt, y, wh, sc = (ctypes.c_void_p(0x10000000 + 0x100000 * i) for i in range(6))
+    null = ctypes.c_void_p(None)
+    call = lambda x_, w_, bt_, y_, wh_, sc_: lib.gws_gemm_fused(ctypes.byref(d), m, x_, w_, bt_, y_, wh_, sc_, null, 128, null)
+    before = gws.launch_count()
+    assert call(x, w, bt, y, w, null) == binding.ERR_ALIAS                                 # w_hat_out on top of w
+    assert call(x, w, bt, y, ctypes.c_void_p(w.value + 2 * n * k - 32), null) == binding.ERR_ALIAS   # ... or only touching its tail
+    assert call(x, w, bt, x, null, null) == binding.ERR_ALIAS                              # y on top of x
+    assert call(x, w, bt, w, null, null) == binding.ERR_ALIAS                              # y on top of w
+    assert call(x, w, bt, y, y, null) == binding.ERR_ALIAS                                 # the two outputs on each other
+    assert call(x, w, bt, y, wh, bt) == binding.ERR_ALIAS                                  # scale_out on top of bt
+    assert gws.launch_count() == before

@@ -91,3 +91,40 @@ def test_module_noise_changes_only_when_advanced():
     with torch.no_grad():
         other.weight.copy_(layer.weight)
     assert not torch.equal(other.sampled_weight().detach(), c) and other.seed != layer.seed
+
+
+def test_module_adds_the_bitwidth_loss_term_once_per_update():
+    # Eq. 12's term belongs to the update, not to the micro-batch: two accumulated backward passes at one step give
+    # twice the Eq. 4 gradient but the lambda term once; after advance() the next backward pass carries it again
+    torch.manual_seed(1)
+    lam = 0.5
+    layer = GaussWSLinear(128, 64, bias=False, group=(1, 128), b_init=6.0, b_target=4.0, lam=lam, user_seed=2, layer_index=5)
+    with torch.no_grad():
+        layer.b_i.uniform_(0.2, 1.2)
+    x = torch.randn(16, 128, device=DEV, dtype=torch.bfloat16)
+    upstream = torch.randn(16, 64, device=DEV, dtype=torch.bfloat16) * 1e-2
+
+    def one_backward():
+        layer.b_i.grad = None
+        layer.weight.grad = None
+        layer(x).backward(upstream)
+        return layer.b_i.grad.detach().cpu().numpy().astype(np.float64)
+
+    bt = orc.bitwidth(layer.b_i.detach().cpu().numpy(), 6.0, 4.0)
+    with_term = one_backward()            # first backward pass of the update: chain rule + lambda term
+    without_term = one_backward()         # second one of the same update: chain rule only
+    m = bt.size
+    term = (6.0 - 4.0) * lam / m * np.sign(bt.astype(np.float64) - 4.0)
+    assert np.abs(with_term - without_term - term).max() <= 1e-6 * np.abs(term).max() + 1e-12
+    # accumulated over the two micro-batches
+    layer.advance()
+    layer.b_i.grad = None
+    layer(x).backward(upstream)
+    layer(x).backward(upstream)
+    acc = layer.b_i.grad.detach().cpu().numpy().astype(np.float64)
+    layer.advance()
+    layer.step -= 1                        # same noise, a fresh update
+    layer.b_i.grad = None
+    layer(x).backward(upstream)
+    single = layer.b_i.grad.detach().cpu().numpy().astype(np.float64)
+    assert np.abs(acc - (2.0 * single - term)).max() <= 1e-5 * np.abs(single).max()

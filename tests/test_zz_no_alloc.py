@@ -8,6 +8,8 @@ table, so the second call here uses a different tensor set, order and step on pu
 
 Collected last (file name), so a run that stops at the first failure has seen every other test first.
 """
+import ctypes
+
 import pytest
 import torch
 
@@ -42,8 +44,11 @@ def _same_bits(a, b):
 def test_static_table_forward_matches_workspace_forward_on_two_calls_in_a_row():
     first = [syn.TensorSpec("q", 96, 2048, 1, 128), syn.TensorSpec("fc", 40, 768, 1, 0), syn.TensorSpec("wide", 3, 8192, 1, 0),
              syn.TensorSpec("g32", 33, 96, 1, 32), syn.TensorSpec("ragged", 10, 100, 1, 48)]
-    second = [syn.TensorSpec("row", 70, 3072, 1, 0), syn.TensorSpec("down", 64, 5632, 1, 128),
-              syn.TensorSpec("sq", 64, 64, 32, 32)]
+    # "odd" (groups of 24 that do not divide the row) and "tall" (2-D groups that are not whole 32 x 32 blocks) run on
+    # the kernel class that reads its tensor records from the built-in array on the device: the second call must
+    # find its own records there, at other positions than the first call's "ragged" one had
+    second = [syn.TensorSpec("odd", 7, 200, 1, 24), syn.TensorSpec("row", 70, 3072, 1, 0), syn.TensorSpec("down", 64, 5632, 1, 128),
+              syn.TensorSpec("sq", 64, 64, 32, 32), syn.TensorSpec("tall", 20, 40, 4, 8)]
     for call, (specs, base, step) in enumerate([(first, 0, 5), (second, 100, 6)]):
         descs, W, BT = _tensor_set(specs, base)
         want_hat, want_sc = _outputs(specs, W)
@@ -81,3 +86,36 @@ def test_static_table_rejects_more_tensors_than_it_holds():
     assert "maximum" in gws.status_string(binding.ERR_LIMIT)
     assert lib.gws_sample_fwd_multi_static(-1, descs, ctypes.byref(ptrs), 0, None) == binding.ERR_SHAPE
     assert lib.gws_sample_fwd_multi_static(1, None, ctypes.byref(ptrs), 0, None) == binding.ERR_NULL
+    # MX outputs belong to gws_sample_fwd_mx_multi: refused here before the array is touched
+    mx = binding._MultiPtrs(arr, arr, arr, None, None, None, None, 1)
+    assert lib.gws_sample_fwd_multi_static(1, descs, ctypes.byref(mx), 0, None) == binding.ERR_UNSUPPORTED
+
+
+@pytest.mark.gpu
+@pytest.mark.filterwarnings("ignore:The CUDA Graph is empty")
+def test_static_table_call_is_refused_while_the_stream_is_recording():
+    # the table upload reads host memory that is gone when the call returns, so the call declines to become
+    # part of a recorded graph; an ordinary call right afterwards is unaffected
+    specs = [syn.TensorSpec("q", 16, 256, 1, 128), syn.TensorSpec("ragged", 10, 100, 1, 48)]
+    descs, W, BT = _tensor_set(specs, 3)
+    want_hat, want_sc = _outputs(specs, W)
+    gws.MultiPlan(descs, w=W, bt=BT, w_hat=want_hat, scale=want_sc).sample_fwd_multi(4)
+    got_hat, got_sc = _outputs(specs, W)
+    gws.sample_fwd_multi_static(descs, W, BT, got_hat, got_sc, step=4)     # the device's first call: outside capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        try:
+            with pytest.raises(binding.GwsError) as err:
+                gws.sample_fwd_multi_static(descs, W, BT, got_hat, got_sc, step=4, stream=side)
+            assert err.value.status == binding.ERR_UNSUPPORTED
+        finally:
+            graph.capture_end()
+    torch.cuda.synchronize()
+    got_hat, got_sc = _outputs(specs, W)
+    gws.sample_fwd_multi_static(descs, W, BT, got_hat, got_sc, step=4)
+    torch.cuda.synchronize()
+    for i, s in enumerate(specs):
+        assert _same_bits(got_hat[i], want_hat[i]) and _same_bits(got_sc[i], want_sc[i]), s.name
