@@ -1,11 +1,14 @@
 #!/usr/bin/env python
 """Benchmark of the GaussWS weight-sampling pass on B200.
 
-One "step" = one forward pass (Eq. 3 + BF16 cast) plus one backward pass (Eq. 4, noise
-regenerated) over the whole Llama2-1B-shaped linear weight set (154 tensors, 1,130,364,928 BF16
-elements, groups of 128 along the input dimension, b_t uniform on {4..9}), each pass one launch.
-Inputs are synthetic (seeded N(0, 0.02^2) weights, N(0, 1e-4^2) upstream gradients) and resident
-in HBM when the timed region starts; every pass streams 2.26 GB per tensor set, far beyond L2.
+One "step" = the workload's ten consecutive gradient-update counters: ten times one forward pass
+(Eq. 3 + BF16 cast) plus one backward pass (Eq. 4, noise regenerated) over the whole Llama2-1B-shaped
+linear weight set (154 tensors, 1,130,364,928 BF16 elements, groups of 128 along the input dimension,
+b_t uniform on {4..9}), each pass one launch.  Inputs are synthetic (seeded N(0, 0.02^2) weights,
+N(0, 1e-4^2) upstream gradients) and resident in HBM when the timed region starts; every pass streams
+2.26 GB per tensor set, far beyond L2.  `value` comes from exactly --steps steps; the roofline
+fractions are reported twice: over the first 20 launches of each kernel (a burst at full clocks) and
+sustained (everything after the first 0.3 s, the run extended to at least 1.5 s of device time).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -29,6 +32,9 @@ if ROOT not in sys.path:
 
 METRIC = "sampling fwd+bwd GB/s and Gelem/s at 1 B200; fraction of HBM peak"
 WORKLOAD = "llama2_1b_linear_set_g128"
+PASSES_PER_STEP = 10                       # the workload names ten consecutive step counters
+SUSTAIN_MS = 1500.0                        # device time the launch stream is extended to for the sustained figures
+BURST_LAUNCHES = 20
 FWD_BYTES_PER_ELEM = 2 + 2 + 8 / 128      # read w, write w_hat, read b_t + write scale per 128 elements
 BWD_BYTES_PER_ELEM = 2 + 8 / 128          # read dL/dw_hat, read scale + write dL/db_t per 128 elements
 FALLBACK_HBM_GBS = 6650.0
@@ -115,16 +121,24 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.samples.append((time.time(), line.strip()))
 
-    def stop(self, t0: float, t1: float):
+    def stop(self):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return
         time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
-        rows = [s for (t, s) in self.samples if t0 - 0.05 <= t <= t1 + 0.15] or [s for (_, s) in self.samples]
+
+    def window(self, t0: float, t1: float):
+        """Median SM clock and the throttle reasons seen between two wall-clock times."""
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        rows = [s for (t, s) in self.samples if t0 - 0.03 <= t <= t1 + 0.03]
+        if not rows:      # a window shorter than the sampling period: the nearest sample
+            mid = 0.5 * (t0 + t1)
+            rows = [min(self.samples, key=lambda ts: abs(ts[0] - mid))[1]] if self.samples else []
         mhz, mx, reasons = [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
@@ -171,7 +185,8 @@ def run_reference(args, rank: int, world: int):
         step(args.warmup + k)
     dt = time.perf_counter() - t0
     gbs = elems * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM) * args.steps / dt / 1e9
-    sample_text = "tensors l0.q and l0.gate of the 154 (15,728,640 of 1,130,364,928 elements) per step, fwd+bwd"
+    sample_text = ("tensors l0.q and l0.gate of the 154 (15,728,640 of 1,130,364,928 elements), one forward + backward pass "
+                   "(one step counter of the ten) per step")
     line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16 storage, f32 arithmetic (f64 gradient sum)", "data": "synthetic",
@@ -183,25 +198,78 @@ def run_reference(args, rank: int, world: int):
     print(json.dumps(line), flush=True)
 
 
-def cpu_baseline(specs):
-    """Oracle timed on the host cores: three Llama blocks, forward + backward, one thread."""
+# Instructions the backward kernel k_flat<bwd> executes per 8-element vector and thread, by kind: the Philox4x32-10 and
+# decode counts follow from the source (18 multiplies 32x32->64 and 19 XORs after hoisting; 13 logic operations, 1 right
+# and 6 left shifts for the gradient decode; 8 mixed-precision FMAs), `other` is what ncu counts beyond them
+# (sm__inst_executed_pipe_alu minus the above: index arithmetic, predicates, the tile lookup), see profiles/.
+BWD_INSTRUCTIONS_PER_VECTOR = {"mul_wide": 18, "xor3": 19, "logic": 14, "shl": 6, "fma_bf16": 8, "other_alu": 4}
+
+
+def arithmetic_budget(gws, dev):
+    """Cost of each instruction kind on this chip (gws_issue_probe, cycles per warp instruction and SM sub-partition,
+    from an additive fit that the mixed probes confirm), the cycles per 8-element vector they add up to for the backward
+    pass, and the element rate that budget allows at the measured SM clock."""
+    sink = torch.zeros(8, dtype=torch.int32, device=dev)
+
+    clock = {}
+
+    def cycles(mix, iterations):
+        steps, _ = gws.issue_probe_mix(mix)
+        for _ in range(2):
+            blocks, sms = gws.issue_probe(mix, iterations, sink)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(5):
+            gws.issue_probe(mix, iterations, sink)
+        b.record()
+        torch.cuda.synchronize()
+        # the SM clock comes from the first (longest) probe: cycle counter over nanosecond timer of one of its warps
+        ghz = clock.setdefault("ghz", int(sink[0].item()) / max(int(sink[1].item()), 1))
+        warp_steps = blocks * 8 / (sms * 4) * iterations * steps
+        return a.elapsed_time(b) / 5 * 1e-3 * ghz * 1e9 / warp_steps, ghz, sms
+
+    c_round, ghz, sms = cycles(0, 1024)
+    c_logic = cycles(10, 1024)[0]
+    c_round_2logic = cycles(2, 1024)[0]
+    c_fma = (cycles(8, 1024)[0] - c_round) / 2.0     # the cost of an FMA next to integer work, which is how the pass runs it
+    c_add = (cycles(9, 1024)[0] - c_round) / 2.0
+    c_mul = (c_round - 2.0 * c_logic) / 2.0          # additive: a round is 2 multiplies + 2 XORs
+    n = BWD_INSTRUCTIONS_PER_VECTOR
+    terms = {"mul_wide": n["mul_wide"] * c_mul, "xor3": n["xor3"] * c_logic, "logic": n["logic"] * c_logic,
+             "shl": n["shl"] * c_add, "fma_bf16": n["fma_bf16"] * c_fma, "other_alu": n["other_alu"] * c_logic}
+    budget = sum(terms.values())
+    body = cycles(107, 2048)[0]
+    rate = lambda cyc: sms * 4 * ghz * 1e9 / cyc * 32 * 8 / 1e9            # Gelem/s at `cyc` cycles per warp-vector
+    return {"cycles_per_warp_instruction": {"philox_round_2mul_2xor": c_round, "logic_op": c_logic, "mul_wide_from_round": c_mul,
+                                            "fma_f32_bf16_beside_a_round": c_fma, "integer_add_beside_a_round": c_add,
+                                            "philox_round_plus_2_logic_ops": c_round_2logic,
+                                            "additive_prediction_of_that": c_round + 2.0 * c_logic},
+            "bwd_instructions_per_vector": n, "bwd_cycles_per_vector_terms": terms, "bwd_cycles_per_vector_budget": budget,
+            "bwd_cycles_per_vector_arithmetic_only_measured": body, "sm_clock_ghz": ghz, "sms": sms,
+            "bwd_ceiling_gelem_per_s": rate(budget),
+            "bwd_arithmetic_only_gelem_per_s": rate(body),
+            "bwd_ceiling_is": "sum over instruction kinds of (instructions per 8-element vector) x (measured cycles per warp "
+                              "instruction), at the SM clock the probes measured"}
+
+
+def cpu_baseline(specs, descs, W, BT, G):
+    """The oracle, as it stands, on one full forward + backward pass of the whole weight set (one step counter):
+    one single-threaded oracle process per host core, each with its own tensors (oracle/pool.py)."""
     import numpy as np
-    from oracle import gws_oracle as orc
-    from paper_2505_11170_b200 import synthetic as syn
-    as_bits = lambda t: t.view(torch.int16).numpy().view(np.uint16)
-    idx = list(range(0, 14))             # blocks 0 and 1
-    elems, t = 0, 0.0
-    for i in idx:
-        s = specs[i]
-        w, bt, g = as_bits(syn.weights(s, i)), syn.bitwidths(s, i).numpy(), as_bits(syn.upstream_grad(s, i))
-        t0 = time.perf_counter()
-        _, sc = orc.sample_fwd(w, bt, s.rows, s.cols, 1, s.group_cols, seed=syn.layer_seed(0, i), step=0)
-        orc.sample_bwd(g, sc, s.rows, s.cols, 1, s.group_cols, seed=syn.layer_seed(0, i), step=0)
-        t += time.perf_counter() - t0
-        elems += s.numel
-    return {"value": elems * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM) / t / 1e9, "unit": "GB/s", "cores": 1,
+    from oracle.pool import OraclePool
+    as_bits = lambda t: t.cpu().view(torch.int16).numpy().view(np.uint16)
+    tasks = [dict(rows=s.rows, cols=s.cols, group_rows=1, group_cols=s.group_cols, seed=descs[i].seed, step=0, w=as_bits(W[i]),
+                  bt=BT[i].cpu().numpy(), g=as_bits(G[i])) for i, s in enumerate(specs)]
+    with OraclePool() as pool:
+        res = pool.run(tasks, keep_outputs=False)
+    elems, t = res["elements"], res["seconds"]
+    return {"value": elems * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM) / t / 1e9, "unit": "GB/s", "cores": res["processes"],
             "kind": "oracle", "gelem_per_s": elems / t / 1e9, "seconds": t, "host_cores": os.cpu_count(),
-            "sample": "blocks 0-1 of 22 (14 tensors, 102,760,448 elements), one forward + backward step"}
+            "processes": res["processes"], "threads_per_process": 1,
+            "single_thread_gelem_per_s": elems / res["seconds_in_calls"] / 1e9,
+            "sample": "the whole set: %d tensors, %d elements, one forward + backward pass (one step counter of the ten)"
+                      % (len(specs), elems)}
 
 
 def main():
@@ -214,11 +282,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the side measurements (per-layer launches, copy mode, ALU ceiling)")
+    ap.add_argument("--no-sustain", action="store_true", help="do not extend the launch stream beyond --steps (profiler runs)")
     ap.add_argument("--source-hash", action="store_true", help="print the hash an ncu summary records with its counters")
     args = ap.parse_args()
     if args.impl == "ours":
-        args.steps = 100 if args.steps is None else args.steps            # ~0.15 s of device time at N = 1
-        args.warmup = 5 if args.warmup is None else max(args.warmup, 3)
+        args.steps = 100 if args.steps is None else args.steps            # ~1.3 s of device time at N = 1
+        args.warmup = 3 if args.warmup is None else max(args.warmup, 3)
     else:
         args.steps = 3 if args.steps is None else args.steps              # ~2.4 s of CPU time per step
         args.warmup = 1 if args.warmup is None else args.warmup
@@ -265,38 +334,74 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    step_no = 0
+    def one_step(counter0, events=None):
+        """The ten step counters of one step; with `events`, an event after every launch."""
+        for j in range(PASSES_PER_STEP):
+            if events is not None:
+                e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                e[0].record(stream)
+            plan.sample_fwd_multi(counter0 + j, stream)
+            if events is not None:
+                e[1].record(stream)
+            plan.sample_bwd_multi(counter0 + j, stream)
+            if events is not None:
+                e[2].record(stream)
+                events.append(e)
+
+    counter = 0
     for _ in range(args.warmup):
-        plan.sample_fwd_multi(step_no)
-        plan.sample_bwd_multi(step_no)
-        step_no += 1
+        one_step(counter)
+        counter += PASSES_PER_STEP
     barrier()
 
-    # ---- device-resident timing: K steps, an event after every launch ----
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    # ---- device-resident timing: K steps, an event after every launch; the same launch stream then runs on until
+    # ---- it has covered SUSTAIN_MS, which is where the sustained roofline fractions come from
+    ev = []
     sampler = ClockSampler(local_rank) if rank == 0 else None
     launches0 = gws.launch_count()
     barrier()
     t_wall0 = time.time()
     for k in range(args.steps):
-        ev[k][0].record(stream)
-        plan.sample_fwd_multi(step_no, stream)
-        ev[k][1].record(stream)
-        plan.sample_bwd_multi(step_no, stream)
-        ev[k][2].record(stream)
-        step_no += 1
-    barrier()
-    t_wall1 = time.time()
+        one_step(counter, ev)
+        counter += PASSES_PER_STEP
+    n_timed = len(ev)
     launches = gws.launch_count() - launches0
-    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-    total_ms = ev[0][0].elapsed_time(ev[-1][2])
-    fwd_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
-    bwd_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
-    total_ms, fwd_ms, bwd_ms = max_over_ranks([total_ms, fwd_ms, bwd_ms], dist, dev)
+    while True:      # extension: whole steps, decided from the measured time of what has run so far
+        ev[-1][2].synchronize()
+        done_ms = ev[0][0].elapsed_time(ev[-1][2])
+        if done_ms >= SUSTAIN_MS or args.no_sustain:
+            break
+        per_step = done_ms / (len(ev) / PASSES_PER_STEP)
+        for _ in range(max(1, int((SUSTAIN_MS - done_ms) / per_step) + 1)):
+            one_step(counter, ev)
+            counter += PASSES_PER_STEP
+    barrier()
+    if sampler:
+        sampler.stop()
+    total_ms = ev[0][0].elapsed_time(ev[n_timed - 1][2])
+    fwd_all = [e[0].elapsed_time(e[1]) for e in ev]
+    bwd_all = [e[1].elapsed_time(e[2]) for e in ev]
+    offset = [ev[0][0].elapsed_time(e[0]) for e in ev]                   # ms from the start of the timed region
+    mean = lambda xs: sum(xs) / max(len(xs), 1)
+    sustained = [i for i, t in enumerate(offset) if t >= 300.0] or list(range(len(ev)))
+    burst = list(range(min(BURST_LAUNCHES, len(ev))))
+    fwd_ms, bwd_ms = mean(fwd_all[:n_timed]), mean(bwd_all[:n_timed])
+    fwd_burst, bwd_burst = mean([fwd_all[i] for i in burst]), mean([bwd_all[i] for i in burst])
+    fwd_sus, bwd_sus = mean([fwd_all[i] for i in sustained]), mean([bwd_all[i] for i in sustained])
+    total_ms, fwd_ms, bwd_ms, fwd_burst, bwd_burst, fwd_sus, bwd_sus = max_over_ranks(
+        [total_ms, fwd_ms, bwd_ms, fwd_burst, bwd_burst, fwd_sus, bwd_sus], dist, dev)
+    clocks = None
+    if sampler:
+        wall = lambda i, j=0: t_wall0 + ev[0][0].elapsed_time(ev[i][j]) * 1e-3
+        clocks = sampler.window(t_wall0, wall(n_timed - 1, 2))
+        clocks["burst"] = sampler.window(t_wall0, wall(burst[-1], 2))
+        clocks["sustained"] = sampler.window(wall(sustained[0]), wall(sustained[-1], 2))
+        clocks["sustained"]["device_ms"] = ev[sustained[0]][0].elapsed_time(ev[sustained[-1]][2])
     ms_per_step = total_ms / args.steps
-    bytes_per_step = n_elem * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM)
+    bytes_per_pass = n_elem * (FWD_BYTES_PER_ELEM + BWD_BYTES_PER_ELEM)
+    bytes_per_step = bytes_per_pass * PASSES_PER_STEP
     value = whole_job_throughput(bytes_per_step, world, ms_per_step) / 1e9
-    gelem = whole_job_throughput(n_elem, world, ms_per_step) / 1e9
+    gelem = whole_job_throughput(n_elem * PASSES_PER_STEP, world, ms_per_step) / 1e9
 
     # ---- end to end through the host-buffer entry point: pinned host tensors in, results out ----
     e2e = None
@@ -324,17 +429,18 @@ def main():
 
         host_step(0)
         barrier()
-        e2e_steps = 3
+        e2e_steps = 1                                      # one step = ten passes, about a second behind the host link
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for k in range(e2e_steps):
+        for k in range(e2e_steps * PASSES_PER_STEP):
             host_step(1 + k)
         e1.record(stream)
         barrier()
         e2e_ms = max_over_ranks([e0.elapsed_time(e1) / e2e_steps], dist, dev)[0]
         n_groups = sum(s.n_groups for s in specs)
         e2e = {"value": whole_job_throughput(bytes_per_step, world, e2e_ms) / 1e9, "unit": "GB/s",
-               "h2d_bytes_per_step": int(n_elem * 4 + n_groups * 4), "d2h_bytes_per_step": int(n_elem * 2 + n_groups * 8),
+               "h2d_bytes_per_step": int(n_elem * 4 + n_groups * 4) * PASSES_PER_STEP,
+               "d2h_bytes_per_step": int(n_elem * 2 + n_groups * 8) * PASSES_PER_STEP,
                "ms_per_step": float(e2e_ms), "steps": e2e_steps,
                "note": "gws_sample_step_host per tensor on seven streams; pinned host buffers of one transformer block reused "
                        "for all 22; bound by the host link (6.9 GB cross it per step)"}
@@ -364,9 +470,7 @@ def main():
         copy_plan = gws.MultiPlan(descs, scale=SC, grad_w_hat=G, grad_w=GW, grad_bt=GBT)
         bwd_copy_ms = timed(lambda k: copy_plan.sample_bwd_multi(k), 10)
         del copy_plan, GW
-        probe_desc = Desc.make(n_elem // 2048, 2048, 1, 128, seed=1)
-        sink = gws.noise_alu_probe(probe_desc)
-        probe_ms = timed(lambda k: gws.noise_alu_probe(probe_desc.with_step(k), sink), 10)
+        alu = arithmetic_budget(gws, dev)
         # one rank's share of the same set with every tensor cut into 6 flat shards (6 does not divide the tensors, so
         # every shard has a partial group at each end): the local work of a sharded step, without the two small
         # all-reduces a real job adds
@@ -401,13 +505,11 @@ def main():
                                         "fwd_GB/s": sh_elems * FWD_BYTES_PER_ELEM / (sh_fwd_ms * 1e-3) / 1e9,
                                         "bwd_GB/s": sh_elems * BWD_BYTES_PER_ELEM / (sh_bwd_ms * 1e-3) / 1e9,
                                         "note": "each pass reads %.2f GB, more than L2; a real job adds two all-reduces of %d floats" % (sh_elems * 2 / 1e9, len(specs) * (shard_world + 1))},
-            "per_layer_launches": {"ms_per_step": per_layer_ms, "launches_per_step": 2 * len(specs),
-                                   "GB/s": bytes_per_step / (per_layer_ms * 1e-3) / 1e9},
+            "per_layer_launches": {"ms_per_pass": per_layer_ms, "launches_per_pass": 2 * len(specs),
+                                   "GB/s": bytes_per_pass / (per_layer_ms * 1e-3) / 1e9},
             "bwd_with_grad_w_copy": {"ms_per_launch": bwd_copy_ms, "GB/s": n_elem * (4 + 8 / 128) / (bwd_copy_ms * 1e-3) / 1e9,
                                      "bytes_per_element": 4 + 8 / 128},
-            "noise_arithmetic_ceiling": {"gelem_per_s": n_elem / (probe_ms * 1e-3) / 1e9, "ms": probe_ms,
-                                         "note": "Philox + decode with no memory traffic (gws_noise_alu_probe): "
-                                                 "what the backward pass (2.06 B/element) cannot exceed"},
+            "arithmetic_budget": alu,
         }
 
     if rank != 0:
@@ -419,34 +521,43 @@ def main():
     traffic = ncu_traffic()
     fwd_bytes = n_elem * FWD_BYTES_PER_ELEM
     bwd_bytes = n_elem * BWD_BYTES_PER_ELEM
-    fwd_gbs = fwd_bytes / (fwd_ms * 1e-3) / 1e9
-    bwd_gbs = bwd_bytes / (bwd_ms * 1e-3) / 1e9
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
+    fwd_gbs, bwd_gbs = gbs(fwd_bytes, fwd_sus), gbs(bwd_bytes, bwd_sus)
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
         "config": {"workload": WORKLOAD, "tensors": len(specs), "elements": n_elem, "group": "1x128",
                    "bits": "uniform integers 4..9", "passes": "forward + backward (identity grad_w), one launch each",
+                   "step": "%d consecutive step counters = %d forward + %d backward launches" % (PASSES_PER_STEP, PASSES_PER_STEP, PASSES_PER_STEP),
                    "l2": "inputs larger than L2: each pass streams %.2f GB" % (n_elem * 2 / 1e9),
                    "multi_gpu": "replicas only (no exchange step in the path)"},
         "gelem_per_s": gelem, "hbm_frac": value / world / peak, "hbm_frac_of_nominal_8000": value / world / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "k_flat<fwd> (gws_sample_fwd_multi)", "achieved": fwd_gbs, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": fwd_gbs / peak, "frac_of_nominal_8000": fwd_gbs / NOMINAL_HBM_GBS,
-                     "ms_per_launch": fwd_ms,
+                     "frac_is": "sustained: launches after the first 0.3 s of a launch stream of at least %.1f s" % (SUSTAIN_MS * 1e-3),
+                     "ms_per_launch": fwd_sus, "frac_burst": gbs(fwd_bytes, fwd_burst) / peak, "ms_per_launch_burst": fwd_burst,
+                     "frac_timed_steps": gbs(fwd_bytes, fwd_ms) / peak, "ms_per_launch_timed_steps": fwd_ms,
                      "algorithmic_bytes_per_launch": fwd_bytes, "traffic": traffic.get("fwd_bytes_per_launch")},
         "roofline_bwd": {"bound": "hbm", "kernel": "k_flat<bwd> (gws_sample_bwd_multi)", "achieved": bwd_gbs, "peak": peak,
-                         "unit": "GB/s", "frac": bwd_gbs / peak, "ms_per_launch": bwd_ms,
+                         "unit": "GB/s", "frac": bwd_gbs / peak, "ms_per_launch": bwd_sus,
+                         "frac_burst": gbs(bwd_bytes, bwd_burst) / peak, "ms_per_launch_burst": bwd_burst,
+                         "frac_timed_steps": gbs(bwd_bytes, bwd_ms) / peak, "ms_per_launch_timed_steps": bwd_ms,
                          "algorithmic_bytes_per_launch": bwd_bytes, "traffic": traffic.get("bwd_bytes_per_launch")},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
     }
     if extras is not None:
         line["extras"] = extras
-        # the backward pass is bound by random-bit generation, not by HBM: also report it against that measured ceiling
-        ceiling = extras["noise_arithmetic_ceiling"]["gelem_per_s"]
+        # the backward pass is bound by integer instruction issue, not by HBM: also report it against the ceiling that
+        # follows from the instructions it executes per 8 elements and what each kind costs on this chip
+        alu = extras["arithmetic_budget"]
+        ceiling = alu["bwd_ceiling_gelem_per_s"]
         line["roofline_bwd"].update({"arithmetic_ceiling_gelem_per_s": ceiling,
-                                     "frac_of_arithmetic_ceiling": n_elem / (bwd_ms * 1e-3) / 1e9 / ceiling})
+                                     "frac_of_arithmetic_ceiling": n_elem / (bwd_sus * 1e-3) / 1e9 / ceiling,
+                                     "frac_of_arithmetic_ceiling_burst": n_elem / (bwd_burst * 1e-3) / 1e9 / ceiling,
+                                     "arithmetic_ceiling_is": alu["bwd_ceiling_is"]})
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(syn.llama2_1b())
+        line["cpu_baseline"] = cpu_baseline(specs, descs, W, BT, G)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

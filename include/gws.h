@@ -420,6 +420,22 @@ int gws_philox_words(uint64_t seed, uint64_t step, uint64_t first_vec, int64_t n
 int gws_noise_alu_probe(const gws_desc* desc, uint32_t* sink, void* stream);
 int64_t gws_noise_alu_probe_words(const gws_desc* desc);
 
+/* Issue cost of the instruction kinds the passes are made of (Section 3.4's generation is integer work: per 8
+ * elements Philox4x32-10 takes 18 multiplies 32 x 32 -> 64 and 19 three-input XORs once its launch-uniform part is
+ * hoisted, the AND / OR decode of Eq. 10 another 14 logic operations).  gws_issue_probe runs `iterations` x 32 steps
+ * per thread of instruction mix `mix` on 64 warps per SM with no memory traffic; the caller times the launch.
+ *   gws_issue_probe_mix(mix, counts7)  host only: instructions per step {multiply 32x32->64, XOR fed by it, other
+ *       logic, FP32 FMA, FP32 += BF16*BF16 FMA, integer add, byte permute}; returns the steps per thread and
+ *       iteration (32), or GWS_ERR_UNSUPPORTED for an unknown mix.  mix = 100 + pieces runs the arithmetic of a pass
+ *       instead (pieces 1: Philox; 3: + gradient decode; 7: + the gradient sum's FMAs, i.e. the backward pass; 9:
+ *       Philox + forward decode + Eq. 3's add and BF16 packing); `iterations` then counts 8-element vectors per
+ *       thread (a multiple of 4) and the return value is 1.
+ *   sink        device, u32 [8]: [0] SM cycles and [1] nanoseconds one warp spent in the loop (their ratio is the SM
+ *               clock in GHz during the probe)
+ *   host_info2  host, int32 [2]: thread blocks launched (of 256 threads), SMs of the device */
+int gws_issue_probe_mix(int mix, int32_t* counts7);
+int gws_issue_probe(int mix, int iterations, uint32_t* sink, int32_t* host_info2, void* stream);
+
 /* Host-side evaluation of the same inline decode / Philox code the kernels use (no GPU needed):
  * r8 receives R for the 8 fields of the 4 words; packed receives the nibble word. */
 void gws_host_decode8(const uint32_t* words4, int8_t* r8, uint32_t* packed);

@@ -92,6 +92,8 @@ _SIGNATURES = {
     "gws_noise_alu_probe": (c_int, [POINTER(Desc), c_void_p, c_void_p]),
     "gws_noise_alu_probe_words": (c_int64, [POINTER(Desc)]),
     "gws_host_decode8": (None, [POINTER(c_uint32), POINTER(c_int8), POINTER(c_uint32)]),
+    "gws_issue_probe_mix": (c_int, [c_int, POINTER(c_int32)]),
+    "gws_issue_probe": (c_int, [c_int, c_int, c_void_p, POINTER(c_int32), c_void_p]),
     "gws_host_decode8_pairs": (None, [POINTER(c_uint32), POINTER(c_uint32), POINTER(c_uint32)]),
     "gws_host_philox": (None, [c_uint64, c_uint64, c_uint64, POINTER(c_uint32)]),
     "gws_selfcheck_enabled": (c_int, []),
@@ -455,6 +457,23 @@ def host_decode8(words4: Sequence[int]):
     p = c_uint32(0)
     load_library().gws_host_decode8(w, r, ctypes.byref(p))
     return list(r), int(p.value)
+
+
+def issue_probe_mix(mix: int):
+    """(steps per thread and iteration, instruction counts per step) of an instruction mix of :func:`issue_probe`."""
+    counts = (c_int32 * 7)()
+    steps = int(load_library().gws_issue_probe_mix(mix, counts))
+    if steps < 0:
+        raise GwsError(steps)
+    return steps, list(counts)
+
+
+def issue_probe(mix: int, iterations: int, sink: torch.Tensor, stream=None):
+    """Launches one issue-cost probe; returns (thread blocks launched, SMs).  ``sink``: int32 [8] on the device."""
+    _require_cuda(sink)
+    info = (c_int32 * 2)()
+    _check(load_library().gws_issue_probe(mix, iterations, _ptr(sink), info, _stream(stream)))
+    return int(info[0]), int(info[1])
 
 
 def host_decode8_pairs(words4: Sequence[int]):

@@ -15,6 +15,7 @@
 #define GWS_FLAT_CPT_BWD 2
 #endif
 #include "gws_kernels.cuh"
+#include "gws_probe.cuh"
 
 namespace {
 
@@ -612,6 +613,92 @@ int gws_noise_alu_probe(const gws_desc* desc, uint32_t* sink, void* stream) {
       sink, n_words, desc->elem_offset >> 3, static_cast<uint32_t>(desc->seed), static_cast<uint32_t>(desc->seed >> 32),
       static_cast<uint32_t>(desc->step), static_cast<uint32_t>(desc->step >> 32));
   return check_launch("noise arithmetic probe");
+}
+
+// Instruction mixes of gws_issue_probe: {multiplies 32x32->64, XORs fed by them, other three-input logic operations,
+// FP32 FMAs, mixed-precision FMAs, integer additions, byte permutes} per step of one chain.
+static const int32_t kIssueMixes[][7] = {
+    {2, 2, 0, 0, 0, 0, 0},  //  0  one Philox round
+    {2, 2, 1, 0, 0, 0, 0},  //  1  ... + 1 logic operation
+    {2, 2, 2, 0, 0, 0, 0},  //  2
+    {2, 2, 4, 0, 0, 0, 0},  //  3
+    {2, 2, 0, 1, 0, 0, 0},  //  4  ... + 1 FP32 FMA
+    {2, 2, 0, 2, 0, 0, 0},  //  5
+    {2, 2, 0, 4, 0, 0, 0},  //  6
+    {2, 2, 0, 0, 1, 0, 0},  //  7  ... + 1 mixed-precision FMA
+    {2, 2, 0, 0, 2, 0, 0},  //  8
+    {2, 2, 0, 0, 0, 2, 0},  //  9  ... + 2 integer additions
+    {0, 0, 1, 0, 0, 0, 0},  // 10  logic alone
+    {0, 0, 0, 1, 0, 0, 0},  // 11  FP32 FMA alone
+    {0, 0, 0, 0, 1, 0, 0},  // 12  mixed-precision FMA alone
+    {0, 0, 0, 0, 0, 1, 0},  // 13  integer addition alone
+    {0, 0, 0, 0, 0, 0, 1},  // 14  byte permute alone
+    {0, 0, 1, 1, 0, 0, 0},  // 15  logic + FP32 FMA
+    {0, 0, 1, 0, 1, 0, 0},  // 16  logic + mixed-precision FMA
+    {1, 1, 0, 0, 0, 0, 0},  // 17  half a round
+    {1, 1, 1, 0, 0, 0, 0},  // 18
+    {1, 1, 2, 0, 0, 0, 0},  // 19
+};
+constexpr int kIssueMixCount = static_cast<int>(sizeof(kIssueMixes) / sizeof(kIssueMixes[0]));
+constexpr int kBodyProbeBase = 100;   // mix = 100 + pieces: the arithmetic of a pass without its memory traffic
+
+int gws_issue_probe_mix(int mix, int32_t* counts7) {
+  if (counts7 == nullptr) return GWS_ERR_NULL;
+  if (mix >= 0 && mix < kIssueMixCount) {
+    for (int k = 0; k < 7; ++k) counts7[k] = kIssueMixes[mix][k];
+    return 32;   // steps per thread and iteration: 4 chains x 8
+  }
+  const int pieces = mix - kBodyProbeBase;
+  if (pieces == 1 || pieces == 3 || pieces == 7 || pieces == 9) {
+    for (int k = 0; k < 7; ++k) counts7[k] = 0;
+    return 1;    // "iterations" counts 8-element vectors per thread
+  }
+  return GWS_ERR_UNSUPPORTED;
+}
+
+int gws_issue_probe(int mix, int iterations, uint32_t* sink, int32_t* host_info2, void* stream) {
+  int32_t counts[7];
+  const int steps = gws_issue_probe_mix(mix, counts);
+  if (steps < 0) return steps;
+  if (iterations <= 0 || iterations > (1 << 20)) return GWS_ERR_SHAPE;
+  if (sink == nullptr || host_info2 == nullptr) return GWS_ERR_NULL;
+  if (!aligned(sink, 4)) return GWS_ERR_ALIGN;
+  int dev = 0, sms = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err == cudaSuccess) err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) return cuda_fail(err, "device query");
+  const unsigned blocks = static_cast<unsigned>(sms) * 8u;   // 2048 threads per SM: 16 warps on every sub-partition
+  host_info2[0] = static_cast<int32_t>(blocks);
+  host_info2[1] = sms;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const uint32_t k0 = 0x1234567u, k1 = 0x89ABCDEFu;
+  const float f0 = 1.0001f;
+#define GWS_ISSUE_CASE(ID, NW, K, F, B, I, P) \
+  case ID: gws::k_issue_probe<NW, K, F, B, I, P><<<blocks, 256, 0, s>>>(sink, k0, k1, f0, iterations); break;
+  if (mix < kBodyProbeBase) {
+    switch (mix) {
+      GWS_ISSUE_CASE(0, 2, 0, 0, 0, 0, 0) GWS_ISSUE_CASE(1, 2, 1, 0, 0, 0, 0) GWS_ISSUE_CASE(2, 2, 2, 0, 0, 0, 0)
+      GWS_ISSUE_CASE(3, 2, 4, 0, 0, 0, 0) GWS_ISSUE_CASE(4, 2, 0, 1, 0, 0, 0) GWS_ISSUE_CASE(5, 2, 0, 2, 0, 0, 0)
+      GWS_ISSUE_CASE(6, 2, 0, 4, 0, 0, 0) GWS_ISSUE_CASE(7, 2, 0, 0, 1, 0, 0) GWS_ISSUE_CASE(8, 2, 0, 0, 2, 0, 0)
+      GWS_ISSUE_CASE(9, 2, 0, 0, 0, 2, 0) GWS_ISSUE_CASE(10, 0, 1, 0, 0, 0, 0) GWS_ISSUE_CASE(11, 0, 0, 1, 0, 0, 0)
+      GWS_ISSUE_CASE(12, 0, 0, 0, 1, 0, 0) GWS_ISSUE_CASE(13, 0, 0, 0, 0, 1, 0) GWS_ISSUE_CASE(14, 0, 0, 0, 0, 0, 1)
+      GWS_ISSUE_CASE(15, 0, 1, 1, 0, 0, 0) GWS_ISSUE_CASE(16, 0, 1, 0, 1, 0, 0) GWS_ISSUE_CASE(17, 1, 0, 0, 0, 0, 0)
+      GWS_ISSUE_CASE(18, 1, 1, 0, 0, 0, 0) GWS_ISSUE_CASE(19, 1, 2, 0, 0, 0, 0)
+      default: return GWS_ERR_UNSUPPORTED;
+    }
+  } else {
+    if (iterations % 4 != 0) return GWS_ERR_SHAPE;
+    const gws::PhiloxPre pre = gws::philox_pre(0u, 3u, 0u, k0, k1);
+    switch (mix - kBodyProbeBase) {
+      case 1: gws::k_body_probe<1><<<blocks, 256, 0, s>>>(sink, k0, k1, pre, 0x3C003C00u, iterations); break;
+      case 3: gws::k_body_probe<3><<<blocks, 256, 0, s>>>(sink, k0, k1, pre, 0x3C003C00u, iterations); break;
+      case 7: gws::k_body_probe<7><<<blocks, 256, 0, s>>>(sink, k0, k1, pre, 0x3C003C00u, iterations); break;
+      case 9: gws::k_body_probe<9><<<blocks, 256, 0, s>>>(sink, k0, k1, pre, 0x3C003C00u, iterations); break;
+      default: return GWS_ERR_UNSUPPORTED;
+    }
+  }
+#undef GWS_ISSUE_CASE
+  return check_launch("issue probe");
 }
 
 int gws_philox_words(uint64_t seed, uint64_t step, uint64_t first_vec, int64_t n_vec, uint32_t* out4, void* stream) {

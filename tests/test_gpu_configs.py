@@ -1,7 +1,9 @@
 """The benchmark configurations at full size, in the launch configuration the benchmark times
-(one multi-tensor launch per kernel class), against the oracle: completely where the oracle
-finishes in seconds, on sampled tensors / row slices otherwise (every group is independent, and
-a row slice with elem_offset = first_row * cols reproduces the noise stream of the full tensor)."""
+(one multi-tensor launch per kernel class), against the oracle.  Whole weight sets and whole matrices are
+compared element by element and group by group: the oracle runs as one single-threaded process per host
+core over disjoint tensors or row bands (oracle/pool.py; a row band with elem_offset = first_row * cols
+reproduces the noise stream of the full tensor).  Only the 28672 x 8192 matrix of the stress sweep and the
+intermediate step counters of the ten-step run are checked on row slices."""
 import numpy as np
 import pytest
 import torch
@@ -10,6 +12,7 @@ import paper_2505_11170_b200 as gws
 from oracle import gws_oracle as orc
 from paper_2505_11170_b200 import synthetic as syn
 from paper_2505_11170_b200.binding import Desc
+from oracle.pool import OraclePool
 from util import bits_of
 
 pytestmark = pytest.mark.gpu
@@ -40,6 +43,46 @@ def _slice_check(spec, desc_seed, step, w, bt, w_hat, scale, g, gbt, r0, nrows):
         assert np.abs(got - want).max() <= REL * np.abs(want).max() + 1e-45
 
 
+def _bands(rows, want):
+    """Splits `rows` into about `want` bands of whole rows: (first row, number of rows)."""
+    per = max(1, -(-rows // want))
+    return [(r0, min(per, rows - r0)) for r0 in range(0, rows, per)]
+
+
+def _whole_check(pool, specs, seeds, step, W, BT, WH, SC, G, GBT, min_tasks=32):
+    """Every element of w_hat, every scale and every grad_bt of a tensor set against the oracle."""
+    host = lambda t: t.cpu()
+    tasks, where = [], []
+    per_tensor = max(1, min_tasks // len(specs))
+    for i, s in enumerate(specs):
+        assert s.group_rows == 1
+        gc = s.group_cols or s.cols
+        gpr = s.cols // gc
+        w, bt, g = bits_of(host(W[i])).reshape(s.rows, s.cols), host(BT[i]).numpy(), bits_of(host(G[i])).reshape(s.rows, s.cols)
+        for r0, nr in _bands(s.rows, per_tensor):
+            tasks.append(dict(rows=nr, cols=s.cols, group_rows=1, group_cols=s.group_cols, seed=seeds[i], step=step,
+                              elem_offset=r0 * s.cols, w=w[r0:r0 + nr], bt=bt[r0 * gpr:(r0 + nr) * gpr], g=g[r0:r0 + nr]))
+            where.append((i, r0, nr, gpr))
+    res = pool.run(tasks, bound=True)
+    got_hat = [bits_of(host(t)).reshape(s.rows, s.cols) for t, s in zip(WH, specs)]
+    got_sc = [host(t).numpy() for t in SC]
+    got_gbt = [host(t).numpy().astype(np.float64) for t in GBT]
+    worst = {}
+    for k, (i, r0, nr, gpr) in enumerate(where):
+        name = specs[i].name
+        assert np.array_equal(got_hat[i][r0:r0 + nr].ravel(), np.asarray(res["w_hat"][k]).ravel()), (name, step, r0)
+        gsl = slice(r0 * gpr, (r0 + nr) * gpr)
+        assert np.array_equal(got_sc[i][gsl].view(np.uint32), np.asarray(res["scale"][k]).view(np.uint32)), (name, step, r0)
+        want = np.asarray(res["grad_bt"][k]).astype(np.float64)
+        err = np.abs(got_gbt[i][gsl] - want)
+        assert (err <= REL * np.asarray(res["grad_bt_bound"][k]) + 1e-45).all(), (name, step, r0)
+        e, m = worst.get(i, (0.0, 0.0))
+        worst[i] = (max(e, float(err.max())), max(m, float(np.abs(want).max())))
+    for i, (e, m) in worst.items():
+        assert e <= REL * m + 1e-45, (specs[i].name, step)
+    return res["elements"]
+
+
 @pytest.mark.parametrize("literal", [False, True])
 def test_config1_gpt2_single_mlp_weight(literal):
     spec = syn.gpt2_124m_single(literal)[0]
@@ -65,7 +108,7 @@ def _device_set(specs, device=DEV):
     return descs, W, BT, G, WH, SC, GBT
 
 
-def test_config2_gpt2_all_linear_weights_forward_backward():
+def test_config2_gpt2_all_linear_weights_forward_backward_whole_set():
     specs = syn.gpt2_124m_all()
     assert syn.total_elements(specs) == 84934656 and sum(s.n_groups for s in specs) == 82944
     descs, W, BT, G, WH, SC, GBT = _device_set(specs)
@@ -74,42 +117,32 @@ def test_config2_gpt2_all_linear_weights_forward_backward():
     plan.sample_fwd_multi(0)
     plan.sample_bwd_multi(0)
     torch.cuda.synchronize()
-    # whole tensors of block 0 and block 11, row slices of the rest
-    for i, s in enumerate(specs):
-        if i < 4 or i >= 44:
-            _slice_check(s, descs[i].seed, 0, W[i], BT[i], WH[i], SC[i], G[i], GBT[i], 0, s.rows)
-        else:
-            r0 = (i * 97) % (s.rows - 16)
-            _slice_check(s, descs[i].seed, 0, W[i], BT[i], WH[i], SC[i], G[i], GBT[i], r0, 16)
+    with OraclePool() as pool:
+        assert _whole_check(pool, specs, [d.seed for d in descs], 0, W, BT, WH, SC, G, GBT) == 84934656
 
 
-def test_config3_llama2_1b_ten_steps():
+def test_config3_llama2_1b_ten_steps_whole_set_at_steps_0_and_9():
     specs = syn.llama2_1b()
     assert syn.total_elements(specs) == 1130364928 and sum(s.n_groups for s in specs) == 8830976
     descs, W, BT, G, WH, SC, GBT = _device_set(specs)
     plan = gws.MultiPlan(descs, w=W, bt=BT, w_hat=WH, scale=SC, grad_w_hat=G, grad_bt=GBT)
     assert plan.launches_per_pass == 1
     rng = np.random.default_rng(3)
+    seeds = [d.seed for d in descs]
     for step in range(10):
         plan.sample_fwd_multi(step)
         plan.sample_bwd_multi(step)
         torch.cuda.synchronize()
         if step in (0, 9):
-            # two whole tensors (one square, one wide) plus a slice of every tensor
-            for i in (0, 6) if step == 0 else (4, 153):
-                _slice_check(specs[i], descs[i].seed, step, W[i], BT[i], WH[i], SC[i], G[i], GBT[i], 0, specs[i].rows)
-            for i, s in enumerate(specs):
-                r0 = int(rng.integers(0, s.rows - 8))
-                _slice_check(s, descs[i].seed, step, W[i], BT[i], WH[i], SC[i], G[i], GBT[i], r0, 8)
+            # all 1,130,364,928 elements and all 8,830,976 groups
+            with OraclePool() as pool:
+                assert _whole_check(pool, specs, seeds, step, W, BT, WH, SC, G, GBT) == 1130364928
         else:
             for i in rng.choice(len(specs), 6, replace=False):
                 s = specs[int(i)]
                 r0 = int(rng.integers(0, s.rows - 8))
                 _slice_check(s, descs[int(i)].seed, step, W[int(i)], BT[int(i)], WH[int(i)], SC[int(i)], G[int(i)],
                              GBT[int(i)], r0, 8)
-    # the last rows (tail tile) of the last tensor
-    s = specs[-1]
-    _slice_check(s, descs[-1].seed, 9, W[-1], BT[-1], WH[-1], SC[-1], G[-1], GBT[-1], s.rows - 8, 8)
 
 
 @pytest.mark.parametrize("shape", syn.STRESS_SHAPES)
@@ -131,9 +164,14 @@ def test_config4_stress_sweep(shape):
                 _, sc = gws.sample_fwd(d, w, bt, w_hat=w_hat)
                 _, gbt = gws.sample_bwd(d, g, sc)
                 torch.cuda.synchronize()
-                nrows = 8 if rows * cols > (1 << 25) else 32
-                for r0 in (0, rows - nrows, int(rng.integers(0, rows - nrows))):
-                    _slice_check(spec, d.seed, case, w, bt, w_hat, sc, g, gbt, r0, nrows)
+                if rows * cols <= (1 << 26):
+                    # 4096^2 and 8192^2: the whole matrix, cut into row bands for the oracle processes
+                    with OraclePool() as pool:
+                        assert _whole_check(pool, [spec], [d.seed], case, [w], [bt], [w_hat], [sc], [g], [gbt]) == rows * cols
+                else:
+                    nrows = 8
+                    for r0 in (0, rows - nrows, int(rng.integers(0, rows - nrows))):
+                        _slice_check(spec, d.seed, case, w, bt, w_hat, sc, g, gbt, r0, nrows)
                 # the outliers are there and the absmax sees them
                 am = gws.group_absmax(d, w)
                 assert float(am.max()) >= 7.9 * sigma

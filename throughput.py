@@ -1,6 +1,6 @@
 """Throughput of the sampling pass on the other workload shapes of the paper (one JSON line each).
 
-    python -m paper_2505_11170_b200.throughput [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [--reps N] [--blocks B]
+    python throughput.py [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [issue] [--reps N] [--blocks B]
 
 gpt2         all GPT2-124M linear weights, one group per row (and the same set with groups of 128)
 gpt2_single  one GPT2-124M MLP weight, both orientations
@@ -9,6 +9,8 @@ square       Llama2-1B-shaped blocks with the paper's 32 x 32 groups (Eq. 3, b_l
 llama        the Llama2-1B-shaped set with groups of 128 (the benchmark's workload; --blocks limits it)
 mx           the same set with w_hat written as MX FP8 / FP6 instead of BF16
 gemm         sampling fused into a tcgen05 GEMM against sampling + library GEMM against the plain library GEMM
+issue        cycles per warp instruction of the instruction kinds the passes are made of, and of the passes' arithmetic
+             without memory traffic (gws_issue_probe): the terms of the arithmetic ceiling of the backward pass
 
 Every timed pass is one multi-tensor launch set over the whole workload, timed with CUDA events on the launching
 stream after three warm-up passes; a 256 MiB buffer is written between passes so that no pass finds its inputs in L2.
@@ -23,11 +25,13 @@ import sys
 
 import torch
 
-from . import binding as gws
-from . import synthetic as syn
-from .binding import Desc
+_ROOT = os.path.dirname(os.path.abspath(__file__))
+if _ROOT not in sys.path:
+    sys.path.insert(0, _ROOT)
 
-_ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+from paper_2505_11170_b200 import binding as gws       # noqa: E402
+from paper_2505_11170_b200 import synthetic as syn     # noqa: E402
+from paper_2505_11170_b200.binding import Desc         # noqa: E402
 
 
 def _peak_gbs() -> float:
@@ -126,6 +130,42 @@ def run_gemm(reps: int, dev) -> dict:
     return line
 
 
+ISSUE_MIXES = list(range(20)) + [101, 103, 107, 109]
+_KINDS = ("mul 32x32->64", "xor3 fed by it", "lop3", "ffma", "fma.f32.bf16", "iadd", "prmt")
+_BODY = {101: "Philox4x32-10 (hoisted), per 8-element vector", 103: "Philox + gradient decode, per vector",
+         107: "Philox + gradient decode + 8 FMAs = backward arithmetic, per vector",
+         109: "Philox + forward decode + Eq. 3 add + BF16 packing = forward arithmetic, per vector"}
+
+
+def run_issue(reps: int, dev) -> list:
+    """Cycles per step (or per 8-element vector) and SM sub-partition for every mix of gws_issue_probe.  The SM clock is
+    the one the probe measures itself (cycle counter over the nanosecond timer of one warp)."""
+    sink = torch.zeros(8, dtype=torch.int32, device=dev)
+    lines = []
+    ghz = None
+    for mix in ISSUE_MIXES:
+        steps, counts = gws.issue_probe_mix(mix)
+        iterations = 1024 if mix < 100 else 2048
+        for _ in range(3):
+            blocks, sms = gws.issue_probe(mix, iterations, sink)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            gws.issue_probe(mix, iterations, sink)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / reps
+        if ghz is None:      # from the first probe, which runs for more than a millisecond
+            ghz = int(sink[0].item()) / int(sink[1].item())
+        warp_steps = blocks * 8 / (sms * 4) * iterations * steps            # per sub-partition
+        line = {"mix": mix, "what": _BODY.get(mix) or " + ".join(f"{c} {k}" for c, k in zip(counts, _KINDS) if c),
+                "ms": ms, "sm_clock_ghz": ghz, "cycles_per_step_per_subpartition": ms * 1e-3 * ghz * 1e9 / warp_steps}
+        print(json.dumps(line), flush=True)
+        lines.append(line)
+    return lines
+
+
 def main(argv=None) -> None:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("which", nargs="*", default=["gpt2", "stress"])
@@ -154,6 +194,8 @@ def main(argv=None) -> None:
             run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev)
         elif w == "gemm":
             run_gemm(args.reps, dev)
+        elif w == "issue":
+            run_issue(args.reps, dev)
         elif w == "mx":
             for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2, gws.MX_FP8_E3M4):
                 run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev, mx_format=fmt)
