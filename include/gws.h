@@ -229,6 +229,16 @@ int gws_sample_fwd_mx(const gws_desc* desc, int format, const void* w, const flo
  */
 int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y,
                    void* w_hat_out, float* scale_out, int* status, int rows_per_block, void* stream);
+
+/* The same product with every sampled tile of W shared by a cluster of thread blocks (Section 3.5's decision, measured
+ * a second way): `cluster_blocks` (1, 2 or 4) blocks of 256 rows of X each, stacked along M, sample 128 / cluster_blocks
+ * rows of each 128 x 128 tile of W and store them into the shared memory of all blocks of the cluster, so a tile is
+ * sampled once per 256 * cluster_blocks rows of X; the sampling of the next step along K overlaps the tensor-core
+ * work of the current one (two stages).  Arguments, results, bits of w_hat_out / scale_out and error behaviour as
+ * for gws_gemm_fused; m must be a multiple of 256 * cluster_blocks.  No load is multicast; the blocks of a cluster
+ * exchange data only through shared-memory stores and mbarrier arrivals, every wait is bounded as above. */
+int gws_gemm_fused_cluster(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y,
+                           void* w_hat_out, float* scale_out, int* status, int cluster_blocks, void* stream);
 const char* gws_gemm_last_error(void);
 /* Diagnostic: runs the fused GEMM's bounded wait on an mbarrier that nothing completes (one thread, about a
  * second).  status2: device, two ints, written: [0] = 1 (the wait gave up, as it must), [1] = SM cycles waited / 1024. */

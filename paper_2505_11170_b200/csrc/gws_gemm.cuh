@@ -282,16 +282,19 @@ int gws_gemm_wait_probe(int* status2, void* stream) {
   return GWS_OK;
 }
 
-int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y, void* w_hat_out,
-                   float* scale_out, int* status, int rows_per_block, void* stream) {
+}  // extern "C"
+
+// Validation, tensor map of X and kernel arguments shared by both forms of the fused GEMM.  `row_multiple`: m must be a
+// multiple of it.  Returns 1 when there is nothing to do.
+static int gemm_prepare(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y, void* w_hat_out,
+                        float* scale_out, int* status, int64_t row_multiple, CUtensorMap& map, GemmArgs& args) {
   if (wdesc == nullptr) return GWS_ERR_NULL;
   if (m < 0 || wdesc->rows < 0 || wdesc->cols < 0) return GWS_ERR_SHAPE;
-  if (m == 0 || wdesc->rows == 0 || wdesc->cols == 0) return GWS_OK;
+  if (m == 0 || wdesc->rows == 0 || wdesc->cols == 0) return 1;
   if (x == nullptr || w == nullptr || bt == nullptr || y == nullptr) return GWS_ERR_NULL;
-  if (rows_per_block != 128 && rows_per_block != 256 && rows_per_block != 512) return GWS_ERR_UNSUPPORTED;
   const int64_t n = wdesc->rows, k = wdesc->cols;
   if (wdesc->group_rows != 1 || wdesc->group_cols != kTileK || wdesc->ld != k || k % kTileK != 0 || n % kTileN != 0 ||
-      m % rows_per_block != 0 || wdesc->elem_offset % 8 != 0)
+      m % row_multiple != 0 || wdesc->elem_offset % 8 != 0)
     return GWS_ERR_UNSUPPORTED;
   const uint64_t first_vec = wdesc->elem_offset >> 3, last_vec = first_vec + static_cast<uint64_t>(n * k / 8) - 1;
   if ((first_vec >> 32) != (last_vec >> 32) || n * k > 0xFFFFFFFFLL || m * k > (1LL << 40)) return GWS_ERR_UNSUPPORTED;
@@ -324,7 +327,6 @@ int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* 
     }
     encode = reinterpret_cast<EncodeTiled>(fn);
   }
-  CUtensorMap map;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(k), static_cast<cuuint64_t>(m)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(k) * 2u};
   const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(kTileM)};
@@ -337,7 +339,6 @@ int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* 
     return GWS_ERR_CUDA;
   }
 
-  GemmArgs args;
   std::memset(&args, 0, sizeof args);
   args.w = w;
   args.bt = bt;
@@ -352,10 +353,41 @@ int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* 
   args.k1 = static_cast<uint32_t>(wdesc->seed >> 32);
   args.pre = gws::philox_pre(static_cast<uint32_t>(first_vec >> 32), static_cast<uint32_t>(wdesc->step), static_cast<uint32_t>(wdesc->step >> 32),
                              args.k0, args.k1);
+  return GWS_OK;
+}
+
+extern "C" {
+
+int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y, void* w_hat_out,
+                   float* scale_out, int* status, int rows_per_block, void* stream) {
+  if (rows_per_block != 128 && rows_per_block != 256 && rows_per_block != 512) return wdesc == nullptr ? GWS_ERR_NULL : GWS_ERR_UNSUPPORTED;
+  CUtensorMap map;
+  GemmArgs args;
+  const int st = gemm_prepare(wdesc, m, x, w, bt, y, w_hat_out, scale_out, status, rows_per_block, map, args);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (rows_per_block == 128) return launch_gemm<1>(map, args, m, s);
   if (rows_per_block == 256) return launch_gemm<2>(map, args, m, s);
   return launch_gemm<4>(map, args, m, s);
+}
+
+}  // extern "C"
+
+#include "gws_gemm_cluster.cuh"
+
+extern "C" {
+
+int gws_gemm_fused_cluster(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y, void* w_hat_out,
+                           float* scale_out, int* status, int cluster_blocks, void* stream) {
+  if (cluster_blocks != 1 && cluster_blocks != 2 && cluster_blocks != 4) return wdesc == nullptr ? GWS_ERR_NULL : GWS_ERR_UNSUPPORTED;
+  CUtensorMap map;
+  GemmArgs args;
+  const int st = gemm_prepare(wdesc, m, x, w, bt, y, w_hat_out, scale_out, status, static_cast<int64_t>(kClMT) * kTileM * cluster_blocks, map, args);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cluster_blocks == 1) return launch_gemm_cluster<1>(map, args, m, s);
+  if (cluster_blocks == 2) return launch_gemm_cluster<2>(map, args, m, s);
+  return launch_gemm_cluster<4>(map, args, m, s);
 }
 
 }  // extern "C"

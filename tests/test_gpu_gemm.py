@@ -54,6 +54,43 @@ def test_fused_gemm_matches_the_oracle(m, n, k, rows_per_block):
     _check_y(y.cpu(), x, f32_of_bits(want_hat).astype(np.float64).reshape(n, k))
 
 
+@pytest.mark.parametrize("m,n,k,cluster", [(256, 128, 128, 1), (512, 256, 384, 2), (1024, 128, 256, 4), (2048, 384, 512, 4),
+                                           (1024, 256, 1024, 2), (768, 128, 640, 1)])
+def test_cluster_form_matches_the_oracle(m, n, k, cluster):
+    # every block of a cluster samples a share of each W tile and stores it into the shared memory of all of them
+    x, w, bt = _inputs(m, n, k, m + n + k + cluster)
+    d = Desc.make(n, k, 1, 128, seed=0xC1A57E4, step=3, elem_offset=1 << 12)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    w_hat_out = torch.zeros(n, k, dtype=torch.bfloat16, device=DEV)
+    scale_out = torch.zeros(n * k // 128, device=DEV)
+    y = torch.full((m, n), float("nan"), dtype=torch.bfloat16, device=DEV)
+    gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), y=y, w_hat_out=w_hat_out, scale_out=scale_out, status=status, cluster=cluster)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    want_hat, want_scale = orc.sample_fwd(bits_of(w), bt.numpy(), n, k, 1, 128, seed=d.seed, step=d.step, elem_offset=d.elem_offset)
+    assert np.array_equal(bits_of(w_hat_out).ravel(), want_hat)
+    assert np.array_equal(scale_out.cpu().numpy().view(np.uint32), want_scale.view(np.uint32))
+    assert not torch.isnan(y.float()).any()
+    _check_y(y.cpu(), x, f32_of_bits(want_hat).astype(np.float64).reshape(n, k))
+    # the same sums in the same order as the single-block form: identical bits
+    y_single = gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), rows_per_block=128 if m % 256 else 256)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), y_single.view(torch.int16))
+
+
+def test_cluster_form_refuses_other_shapes_before_any_launch():
+    lib = gws.load_library()
+    buf = torch.zeros(1 << 21, dtype=torch.bfloat16, device=DEV)
+    f = torch.ones(1 << 14, device=DEV)
+    p, fp = buf.data_ptr(), f.data_ptr()
+    call = lambda d, m, c: lib.gws_gemm_fused_cluster(ctypes.byref(d), m, p, p + (1 << 20), fp, p + (1 << 21), None, None, None, c, None)
+    assert call(Desc.make(128, 128, 1, 128), 256, 3) == binding.ERR_UNSUPPORTED            # cluster size
+    assert call(Desc.make(128, 128, 1, 128), 256, 2) == binding.ERR_UNSUPPORTED            # m not a multiple of 256 * 2
+    assert call(Desc.make(128, 128, 1, 128), 128, 1) == binding.ERR_UNSUPPORTED
+    assert call(Desc.make(128, 128, 1, 32), 256, 1) == binding.ERR_UNSUPPORTED             # group size
+    assert call(Desc.make(128, 128, 1, 128), 0, 4) == binding.OK                           # nothing to do
+
+
 def test_fused_gemm_without_optional_outputs_gives_the_same_y():
     m, n, k = 512, 256, 256
     x, w, bt = _inputs(m, n, k, 5)
@@ -77,8 +114,10 @@ def test_config5_up_projection_on_sampled_rows():
     d = Desc.make(n, k, 1, 128, seed=syn.layer_seed(0, 0), step=0)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     y = gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), status=status, rows_per_block=512)
+    y_cluster = gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), status=status, cluster=4)
     torch.cuda.synchronize()
     assert status.item() == 0
+    assert torch.equal(y.view(torch.int16), y_cluster.view(torch.int16))
     want_hat, _ = orc.sample_fwd(bits_of(w), bt.numpy(), n, k, 1, 128, seed=d.seed, step=0)
     rows = np.concatenate([np.arange(0, 8), np.random.default_rng(1).choice(m, 40, replace=False), np.arange(m - 8, m)])
     rows = torch.from_numpy(np.unique(rows))

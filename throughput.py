@@ -122,8 +122,12 @@ def run_gemm(reps: int, dev) -> dict:
             "plain_gemm_us": timed(lambda i: torch.matmul(x, w.t(), out=y)), "sample_then_gemm_us": timed(unfused)}
     for rpb in (128, 256, 512):
         line[f"fused_{rpb}_rows_per_block_us"] = timed(lambda i: gws.gemm_fused(d.with_step(i), x, w, bt, y=y, status=status, rows_per_block=rpb))
+    for c in (1, 2, 4):
+        line[f"fused_cluster_of_{c}_us"] = timed(lambda i: gws.gemm_fused(d.with_step(i), x, w, bt, y=y, status=status, cluster=c))
     line["status"] = int(status.item())
     line["fused_TFLOP/s"] = line["flops"] / (line["fused_512_rows_per_block_us"] * 1e-6) / 1e12
+    line["fused_cluster_of_4_TFLOP/s"] = line["flops"] / (line["fused_cluster_of_4_us"] * 1e-6) / 1e12
+    line["overhead_fused_cluster_of_4_pct"] = 100.0 * (line["fused_cluster_of_4_us"] / line["plain_gemm_us"] - 1.0)
     line["overhead_unfused_pct"] = 100.0 * (line["sample_then_gemm_us"] / line["plain_gemm_us"] - 1.0)
     line["overhead_fused_pct"] = 100.0 * (line["fused_512_rows_per_block_us"] / line["plain_gemm_us"] - 1.0)
     print(json.dumps(line), flush=True)
