@@ -253,6 +253,29 @@ def arithmetic_budget(gws, dev):
                               "instruction), at the SM clock the probes measured"}
 
 
+def sharded_step_leg(make_sampler, specs, rank, world, dist, device, timer, reps=10):
+    """The one form of the pass that has an exchange step: every tensor cut into `world` flat shards (ZeRO / FSDP style),
+    each rank sampling its shard; groups that reach across a cut go through a MAX all-reduce (forward) and a SUM all-reduce
+    (backward) of world + 1 floats per tensor.  `make_sampler(plans)` returns an object with forward(step) / backward(step)
+    that does the rank's local work and the all-reduces; `timer(fn, reps)` returns milliseconds per call on this rank.
+    Returns the whole-job figures (maximum over ranks of the time, sum over ranks of the elements)."""
+    from paper_2505_11170_b200.sharding import plan_flat_shard
+    plans = [plan_flat_shard(s.rows * s.cols, s.group_cols or s.cols, rank, world) for s in specs]
+    sampler = make_sampler(plans)
+    fwd_ms = timer(lambda k: sampler.forward(k), reps)
+    bwd_ms = timer(lambda k: sampler.backward(k), reps)
+    mine = float(sum(p.n_elements for p in plans))
+    fwd_ms, bwd_ms = max_over_ranks([fwd_ms, bwd_ms], dist, device)
+    t = torch.tensor([mine, float(sum(len(p.pieces) for p in plans))], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    elems, pieces = float(t[0]), int(t[1])
+    return {"world": world, "elements": int(elems), "end_pieces_all_ranks": pieces, "fwd_ms": fwd_ms, "bwd_ms": bwd_ms,
+            "fwd_GB/s": elems * FWD_BYTES_PER_ELEM / (fwd_ms * 1e-3) / 1e9, "bwd_GB/s": elems * BWD_BYTES_PER_ELEM / (bwd_ms * 1e-3) / 1e9,
+            "all_reduce_floats_per_pass": len(specs) * (world + 1),
+            "note": "whole job: every rank samples 1/world of every tensor; times are the slowest rank's, all-reduces included"}
+
+
 def cpu_baseline(specs, descs, W, BT, G):
     """The oracle, as it stands, on one full forward + backward pass of the whole weight set (one step counter):
     one single-threaded oracle process per host core, each with its own tensors (oracle/pool.py)."""
@@ -493,11 +516,13 @@ def main():
             per_elem = 2 + code_bytes + 1 / 32 + 8 / 128
             fwd_mx[name] = {"ms_per_launch": ms, "bytes_per_element": per_elem, "GB/s": n_elem * per_elem / (ms * 1e-3) / 1e9,
                             "gelem_per_s": n_elem / (ms * 1e-3) / 1e9}
-            # the conversion alone, from the BF16 w_hat of the last forward pass (one launch per tensor)
-            q_ms = timed(lambda k: [gws.mx_quantize(descs[i], fmt, WH[i], mx_out=MX[i]) for i in range(len(specs))], 5)
-            fwd_mx[name]["quantize_only"] = {"ms": q_ms, "launches": len(specs),
-                                             "GB/s": n_elem * (2 + code_bytes + 1 / 32) / (q_ms * 1e-3) / 1e9}
-            del mx_plan, MX
+            # the conversion alone, from the BF16 w_hat of the last forward pass: one launch over the whole set
+            q_plan = gws.MultiPlan(descs, w=WH, w_hat=MX, mx_format=fmt)
+            q_ms = timed(lambda k: q_plan.mx_quantize_multi(fmt), 10)
+            q_gbs = n_elem * (2 + code_bytes + 1 / 32) / (q_ms * 1e-3) / 1e9
+            fwd_mx[name]["quantize_only"] = {"ms": q_ms, "launches": q_plan.launches_per_pass, "GB/s": q_gbs,
+                                             "frac_of_measured_hbm": q_gbs / measured_peaks()[0]}
+            del mx_plan, q_plan, MX
         extras = {
             "fwd_mx_output": fwd_mx,
             "sharded_rank_local_work": {"world": shard_world, "rank": shard_rank, "elements": sh_elems, "end_pieces": sh.n_pieces,
@@ -511,6 +536,30 @@ def main():
                                      "bytes_per_element": 4 + 8 / 128},
             "arithmetic_budget": alu,
         }
+
+    # ---- N > 1 only: the sharded form of the step, the one place where ranks exchange anything ----
+    sharded = None
+    if world > 1 and not args.no_extras:
+        from paper_2505_11170_b200.sharding import ShardedSetSampler
+        cut = lambda t, p_: t.view(-1)[p_.begin:p_.end]
+
+        def make_sampler(plans):
+            return ShardedSetSampler(plans, [d.seed for d in descs], [cut(W[i], p_) for i, p_ in enumerate(plans)],
+                                     [BT[i][p_.first_group:p_.first_group + p_.n_local_groups].contiguous() for i, p_ in enumerate(plans)],
+                                     [cut(WH[i], p_) for i, p_ in enumerate(plans)], [cut(G[i], p_) for i, p_ in enumerate(plans)])
+
+        def rank_timer(fn, reps):
+            fn(0)
+            barrier()
+            a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a_.record(stream)
+            for k in range(reps):
+                fn(1 + k)
+            b_.record(stream)
+            barrier()
+            return a_.elapsed_time(b_) / reps
+
+        sharded = sharded_step_leg(make_sampler, specs, rank, world, dist, dev, rank_timer)
 
     if rank != 0:
         if dist is not None:
@@ -546,6 +595,8 @@ def main():
                          "algorithmic_bytes_per_launch": bwd_bytes, "traffic": traffic.get("bwd_bytes_per_launch")},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
     }
+    if sharded is not None:
+        line["extras"] = {"sharded_step": sharded}
     if extras is not None:
         line["extras"] = extras
         # the backward pass is bound by integer instruction issue, not by HBM: also report it against the ceiling that

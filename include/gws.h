@@ -253,7 +253,8 @@ int gws_gemm_wait_probe(int* status2, void* stream);
 
 /* Host arrays of n device pointers each; the meaning of every pointer is that of the
  * single-tensor call.  scale is written by forward and read by backward.  grad_w_hat, grad_w and
- * grad_bt may be NULL arrays if backward is never called; w, bt, w_hat if forward is not. */
+ * grad_bt may be NULL arrays if backward is never called; w, bt, w_hat if forward is not (bt alone may be NULL
+ * in a plan with MX outputs that is only used by gws_mx_quantize_multi). */
 typedef struct gws_multi_ptrs {
   const void* const* w;
   const float* const* bt;
@@ -339,6 +340,12 @@ int gws_sample_fwd_scaled_multi(const gws_multi_plan* plan, uint64_t step, void*
  * what the MX calls support; gws_sample_fwd_multi and gws_sample_fwd_scaled_multi refuse such a plan
  * the same way (they would write 2 bytes per element). */
 int gws_sample_fwd_mx_multi(const gws_multi_plan* plan, int format, uint64_t step, void* stream);
+
+/* gws_mx_quantize for every tensor of such a plan, one launch per kernel class: the plan's `w` pointers are then the
+ * BF16 w_hat tensors to convert (read only) and its `w_hat` pointers the MX buffers; `bt` and `scale` are not used and
+ * the plan may have been prepared with bt = NULL (gws_sample_fwd_mx_multi then returns GWS_ERR_NULL for it).  Same
+ * refusals as gws_sample_fwd_mx_multi. */
+int gws_mx_quantize_multi(const gws_multi_plan* plan, int format, void* stream);
 
 /* ---- bit-width parametrisation and seeds (Section 3.6, "Bitwidth" and "Managing seed") ---------------
  *

@@ -82,6 +82,7 @@ _SIGNATURES = {
     "gws_multi_launch_count": (c_int, [POINTER(_MultiPlan), c_int]),
     "gws_sample_fwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_sample_bwd_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
+    "gws_mx_quantize_multi": (c_int, [POINTER(_MultiPlan), c_int, c_void_p]),
     "gws_sample_fwd_scaled_multi": (c_int, [POINTER(_MultiPlan), c_uint64, c_void_p]),
     "gws_bitwidth": (c_int, [c_int64, c_void_p, c_float, c_float, c_void_p, c_void_p]),
     "gws_bitwidth_loss": (c_int, [c_int64, c_void_p, c_float, c_void_p, c_void_p]),
@@ -366,6 +367,10 @@ class MultiPlan:
     def sample_fwd_mx_multi(self, fmt: int, step: int, stream=None) -> None:
         """Forward with MX output; the plan's ``w_hat`` tensors are MX buffers (uint8, ``mx_layout``)."""
         _check(load_library().gws_sample_fwd_mx_multi(ctypes.byref(self.plan), fmt, step, _stream(stream)))
+
+    def mx_quantize_multi(self, fmt: int, stream=None) -> None:
+        """BF16 -> MX for every tensor: the plan's ``w`` tensors are the BF16 w_hat to convert, its ``w_hat`` tensors the MX buffers."""
+        _check(load_library().gws_mx_quantize_multi(ctypes.byref(self.plan), fmt, _stream(stream)))
 
     def sample_fwd_scaled_multi(self, step: int, stream=None) -> None:
         """Forward with the factors already in the plan's ``scale`` arrays (read, not written)."""

@@ -731,7 +731,8 @@ static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs
   const bool has_fwd = ptrs->w != nullptr;
   const bool has_bwd = ptrs->grad_w_hat != nullptr;
   if (!has_fwd && !has_bwd) return GWS_ERR_NULL;
-  if (has_fwd && (ptrs->bt == nullptr || ptrs->w_hat == nullptr)) return GWS_ERR_NULL;
+  // a plan with MX outputs may come without bit-widths: it then serves gws_mx_quantize_multi only
+  if (has_fwd && (ptrs->w_hat == nullptr || (ptrs->bt == nullptr && ptrs->w_hat_kind == 0))) return GWS_ERR_NULL;
   if (has_bwd && (ptrs->scale == nullptr || ptrs->grad_bt == nullptr)) return GWS_ERR_NULL;
   if (workspace == nullptr || !aligned(workspace, 256) || workspace_bytes < gws_workspace_bytes(n)) return GWS_ERR_WORKSPACE;
   const int kind = ptrs->w_hat_kind;
@@ -750,8 +751,8 @@ static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs
     if (has_fwd) {
       const void* w = ptrs->w[i];
       void* w_hat = ptrs->w_hat[i];
-      const float* bt = ptrs->bt[i];
-      if (w == nullptr || w_hat == nullptr || bt == nullptr) return GWS_ERR_NULL;
+      const float* bt = ptrs->bt ? ptrs->bt[i] : nullptr;
+      if (w == nullptr || w_hat == nullptr || (bt == nullptr && ptrs->bt != nullptr)) return GWS_ERR_NULL;
       if (!aligned(w, 2) || !aligned(w_hat, 2) || !aligned(bt, 4) || !aligned(scale, 4)) return GWS_ERR_ALIGN;
       if (kind != 0 && d->cols % 32 != 0) return GWS_ERR_UNSUPPORTED;
       const size_t out_bytes = kind == 0 ? span_bytes(d) : mx_total_bytes(d->rows * d->cols, kind - 1);
@@ -773,7 +774,7 @@ static int build_tables(int n, const gws_desc* descs, const gws_multi_ptrs* ptrs
     const int64_t tiles = tiles_of(d, cls);
     total += d->rows * d->cols;
     if (has_fwd) {
-      Entry e = make_entry(d, cls, ptrs->w[i], ptrs->w_hat[i], ptrs->bt[i], scale);
+      Entry e = make_entry(d, cls, ptrs->w[i], ptrs->w_hat[i], ptrs->bt ? ptrs->bt[i] : nullptr, scale);
       e.tile_begin = tiles;  // turned into a prefix sum below
       t.fwd[cls].push_back(e);
     }
@@ -914,8 +915,10 @@ static int run_multi_mx(const gws_multi_plan* plan, uint64_t step, void* stream)
     return reinterpret_cast<const Entry*>(static_cast<const char*>(plan->host_tables) + plan->fwd_offset[cls]);
   };
   for (int cls = 0; cls < 4; ++cls)
-    for (int i = 0; i < plan->count[cls]; ++i)
+    for (int i = 0; i < plan->count[cls]; ++i) {
       if (!mx_entry_ok(cls, host_table(cls)[i])) return GWS_ERR_UNSUPPORTED;
+      if (gws::mode_is_mx_fwd(MODE) && host_table(cls)[i].gin == nullptr) return GWS_ERR_NULL;   // sampling needs the bit-widths
+    }
   for (int cls = 0; cls < 4; ++cls) {
     if (plan->count[cls] == 0) continue;
     const int st = launch_mx<MODE>(cls, host_table(cls), plan->count[cls], step, static_cast<cudaStream_t>(stream));
@@ -930,6 +933,13 @@ int gws_sample_fwd_mx_multi(const gws_multi_plan* plan, int format, uint64_t ste
   if (format == GWS_MX_FP8_E4M3) return run_multi_mx<gws::kFwdMx8>(plan, step, stream);
   if (format == GWS_MX_FP6_E3M2) return run_multi_mx<gws::kFwdMx6>(plan, step, stream);
   if (format == GWS_MX_FP8_E3M4) return run_multi_mx<gws::kFwdMx8b>(plan, step, stream);
+  return GWS_ERR_UNSUPPORTED;
+}
+
+int gws_mx_quantize_multi(const gws_multi_plan* plan, int format, void* stream) {
+  if (format == GWS_MX_FP8_E4M3) return run_multi_mx<gws::kQuantMx8>(plan, 0, stream);
+  if (format == GWS_MX_FP6_E3M2) return run_multi_mx<gws::kQuantMx6>(plan, 0, stream);
+  if (format == GWS_MX_FP8_E3M4) return run_multi_mx<gws::kQuantMx8b>(plan, 0, stream);
   return GWS_ERR_UNSUPPORTED;
 }
 

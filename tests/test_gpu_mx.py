@@ -118,6 +118,33 @@ def test_many_tensors_share_launches(fmt_gpu, fmt_orc):
         assert np.array_equal(SC[k].cpu().numpy().view(np.uint32), want_scale.view(np.uint32)), k
 
 
+@pytest.mark.parametrize("fmt_gpu,fmt_orc", FORMATS)
+def test_conversion_alone_over_many_tensors_shares_launches(fmt_gpu, fmt_orc):
+    # gws_mx_quantize_multi: the plan's `w` tensors are BF16 w_hat tensors to convert; no bit-widths are needed
+    shapes = [(64, 256, 1, 128), (33, 768, 1, 0), (64, 64, 32, 32), (20, 512, 1, 32), (7, 8192, 1, 0), (96, 96, 32, 32), (40, 1024, 1, 128)]
+    descs = [Desc.make(r, c, gr, gc, seed=7 + k) for k, (r, c, gr, gc) in enumerate(shapes)]
+    WH = [_weights(r, c, 90 + k).to(DEV) for k, (r, c, gr, gc) in enumerate(shapes)]
+    OUT = [torch.full((gws.mx_layout(d, fmt_gpu)[2],), 0xAB, dtype=torch.uint8, device=DEV) for d in descs]
+    plan = gws.MultiPlan(descs, w=WH, w_hat=OUT, mx_format=fmt_gpu)
+    before = gws.launch_count()
+    plan.mx_quantize_multi(fmt_gpu)
+    launches = gws.launch_count() - before
+    torch.cuda.synchronize()
+    assert launches <= 5
+    for k, (r, c, gr, gc) in enumerate(shapes):
+        want_codes, want_scales = _want(bits_of(WH[k]), r, c, gr, gc, fmt_orc)
+        codes, scales, gap, tail = _unpack(OUT[k], descs[k], fmt_gpu)
+        assert np.array_equal(codes, want_codes), k
+        assert np.array_equal(scales, want_scales), k
+        assert (gap == 0xAB).all() and (tail == 0xAB).all()
+    # without bit-widths the plan cannot sample; with another format it cannot convert
+    lib = gws.load_library()
+    before = gws.launch_count()
+    assert lib.gws_sample_fwd_mx_multi(ctypes.byref(plan.plan), fmt_gpu, 1, None) == binding.ERR_NULL
+    assert lib.gws_mx_quantize_multi(ctypes.byref(plan.plan), (fmt_gpu + 1) % 3, None) == binding.ERR_UNSUPPORTED
+    assert gws.launch_count() == before
+
+
 def test_unsupported_shapes_are_refused_before_any_launch():
     lib = gws.load_library()
     w = torch.zeros(64 * 96 + 64, dtype=torch.bfloat16, device=DEV)
