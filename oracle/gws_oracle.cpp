@@ -517,4 +517,75 @@ uint64_t gwso_layer_seed(uint64_t user_seed, uint64_t layer) {
   return static_cast<uint64_t>(o[0]) | (static_cast<uint64_t>(o[1]) << 32);
 }
 
+// ---- comparison noises (Section 4, first paragraph: "DiffQ" = this method with BF16 U(-0.5, 0.5) in place of R; Section 3.4
+// and the "bm" series of the forward benchmark: R = round(N(0,1) / 2) with the normals from the Box-Muller transform) -----------
+
+// BF16 U(-0.5, 0.5): element e takes the 16-bit field x at bits [16 (e & 1), +16) of word (e >> 1) & 3 of the Philox output
+// for vector e >> 3; u = ((x + 1/2) / 2^16 - 1/2) rounded to BF16 (nearest even).  (x + 1/2) / 2^16 is the midpoint rule for
+// "random integer divided by its maximum": symmetric about 0 and never exactly -1/2 before rounding.
+static uint16_t uniform_bf16_of_field(uint32_t x) {
+  const double u = (static_cast<double>(x & 0xFFFFu) + 0.5) / 65536.0 - 0.5;
+  return f32_to_bf16_rne(static_cast<float>(u));   // u is a multiple of 2^-17 below 1 in magnitude: exact in float
+}
+
+void gwso_noise_uniform(uint64_t seed, uint64_t step, uint64_t first_elem, int64_t n, uint16_t* u_bf16) {
+  for (int64_t k = 0; k < n; ++k) {
+    const uint64_t e = first_elem + static_cast<uint64_t>(k);
+    uint32_t o[4];
+    philox_for_vector(seed, step, e >> 3, o);
+    const unsigned t = static_cast<unsigned>(e & 7u);
+    u_bf16[k] = uniform_bf16_of_field((o[t >> 1] >> (16u * (t & 1u))) & 0xFFFFu);
+  }
+}
+
+// Box-Muller: one Philox call (counter = e >> 2 in place of the vector index) serves 4 elements; words (o0, o1) give the
+// normals of elements 4c and 4c + 1, words (o2, o3) those of 4c + 2 and 4c + 3:
+//   u1 = ((a >> 8) + 1) / 2^24 in (0, 1],  u2 = (b >> 8) / 2^24 in [0, 1),
+//   z0 = sqrt(-2 ln u1) cos(2 pi u2),  z1 = sqrt(-2 ln u1) sin(2 pi u2).
+static void box_muller_pair(uint32_t a, uint32_t b, double* z0, double* z1) {
+  const double u1 = (static_cast<double>(a >> 8) + 1.0) / 16777216.0, u2 = static_cast<double>(b >> 8) / 16777216.0;
+  const double radius = std::sqrt(-2.0 * std::log(u1)), angle = 6.283185307179586476925286766559 * u2;
+  *z0 = radius * std::cos(angle);
+  *z1 = radius * std::sin(angle);
+}
+
+void gwso_noise_bm_z(uint64_t seed, uint64_t step, uint64_t first_elem, int64_t n, double* z) {
+  for (int64_t k = 0; k < n; ++k) {
+    const uint64_t e = first_elem + static_cast<uint64_t>(k);
+    uint32_t o[4];
+    philox_for_vector(seed, step, e >> 2, o);
+    double z0, z1;
+    box_muller_pair(o[(e & 2u) ? 2 : 0], o[(e & 2u) ? 3 : 1], &z0, &z1);
+    z[k] = (e & 1u) ? z1 : z0;
+  }
+}
+
+// R = round-half-even(z / 2), the rounded normal the method approximates (Section 3.4).
+void gwso_noise_bm_r(uint64_t seed, uint64_t step, uint64_t first_elem, int64_t n, int8_t* r) {
+  for (int64_t k = 0; k < n; ++k) {
+    double z;
+    gwso_noise_bm_z(seed, step, first_elem + static_cast<uint64_t>(k), 1, &z);
+    r[k] = static_cast<int8_t>(std::nearbyint(0.5 * z));   // default rounding mode: to nearest, ties to even
+  }
+}
+
+// Eq. 3 + the BF16 cast with a real-valued noise u given as BF16 bit patterns, one per element in logical order:
+// w_hat = bf16( fl32( float(w) + fl32( float(u) * s_g ) ) ), s_g as in gwso_sample_fwd.
+void gwso_sample_fwd_bf16_noise(int64_t rows, int64_t cols, int64_t ld, int64_t group_rows, int64_t group_cols,
+                                const uint16_t* w, const float* bt, const uint16_t* u_bf16, uint16_t* w_hat,
+                                float* scale_out, float* absmax_scratch) {
+  const Geometry geo = make_geometry(rows, cols, ld, group_rows, group_cols);
+  gwso_group_absmax(rows, cols, ld, group_rows, group_cols, w, absmax_scratch);
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const int64_t g = group_of(geo, i, j);
+      const float s = scale_of(absmax_scratch[g], bt[g]);
+      const float pqn = bf16_to_f32(u_bf16[i * cols + j]) * s;
+      const float y = bf16_to_f32(w[i * ld + j]) + pqn;
+      w_hat[i * ld + j] = f32_to_bf16_rne(y);
+    }
+  if (scale_out)
+    for (int64_t g = 0; g < geo.n_groups; ++g) scale_out[g] = scale_of(absmax_scratch[g], bt[g]);
+}
+
 }  // extern "C"

@@ -77,6 +77,14 @@ def lib() -> ctypes.CDLL:
         L.gwso_sample_fwd.restype = None
         L.gwso_sample_fwd_scaled.argtypes = [c_int64] * 5 + [c_uint64] * 3 + [u16p, f32p, u16p]
         L.gwso_sample_fwd_scaled.restype = None
+        L.gwso_noise_uniform.argtypes = [c_uint64, c_uint64, c_uint64, c_int64, u16p]
+        L.gwso_noise_uniform.restype = None
+        L.gwso_noise_bm_z.argtypes = [c_uint64, c_uint64, c_uint64, c_int64, f64p]
+        L.gwso_noise_bm_z.restype = None
+        L.gwso_noise_bm_r.argtypes = [c_uint64, c_uint64, c_uint64, c_int64, i8p]
+        L.gwso_noise_bm_r.restype = None
+        L.gwso_sample_fwd_bf16_noise.argtypes = [c_int64] * 5 + [u16p, f32p, u16p, u16p, f32p, f32p]
+        L.gwso_sample_fwd_bf16_noise.restype = None
         u8p = POINTER(ctypes.c_uint8)
         L.gwso_mx_decode.argtypes = [c_int, c_uint32]
         L.gwso_mx_decode.restype = c_double
@@ -242,6 +250,45 @@ def sample_bwd(g, scale_, rows, cols, group_rows=1, group_cols=0, seed=0, step=0
         lib().gwso_sample_bwd_injected(rows, cols, ld, group_rows, group_cols, _p(g, c_uint16), _p(sc, c_float),
                                        _p(r, c_int8), _p(gw, c_uint16), _p(gbt, c_float), _p(acc, c_double))
     return gw, gbt
+
+
+# ---- comparison noises (Section 4: "DiffQ" = BF16 U(-0.5, 0.5) in place of R; Section 3.4 / "bm": Box-Muller) ----------
+
+def noise_uniform(seed: int, step: int, first_elem: int, n: int) -> np.ndarray:
+    """BF16 bit patterns of the U(-0.5, 0.5) comparison noise of elements first_elem .. first_elem + n - 1."""
+    out = np.empty(n, np.uint16)
+    lib().gwso_noise_uniform(seed, step, first_elem, n, _p(out, c_uint16))
+    return out
+
+
+def noise_bm_z(seed: int, step: int, first_elem: int, n: int) -> np.ndarray:
+    """The Box-Muller normals (float64, before halving and rounding)."""
+    out = np.empty(n, np.float64)
+    lib().gwso_noise_bm_z(seed, step, first_elem, n, _p(out, c_double))
+    return out
+
+
+def noise_bm_r(seed: int, step: int, first_elem: int, n: int) -> np.ndarray:
+    """R = round-half-even(N(0, 1) / 2) from the Box-Muller normals."""
+    out = np.empty(n, np.int8)
+    lib().gwso_noise_bm_r(seed, step, first_elem, n, _p(out, c_int8))
+    return out
+
+
+def sample_fwd_bf16_noise(w, bt, u_bf16, rows, cols, group_rows=1, group_cols=0, ld=None):
+    """Eq. 3 + cast with a BF16-valued noise (uint16 [rows*cols], logical order).  Returns (w_hat, scale)."""
+    ld = cols if ld is None else ld
+    w = _check_w(w, rows, cols, ld)
+    ng = n_groups(rows, cols, group_rows, group_cols)
+    bt = _c(bt, np.float32)
+    u = _c(u_bf16, np.uint16)
+    assert bt.size == ng and u.size == rows * cols
+    w_hat = w.copy()
+    sc = np.empty(ng, np.float32)
+    scratch = np.empty(ng, np.float32)
+    lib().gwso_sample_fwd_bf16_noise(rows, cols, ld, group_rows, group_cols, _p(w, c_uint16), _p(bt, c_float), _p(u, c_uint16),
+                                     _p(w_hat, c_uint16), _p(sc, c_float), _p(scratch, c_float))
+    return w_hat, sc
 
 
 # ---- bit-width parametrisation and seeds (Section 3.6) -------------------------------------------------
