@@ -423,6 +423,29 @@ int gws_sample_step_host(const gws_desc* desc, const void* h_w, const float* h_b
                          void* h_w_hat, float* h_scale, float* h_grad_bt, void* d_w, void* d_w_hat, void* d_grad,
                          float* d_bt, float* d_scale, float* d_grad_bt, void* stream);
 
+/* ---- comparison noises ----------------------------------------------------------------------------
+ * The forward pass of Eq. 3 with the noise R replaced by what the paper measures its generation against, on the same
+ * kernel shape, so that the cost of the noise can be compared on one harness (Section 4.2 "Overhead": forward unit
+ * benchmark with the series "ours" and "bm"; Section 4, first paragraph: "DiffQ" = the method with BF16 U(-0.5, 0.5)
+ * in place of R).  Not part of the sampling pass.
+ *   GWS_NOISE_UNIFORM_BF16   u = bf16_rne((x + 1/2) / 2^16 - 1/2), x the 16-bit field at bits [16 (e & 1), +16) of
+ *                            word (e >> 1) & 3 of Philox4x32-10(counter = (e >> 3, step), key = seed)
+ *   GWS_NOISE_BOX_MULLER     R = round-half-even(z / 2), z the Box-Muller normal of element e: one Philox call with
+ *                            counter (e >> 2, step) serves 4 elements, words (o0, o1) give elements 4c, 4c + 1 and
+ *                            (o2, o3) give 4c + 2, 4c + 3; u1 = ((a >> 8) + 1) / 2^24, u2 = (b >> 8) / 2^24,
+ *                            z = sqrt(-2 ln u1) * (cos, sin)(2 pi u2) in FP32 (so an R may differ from an FP64
+ *                            evaluation where z / 2 is within rounding of k + 1/2)
+ * w_hat = bf16( fl32( float(w) + fl32( noise * scale_g ) ) ), scale_g as in gws_sample_fwd.
+ * Shapes: dense, group_rows = 1, group_cols in {32, 64, 128, 256} dividing cols, elem_offset % 32 == 0, w and w_hat
+ * 32-byte aligned; anything else GWS_ERR_UNSUPPORTED.  Arguments as gws_sample_fwd. */
+typedef enum gws_noise_kind { GWS_NOISE_UNIFORM_BF16 = 0, GWS_NOISE_BOX_MULLER = 1 } gws_noise_kind;
+int gws_sample_fwd_compare(const gws_desc* desc, int noise_kind, const void* w, const float* bt, void* w_hat,
+                           float* scale_out, void* stream);
+/* The comparison noise alone for rows * cols elements (a multiple of 8, as is elem_offset).  out: device, 16-byte aligned;
+ * GWS_NOISE_UNIFORM_BF16: one BF16 pattern per element (u16 [rows * cols]); GWS_NOISE_BOX_MULLER: sign-magnitude nibbles
+ * as written by gws_noise (u32 [rows * cols / 8], |R| <= 3). */
+int gws_noise_compare(const gws_desc* desc, int noise_kind, void* out, void* stream);
+
 /* ---- diagnostics -----------------------------------------------------------------------------*/
 
 /* Raw Philox4x32-10 output words for vectors first_vec .. first_vec+n_vec-1 (4 words each):

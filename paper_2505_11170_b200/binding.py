@@ -94,6 +94,8 @@ _SIGNATURES = {
     "gws_noise_alu_probe": (c_int, [POINTER(Desc), c_void_p, c_void_p]),
     "gws_noise_alu_probe_words": (c_int64, [POINTER(Desc)]),
     "gws_host_decode8": (None, [POINTER(c_uint32), POINTER(c_int8), POINTER(c_uint32)]),
+    "gws_sample_fwd_compare": (c_int, [POINTER(Desc), c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gws_noise_compare": (c_int, [POINTER(Desc), c_int, c_void_p, c_void_p]),
     "gws_issue_probe_mix": (c_int, [c_int, POINTER(c_int32)]),
     "gws_issue_probe": (c_int, [c_int, c_int, c_void_p, POINTER(c_int32), c_void_p]),
     "gws_host_decode8_pairs": (None, [POINTER(c_uint32), POINTER(c_uint32), POINTER(c_uint32)]),
@@ -467,6 +469,30 @@ def host_decode8(words4: Sequence[int]):
     p = c_uint32(0)
     load_library().gws_host_decode8(w, r, ctypes.byref(p))
     return list(r), int(p.value)
+
+
+NOISE_UNIFORM_BF16, NOISE_BOX_MULLER = 0, 1
+
+
+def sample_fwd_compare(desc: Desc, noise_kind: int, w: torch.Tensor, bt: torch.Tensor, w_hat: Optional[torch.Tensor] = None,
+                       scale: Optional[torch.Tensor] = None, stream=None):
+    """Eq. 3 + cast with a comparison noise (BF16 uniform or Box-Muller rounded normal) in place of R.  Returns (w_hat, scale)."""
+    _require_cuda(w, bt, w_hat, scale)
+    if w_hat is None:
+        w_hat = torch.empty_like(w)
+    if scale is None:
+        scale = torch.empty(n_groups(desc), dtype=torch.float32, device=w.device)
+    _check(load_library().gws_sample_fwd_compare(ctypes.byref(desc), noise_kind, _ptr(w), _ptr(bt), _ptr(w_hat), _ptr(scale), _stream(stream)))
+    return w_hat, scale
+
+
+def noise_compare(desc: Desc, noise_kind: int, device="cuda", stream=None) -> torch.Tensor:
+    """The comparison noise alone: BF16 values (uniform) or packed sign-magnitude nibbles as int32 words (Box-Muller)."""
+    n = desc.rows * desc.cols
+    out = torch.empty(n, dtype=torch.bfloat16, device=device) if noise_kind == NOISE_UNIFORM_BF16 else \
+        torch.empty(n // 8, dtype=torch.int32, device=device)
+    _check(load_library().gws_noise_compare(ctypes.byref(desc), noise_kind, _ptr(out), _stream(stream)))
+    return out
 
 
 def issue_probe_mix(mix: int):

@@ -16,6 +16,7 @@
 #endif
 #include "gws_kernels.cuh"
 #include "gws_probe.cuh"
+#include "gws_compare.cuh"
 
 namespace {
 
@@ -699,6 +700,73 @@ int gws_issue_probe(int mix, int iterations, uint32_t* sink, int32_t* host_info2
   }
 #undef GWS_ISSUE_CASE
   return check_launch("issue probe");
+}
+
+// ---- comparison noises (not part of the sampling pass: timed beside it) -----------------------------------------
+
+// Shapes the comparison kernels take: dense tensors, groups of 32, 64, 128 or 256 contiguous elements that divide the row,
+// 32-byte aligned pointers, and counters that do not cross a multiple of 2^32 inside the tensor.
+static int compare_counters(const gws_desc* d, int kind, uint32_t* ctr_lo, gws::PhiloxPre* pre) {
+  const int shift = kind == gws::kNoiseUniformBf16 ? 3 : 2;
+  const uint64_t n = static_cast<uint64_t>(d->rows) * static_cast<uint64_t>(d->cols);
+  const uint64_t first = d->elem_offset >> shift, last = (d->elem_offset + n - 1u) >> shift;
+  if ((first >> 32) != (last >> 32) || n > 0xFFFFFFFFull) return GWS_ERR_UNSUPPORTED;
+  *ctr_lo = static_cast<uint32_t>(first);
+  *pre = gws::philox_pre(static_cast<uint32_t>(first >> 32), static_cast<uint32_t>(d->step), static_cast<uint32_t>(d->step >> 32),
+                         static_cast<uint32_t>(d->seed), static_cast<uint32_t>(d->seed >> 32));
+  return GWS_OK;
+}
+
+int gws_sample_fwd_compare(const gws_desc* desc, int noise_kind, const void* w, const float* bt, void* w_hat, float* scale_out,
+                           void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (noise_kind != gws::kNoiseUniformBf16 && noise_kind != gws::kNoiseBoxMuller) return GWS_ERR_UNSUPPORTED;
+  if (w == nullptr || bt == nullptr || w_hat == nullptr) return GWS_ERR_NULL;
+  if (!aligned(w, 2) || !aligned(w_hat, 2) || !aligned(bt, 4) || !aligned(scale_out, 4)) return GWS_ERR_ALIGN;
+  if (overlaps(w, span_bytes(desc), w_hat, span_bytes(desc))) return GWS_ERR_ALIAS;
+  const int64_t gc = resolved_group_cols(desc);
+  if (desc->group_rows != 1 || desc->ld != desc->cols || (gc != 32 && gc != 64 && gc != 128 && gc != 256) || desc->cols % gc != 0 ||
+      desc->elem_offset % 32 != 0 || !aligned(w, 32) || !aligned(w_hat, 32))
+    return GWS_ERR_UNSUPPORTED;
+  gws::CompareArgs a;
+  std::memset(&a, 0, sizeof a);
+  const int cst = compare_counters(desc, noise_kind, &a.ctr_lo, &a.pre);
+  if (cst != GWS_OK) return cst;
+  a.w = w;
+  a.bt = bt;
+  a.w_hat = w_hat;
+  a.scale_out = scale_out;
+  a.n_chunks = static_cast<uint32_t>(desc->rows * desc->cols / 32);
+  a.lanes_log2 = gc == 32 ? 0u : (gc == 64 ? 1u : (gc == 128 ? 2u : 3u));
+  a.k0 = static_cast<uint32_t>(desc->seed);
+  a.k1 = static_cast<uint32_t>(desc->seed >> 32);
+  const unsigned blocks = (a.n_chunks + 2u * gws::kFlatThreads - 1u) / (2u * gws::kFlatThreads);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (noise_kind == gws::kNoiseUniformBf16) gws::k_compare_fwd<gws::kNoiseUniformBf16><<<blocks, gws::kFlatThreads, 0, s>>>(a);
+  else gws::k_compare_fwd<gws::kNoiseBoxMuller><<<blocks, gws::kFlatThreads, 0, s>>>(a);
+  return check_launch("comparison forward kernel");
+}
+
+int gws_noise_compare(const gws_desc* desc, int noise_kind, void* out, void* stream) {
+  const int st = precheck(desc);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  if (noise_kind != gws::kNoiseUniformBf16 && noise_kind != gws::kNoiseBoxMuller) return GWS_ERR_UNSUPPORTED;
+  if (out == nullptr) return GWS_ERR_NULL;
+  if (!aligned(out, 16)) return GWS_ERR_ALIGN;
+  const uint64_t n = static_cast<uint64_t>(desc->rows) * static_cast<uint64_t>(desc->cols);
+  if (n % 8 != 0 || desc->elem_offset % 8 != 0) return GWS_ERR_UNSUPPORTED;
+  uint32_t ctr_lo;
+  gws::PhiloxPre pre;
+  const int cst = compare_counters(desc, noise_kind, &ctr_lo, &pre);
+  if (cst != GWS_OK) return cst;
+  const uint32_t n_vec = static_cast<uint32_t>(n / 8);
+  const unsigned blocks = (n_vec + 255u) / 256u;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const uint32_t k0 = static_cast<uint32_t>(desc->seed), k1 = static_cast<uint32_t>(desc->seed >> 32);
+  if (noise_kind == gws::kNoiseUniformBf16) gws::k_compare_noise<gws::kNoiseUniformBf16><<<blocks, 256, 0, s>>>(out, n_vec, ctr_lo, k0, k1, pre);
+  else gws::k_compare_noise<gws::kNoiseBoxMuller><<<blocks, 256, 0, s>>>(out, n_vec, ctr_lo, k0, k1, pre);
+  return check_launch("comparison noise kernel");
 }
 
 int gws_philox_words(uint64_t seed, uint64_t step, uint64_t first_vec, int64_t n_vec, uint32_t* out4, void* stream) {

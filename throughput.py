@@ -1,6 +1,6 @@
 """Throughput of the sampling pass on the other workload shapes of the paper (one JSON line each).
 
-    python throughput.py [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [issue] [--reps N] [--blocks B]
+    python throughput.py [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [issue] [compare] [--reps N] [--blocks B]
 
 gpt2         all GPT2-124M linear weights, one group per row (and the same set with groups of 128)
 gpt2_single  one GPT2-124M MLP weight, both orientations
@@ -9,6 +9,8 @@ square       Llama2-1B-shaped blocks with the paper's 32 x 32 groups (Eq. 3, b_l
 llama        the Llama2-1B-shaped set with groups of 128 (the benchmark's workload; --blocks limits it)
 mx           the same set with w_hat written as MX FP8 / FP6 instead of BF16
 gemm         sampling fused into a tcgen05 GEMM against sampling + library GEMM against the plain library GEMM
+compare      forward pass with the method's noise against the same kernel shape with Box-Muller and with BF16 uniform noise
+             (the series "ours", "bm" and the DiffQ-style noise of the paper's forward benchmark), matrices of its range
 issue        cycles per warp instruction of the instruction kinds the passes are made of, and of the passes' arithmetic
              without memory traffic (gws_issue_probe): the terms of the arithmetic ceiling of the backward pass
 
@@ -134,6 +136,43 @@ def run_gemm(reps: int, dev) -> dict:
     return line
 
 
+COMPARE_SHAPES = [(2048, 512), (2048, 2048), (2048, 8192), (4096, 4096), (8192, 8192), (16384, 4096), (16384, 16384)]
+
+
+def run_compare(reps: int, dev) -> list:
+    """Forward pass (Eq. 3 + cast, groups of 128, 6 bits) in 10^9 elements per second with three noises: the method's AND / OR
+    generation, the rounded normal from Box-Muller, and BF16 uniform noise; L2 flushed between passes."""
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    lines = []
+    for rows, cols in COMPARE_SHAPES:
+        spec = syn.TensorSpec("m", rows, cols, 1, 128)
+        w, bt = syn.weights(spec, 0, device=dev), syn.bitwidths(spec, 0, fixed=6.0, device=dev)
+        d = Desc.make(rows, cols, 1, 128, seed=syn.layer_seed(0, 0))
+        w_hat, scale = torch.empty_like(w), torch.empty(spec.n_groups, device=dev)
+        calls = {"ours": lambda k: gws.sample_fwd(d.with_step(k), w, bt, w_hat, scale),
+                 "bm": lambda k: gws.sample_fwd_compare(d.with_step(k), gws.NOISE_BOX_MULLER, w, bt, w_hat, scale),
+                 "uniform_bf16": lambda k: gws.sample_fwd_compare(d.with_step(k), gws.NOISE_UNIFORM_BF16, w, bt, w_hat, scale),
+                 "copy": lambda k: w_hat.copy_(w)}
+        line = {"workload": f"forward {rows}x{cols}, groups of 128, 6 bits", "elements": rows * cols, "reps": reps}
+        for name, fn in calls.items():
+            total = 0.0
+            for k in range(3 + reps):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn(k)
+                b.record()
+                torch.cuda.synchronize()
+                if k >= 3:
+                    total += a.elapsed_time(b)
+            us = total / reps * 1e3
+            line[name + "_us"] = us
+            line[name + "_gelem_per_s"] = rows * cols / us / 1e3
+        print(json.dumps(line), flush=True)
+        lines.append(line)
+    return lines
+
+
 ISSUE_MIXES = list(range(20)) + [101, 103, 107, 109]
 _KINDS = ("mul 32x32->64", "xor3 fed by it", "lop3", "ffma", "fma.f32.bf16", "iadd", "prmt")
 _BODY = {101: "Philox4x32-10 (hoisted), per 8-element vector", 103: "Philox + gradient decode, per vector",
@@ -200,6 +239,8 @@ def main(argv=None) -> None:
             run_gemm(args.reps, dev)
         elif w == "issue":
             run_issue(args.reps, dev)
+        elif w == "compare":
+            run_compare(args.reps, dev)
         elif w == "mx":
             for fmt in (gws.MX_FP8_E4M3, gws.MX_FP6_E3M2, gws.MX_FP8_E3M4):
                 run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev, mx_format=fmt)
