@@ -20,8 +20,8 @@ import torch
 from paper_2505_11170_b200 import _build, binding
 from paper_2505_11170_b200.binding import Desc
 import os
-# the build made with the main library travels with the tree; compile only if it is missing
-binding.load_library(_build.CHECK_LIB_PATH if os.path.exists(_build.CHECK_LIB_PATH) else _build.build(self_check=True))
+# the build made with the main library travels with the tree; compiled here only if it is missing or older than its sources
+binding.load_library(_build.build(self_check=True))
 assert binding.selfcheck_enabled()
 dev = "cuda"
 arena = torch.zeros(128 << 20, dtype=torch.uint8, device=dev)
