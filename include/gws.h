@@ -504,6 +504,23 @@ const char* gws_last_cuda_error(void);
 /* Count of kernel launches the library has enqueued since load (all threads). */
 uint64_t gws_launch_count(void);
 
+/* Launch overlap (off when the library is loaded; the setting is process-wide and read at every launch).
+ *
+ * The sampling pass on a small weight set is a handful of launches of some tens of microseconds each, and every launch
+ * spends several microseconds filling the GPU and several more draining it (the per-step cost Section 3.5 counts as
+ * "separate kernels").  With the overlap enabled, the kernels of the flat-group, whole-row and square-block classes are
+ * launched with programmatic stream serialization: the blocks of a launch may become resident while the last blocks of
+ * the kernel BEFORE it on the same stream still run.  They read nothing but their kernel parameters until that kernel
+ * has completed and its writes are visible (griddepcontrol.wait stands before their first access to global memory), so
+ * every result is bit for bit that of an ordinary launch and stream order still holds between any two kernels; only the
+ * fill of one launch now overlaps the drain of the one before.  The vector and general kernels are launched as before,
+ * and so is every kernel enqueued on a stream that is recording a CUDA graph.
+ *
+ * enable: 0 = ordinary launches, anything else = overlapping launches.  Returns the previous setting (0 or 1); never
+ * fails and enqueues nothing.  A kernel of another library that follows one of these on the stream is unaffected (it is
+ * not launched with the attribute); one that precedes them is simply waited for. */
+int gws_set_launch_overlap(int enable);
+
 #ifdef __cplusplus
 }
 #endif

@@ -106,6 +106,7 @@ _SIGNATURES = {
     "gws_status_string": (c_char_p, [c_int]),
     "gws_last_cuda_error": (c_char_p, []),
     "gws_launch_count": (c_uint64, []),
+    "gws_set_launch_overlap": (c_int, [c_int]),
 }
 
 
@@ -171,6 +172,11 @@ def kernel_class(desc: Desc) -> int:
 
 def launch_count() -> int:
     return int(load_library().gws_launch_count())
+
+
+def set_launch_overlap(enable: bool) -> bool:
+    """Overlapping launches of the chunk kernels on or off (process-wide); returns the previous setting."""
+    return bool(load_library().gws_set_launch_overlap(1 if enable else 0))
 
 
 def group_absmax(desc: Desc, w: torch.Tensor, absmax: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

@@ -147,6 +147,33 @@ uint32_t mx_scales_off16(const Entry& e) {
   return static_cast<uint32_t>(mx_scales_offset(e.rows * e.cols, gws::mode_mx_format(MODE)) / 16u);
 }
 
+// ---- launches of the chunk kernels (flat groups, rows, square blocks) ----------------------------------
+
+// When set, the chunk kernels are launched with programmatic stream serialization: their blocks may become resident while
+// the last blocks of the kernel before them on the stream still run, and wait there (griddepcontrol.wait, before their first
+// access to global memory) until that kernel has completed.  Results are those of an ordinary launch; what changes is that the
+// start of one launch overlaps the end of the one before it.
+std::atomic<int> g_launch_overlap{0};
+
+template <typename Kernel, typename Batch>
+void launch_chunk_kernel(Kernel kernel, unsigned grid, unsigned block, cudaStream_t stream, const Batch& batch) {
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 0;
+  if (g_launch_overlap.load(std::memory_order_relaxed) != 0) {   // a stream that records a graph gets ordinary launches
+    cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &capture) == cudaSuccess && capture == cudaStreamCaptureStatusNone) cfg.numAttrs = 1;
+  }
+  cudaLaunchKernelEx(&cfg, kernel, batch);   // the error, if any, is read by check_launch
+}
+
 // ---- flat-group launches: tensor records by value in the kernel parameters ---------------------------
 
 gws::FlatRec to_flat_rec(const Entry& e) {
@@ -179,7 +206,7 @@ int launch_flat_batch(gws::FlatRec* recs, int count, uint32_t lo, uint32_t hi, c
   const int64_t tiles = gws::fill_flat_batch<CAP>(b, recs, count, CPT, lo, hi);
   if (tiles < 0) return GWS_ERR_LIMIT;
   if (tiles == 0) return GWS_OK;
-  gws::k_flat<MODE, VARIANT, CAP, CPT><<<static_cast<unsigned>(tiles), gws::kFlatThreads, 0, stream>>>(b);
+  launch_chunk_kernel(gws::k_flat<MODE, VARIANT, CAP, CPT>, static_cast<unsigned>(tiles), gws::kFlatThreads, stream, b);
   return check_launch("flat-group kernel");
 }
 
@@ -260,7 +287,7 @@ int launch_row_batch(const gws::RowRec* recs, int count, uint32_t lo, uint32_t h
   const int64_t tiles = gws::fill_row_batch<CAP>(b, recs, count, BLOCK, lo, hi);
   if (tiles < 0) return GWS_ERR_LIMIT;
   if (tiles == 0) return GWS_OK;
-  gws::k_row<MODE, BLOCK, CAP, MAXCPT><<<static_cast<unsigned>(tiles), gws::kRowThreads, 0, stream>>>(b);
+  launch_chunk_kernel(gws::k_row<MODE, BLOCK, CAP, MAXCPT>, static_cast<unsigned>(tiles), gws::kRowThreads, stream, b);
   return check_launch("row kernel");
 }
 
@@ -352,7 +379,7 @@ int launch_square_batch(const Entry* const* entries, int count, uint32_t lo, uin
   const int64_t tiles = gws::fill_square_batch<CAP>(b, recs, bands, count, lo, hi);
   if (tiles < 0) return GWS_ERR_LIMIT;
   if (tiles == 0) return GWS_OK;
-  gws::k_square<MODE, CAP><<<static_cast<unsigned>(tiles), gws::kFlatThreads, 0, stream>>>(b);
+  launch_chunk_kernel(gws::k_square<MODE, CAP>, static_cast<unsigned>(tiles), gws::kFlatThreads, stream, b);
   return check_launch("square-block kernel");
 }
 
@@ -1295,6 +1322,8 @@ const char* gws_status_string(int status) {
 const char* gws_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
 
 uint64_t gws_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int gws_set_launch_overlap(int enable) { return g_launch_overlap.exchange(enable != 0 ? 1 : 0, std::memory_order_relaxed); }
 
 }  // extern "C"
 

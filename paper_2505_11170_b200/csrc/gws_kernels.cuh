@@ -74,6 +74,15 @@ struct __align__(16) Entry {
 };
 static_assert(sizeof(Entry) == 112, "Entry layout");
 
+// First statement of the chunk kernels after their index arithmetic (which reads kernel parameters only) and before their
+// first access to global memory.  In a launch that was allowed to overlap the end of the kernel before it on the stream
+// (programmatic stream serialization), a block may become resident while that kernel's last blocks still run; it stops here
+// until that kernel has completed and its writes are visible.  In an ordinary launch both instructions do nothing.
+__device__ __forceinline__ void wait_for_previous_kernel() {
+  asm volatile("griddepcontrol.launch_dependents;");   // the next launch may become resident once all blocks of this one have started
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 constexpr int kFlatThreads = 256, kFlatVecs = 4;        // 1024 vectors = 16 KiB of BF16 per tile
 constexpr int kRowWarpThreads = 256, kRowWarpVecs = 16; // 8 rows per tile, <= 512 vectors per row
 constexpr int kRowCtaThreads = 512, kRowCtaVecs = 16;   // 1 row per tile, <= 8192 vectors per row
@@ -687,6 +696,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ F
   while (idx + 1 < b.n && b.e[idx + 1].tile_begin <= tile) ++idx;
   const FlatRec& e = b.e[idx];
   const uint32_t chunk = static_cast<uint32_t>(tile - e.tile_begin) * (kFlatThreads * CPT) + threadIdx.x;
+  wait_for_previous_kernel();
   if (VARIANT == kNarrow) {
     flat_narrow<MODE>(e, chunk, e.lanes_log2);
   } else {
@@ -775,6 +785,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_square(const __grid_constant__
   const uint32_t piece0 = ((band * 32u + (lane >> 2)) * cpr + blk) * 2u + half, piece_step = 16u * cpr;   // 8 rows on
   uint32_t piece[4];                              // index of the 32-byte piece in the tensor
   uint32_t x[4][8];
+  wait_for_previous_kernel();
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     piece[k] = piece0 + static_cast<uint32_t>(k) * piece_step;
@@ -940,6 +951,7 @@ __global__ void __launch_bounds__(kRowThreads) k_row(const __grid_constant__ Row
   const uint32_t row = okr ? row0 : e.rows - 1u;   // keeps warps whole for the shuffles; nothing is stored for it
   const uint32_t cpr = e.cpr, cpt = e.cpt;
   const uint32_t row_chunk0 = row * cpr;
+  wait_for_previous_kernel();
 
   Chunk c[MAXCPT];
   bool ok[MAXCPT];

@@ -193,3 +193,11 @@ def test_fused_gemm_refuses_outputs_that_overlap_inputs(lib):
     assert call(x, w, bt, y, y, null) == binding.ERR_ALIAS                                 # the two outputs on each other
     assert call(x, w, bt, y, wh, bt) == binding.ERR_ALIAS                                  # scale_out on top of bt
     assert gws.launch_count() == before
+
+
+def test_launch_overlap_setting_is_off_at_load_and_returns_the_previous_value(lib):
+    assert lib.gws_set_launch_overlap(0) == 0          # off when the library is loaded
+    assert lib.gws_set_launch_overlap(7) == 0          # any non-zero value switches it on ...
+    assert lib.gws_set_launch_overlap(1) == 1          # ... and is reported as 1
+    assert gws.set_launch_overlap(False) is True
+    assert gws.set_launch_overlap(False) is False

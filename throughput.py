@@ -17,6 +17,8 @@ issue        cycles per warp instruction of the instruction kinds the passes are
 Every timed pass is one multi-tensor launch set over the whole workload, timed with CUDA events on the launching
 stream after three warm-up passes; a 256 MiB buffer is written between passes so that no pass finds its inputs in L2.
 Bytes are the algorithmic ones (read W, write w_hat, read b_t, write scale; read grad, read scale, write grad_bt).
+With more than one repetition every workload line also times forward + backward as a pair (no event between the two)
+and as ten pairs in a row, with ordinary launches and with overlapping ones (gws_set_launch_overlap).
 """
 from __future__ import annotations
 
@@ -77,6 +79,31 @@ def run(name: str, specs, reps: int, dev, mx_format=None) -> dict:
             t_fwd += e[0].elapsed_time(e[1])
             t_bwd += e[1].elapsed_time(e[2])
     t_fwd, t_bwd = t_fwd / reps, t_bwd / reps
+
+    # forward + backward as a pair (no event between them) and as ten pairs in a row (after a flush; inside the ten the
+    # L2 holds what it can), with ordinary launches and with overlapping ones (gws_set_launch_overlap)
+    def pairs(chain: int, overlap: bool) -> float:
+        previous = gws.set_launch_overlap(overlap)
+        try:
+            total = 0.0
+            for k in range(3 + reps):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for c in range(chain):
+                    forward(k * chain + c)
+                    bwd_plan.sample_bwd_multi(k * chain + c)
+                b.record()
+                torch.cuda.synchronize()
+                if k >= 3:
+                    total += a.elapsed_time(b)
+        finally:
+            gws.set_launch_overlap(previous)
+        return total / reps / chain
+    pair = {}
+    for c in ((1, 10) if reps > 1 else ()):   # --reps 1 is what the profiler commands use: the two timed launches only
+        for o in (False, True, False, True):  # off, on, off, on: a drift of the clocks falls on both settings alike
+            pair[c, o] = pair.get((c, o), 0.0) + 0.5 * pairs(c, o)
     fwd_bytes = n * (2.0 + out_bytes) + n_groups * 8
     bwd_bytes = n * 2.0 + n_groups * 8
     peak = _peak_gbs()
@@ -84,6 +111,11 @@ def run(name: str, specs, reps: int, dev, mx_format=None) -> dict:
             "fwd_us": t_fwd * 1e3, "fwd_GB/s": fwd_bytes / t_fwd / 1e6, "fwd_frac_of_measured_hbm": fwd_bytes / t_fwd / 1e6 / peak,
             "bwd_us": t_bwd * 1e3, "bwd_GB/s": bwd_bytes / t_bwd / 1e6, "bwd_frac_of_measured_hbm": bwd_bytes / t_bwd / 1e6 / peak,
             "launches_fwd": fwd_plan.launches_per_pass, "launches_bwd": bwd_plan.launches_per_pass, "reps": reps, "l2": "flushed between passes"}
+    if pair:
+        line.update({"pair_us": pair[1, False] * 1e3, "pair_overlap_us": pair[1, True] * 1e3,
+                     "pair_in_chain_of_10_us": pair[10, False] * 1e3, "pair_in_chain_of_10_overlap_us": pair[10, True] * 1e3,
+                     "pair_frac_of_measured_hbm": (fwd_bytes + bwd_bytes) / pair[1, False] / 1e6 / peak,
+                     "pair_overlap_frac_of_measured_hbm": (fwd_bytes + bwd_bytes) / pair[1, True] / 1e6 / peak})
     print(json.dumps(line), flush=True)
     return line
 
