@@ -239,6 +239,16 @@ int gws_gemm_fused(const gws_desc* wdesc, int64_t m, const void* x, const void* 
  * exchange data only through shared-memory stores and mbarrier arrivals, every wait is bounded as above. */
 int gws_gemm_fused_cluster(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y,
                            void* w_hat_out, float* scale_out, int* status, int cluster_blocks, void* stream);
+
+/* The cluster form with 256 x 256 tiles of Y per thread block: tcgen05.mma instructions of N = 256 read a third less
+ * shared memory per unit of tensor-core work than those of N = 128 (the X operand is read once for twice the columns) and
+ * halve the number of instructions to issue; both accumulators of a block take all 512 columns of an SM's tensor memory.
+ * `cluster_blocks` (1, 2 or 4) blocks stacked along M sample 256 / cluster_blocks rows of each 256 x 128 tile of W each and
+ * store them into the shared memory of all blocks of the cluster; X arrives by TMA in steps of 64 along K (three stages).
+ * Arguments, results, bits of w_hat_out / scale_out and error behaviour as for gws_gemm_fused; wdesc->rows must be a
+ * multiple of 256 and m a multiple of 256 * cluster_blocks.  No load is multicast; every wait is bounded as above. */
+int gws_gemm_fused_wide(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y,
+                        void* w_hat_out, float* scale_out, int* status, int cluster_blocks, void* stream);
 const char* gws_gemm_last_error(void);
 /* Diagnostic: runs the fused GEMM's bounded wait on an mbarrier that nothing completes (one thread, about a
  * second).  status2: device, two ints, written: [0] = 1 (the wait gave up, as it must), [1] = SM cycles waited / 1024. */

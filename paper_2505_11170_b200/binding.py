@@ -72,6 +72,7 @@ _SIGNATURES = {
     "gws_sample_fwd_mx_multi": (c_int, [POINTER(_MultiPlan), c_int, c_uint64, c_void_p]),
     "gws_gemm_fused": (c_int, [POINTER(Desc), c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
     "gws_gemm_fused_cluster": (c_int, [POINTER(Desc), c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
+    "gws_gemm_fused_wide": (c_int, [POINTER(Desc), c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
     "gws_gemm_last_error": (c_char_p, []),
     "gws_gemm_wait_probe": (c_int, [c_void_p, c_void_p]),
     "gws_workspace_bytes": (c_size_t, [c_int]),
@@ -269,18 +270,22 @@ def sample_fwd_mx(desc: Desc, fmt: int, w: torch.Tensor, bt: torch.Tensor, mx_ou
 
 def gemm_fused(wdesc: Desc, x: torch.Tensor, w: torch.Tensor, bt: torch.Tensor, y: Optional[torch.Tensor] = None,
                w_hat_out: Optional[torch.Tensor] = None, scale_out: Optional[torch.Tensor] = None,
-               status: Optional[torch.Tensor] = None, rows_per_block: int = 512, stream=None, cluster: Optional[int] = None) -> torch.Tensor:
+               status: Optional[torch.Tensor] = None, rows_per_block: int = 512, stream=None, cluster: Optional[int] = None,
+               wide: bool = False) -> torch.Tensor:
     """Y = X @ W_hat^T with W_hat sampled inside the GEMM (never stored unless ``w_hat_out`` is given).  Returns Y.
 
     ``cluster`` = 1, 2 or 4 selects the form in which a cluster of that many thread blocks (256 rows of X each) shares
-    every sampled tile (gws_gemm_fused_cluster); otherwise ``rows_per_block`` rows of X share it inside one block."""
+    every sampled tile (gws_gemm_fused_cluster; with ``wide`` the form with 256 x 256 tiles of Y per block,
+    gws_gemm_fused_wide); otherwise ``rows_per_block`` rows of X share it inside one block."""
     _require_cuda(x, w, bt, y, w_hat_out, scale_out, status)
     if x.dim() != 2 or x.shape[1] != wdesc.cols or not x.is_contiguous() or x.dtype != torch.bfloat16:
         raise ValueError("gws: x must be a contiguous BF16 [m, k] tensor with k = cols of W")
     if y is None:
         y = torch.empty((x.shape[0], wdesc.rows), dtype=torch.bfloat16, device=x.device)
     lib = load_library()
-    fn, arg = (lib.gws_gemm_fused, rows_per_block) if cluster is None else (lib.gws_gemm_fused_cluster, cluster)
+    if wide and cluster is None:
+        raise ValueError("gws: the wide form takes a cluster size (1, 2 or 4)")
+    fn, arg = (lib.gws_gemm_fused, rows_per_block) if cluster is None else ((lib.gws_gemm_fused_wide if wide else lib.gws_gemm_fused_cluster), cluster)
     st = fn(ctypes.byref(wdesc), x.shape[0], _ptr(x), _ptr(w), _ptr(bt), _ptr(y), _ptr(w_hat_out), _ptr(scale_out),
             _ptr(status), arg, _stream(stream))
     if st != OK:

@@ -391,3 +391,23 @@ int gws_gemm_fused_cluster(const gws_desc* wdesc, int64_t m, const void* x, cons
 }
 
 }  // extern "C"
+
+#include "gws_gemm_wide.cuh"
+
+extern "C" {
+
+int gws_gemm_fused_wide(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y, void* w_hat_out,
+                        float* scale_out, int* status, int cluster_blocks, void* stream) {
+  if (cluster_blocks != 1 && cluster_blocks != 2 && cluster_blocks != 4) return wdesc == nullptr ? GWS_ERR_NULL : GWS_ERR_UNSUPPORTED;
+  if (wdesc != nullptr && wdesc->rows > 0 && wdesc->rows % kWdN != 0) return GWS_ERR_UNSUPPORTED;
+  CUtensorMap map;
+  GemmArgs args;
+  const int st = gemm_prepare(wdesc, m, x, w, bt, y, w_hat_out, scale_out, status, static_cast<int64_t>(kWdMT) * kTileM * cluster_blocks, map, args);
+  if (st != GWS_OK) return st < 0 ? st : GWS_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cluster_blocks == 1) return launch_gemm_wide<1>(map, args, m, s);
+  if (cluster_blocks == 2) return launch_gemm_wide<2>(map, args, m, s);
+  return launch_gemm_wide<4>(map, args, m, s);
+}
+
+}  // extern "C"

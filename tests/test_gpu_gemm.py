@@ -78,6 +78,29 @@ def test_cluster_form_matches_the_oracle(m, n, k, cluster):
     assert torch.equal(y.view(torch.int16), y_single.view(torch.int16))
 
 
+@pytest.mark.parametrize("m,n,k,cluster", [(256, 256, 128, 1), (512, 256, 384, 2), (1024, 512, 256, 4), (2048, 256, 512, 4),
+                                           (1024, 256, 1024, 2), (768, 512, 640, 1), (512, 768, 2048, 2)])
+def test_wide_form_matches_the_oracle(m, n, k, cluster):
+    # 256 x 256 tiles of Y per block (MMAs of N = 256), W in stages of 128 along K, X in stages of 64
+    x, w, bt = _inputs(m, n, k, m + n + k + cluster + 1)
+    d = Desc.make(n, k, 1, 128, seed=0x71DE, step=6, elem_offset=1 << 13)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    w_hat_out = torch.zeros(n, k, dtype=torch.bfloat16, device=DEV)
+    scale_out = torch.zeros(n * k // 128, device=DEV)
+    y = torch.full((m, n), float("nan"), dtype=torch.bfloat16, device=DEV)
+    gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), y=y, w_hat_out=w_hat_out, scale_out=scale_out, status=status, cluster=cluster, wide=True)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    want_hat, want_scale = orc.sample_fwd(bits_of(w), bt.numpy(), n, k, 1, 128, seed=d.seed, step=d.step, elem_offset=d.elem_offset)
+    assert np.array_equal(bits_of(w_hat_out).ravel(), want_hat)
+    assert np.array_equal(scale_out.cpu().numpy().view(np.uint32), want_scale.view(np.uint32))
+    assert not torch.isnan(y.float()).any()
+    _check_y(y.cpu(), x, f32_of_bits(want_hat).astype(np.float64).reshape(n, k))
+    y_single = gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), rows_per_block=256)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), y_single.view(torch.int16))
+
+
 def test_cluster_form_refuses_other_shapes_before_any_launch():
     lib = gws.load_library()
     buf = torch.zeros(1 << 21, dtype=torch.bfloat16, device=DEV)
@@ -89,6 +112,11 @@ def test_cluster_form_refuses_other_shapes_before_any_launch():
     assert call(Desc.make(128, 128, 1, 128), 128, 1) == binding.ERR_UNSUPPORTED
     assert call(Desc.make(128, 128, 1, 32), 256, 1) == binding.ERR_UNSUPPORTED             # group size
     assert call(Desc.make(128, 128, 1, 128), 0, 4) == binding.OK                           # nothing to do
+    wide = lambda d, m, c: lib.gws_gemm_fused_wide(ctypes.byref(d), m, p, p + (1 << 20), fp, p + (1 << 21), None, None, None, c, None)
+    assert wide(Desc.make(128, 128, 1, 128), 256, 1) == binding.ERR_UNSUPPORTED            # rows of W not a multiple of 256
+    assert wide(Desc.make(256, 128, 1, 128), 256, 2) == binding.ERR_UNSUPPORTED            # m not a multiple of 256 * 2
+    assert wide(Desc.make(256, 128, 1, 128), 256, 3) == binding.ERR_UNSUPPORTED
+    assert wide(Desc.make(256, 128, 1, 128), 0, 2) == binding.OK
 
 
 def test_fused_gemm_without_optional_outputs_gives_the_same_y():
@@ -115,9 +143,11 @@ def test_config5_up_projection_on_sampled_rows():
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     y = gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), status=status, rows_per_block=512)
     y_cluster = gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), status=status, cluster=4)
+    y_wide = gws.gemm_fused(d, x.to(DEV), w.to(DEV), bt.to(DEV), status=status, cluster=2, wide=True)
     torch.cuda.synchronize()
     assert status.item() == 0
     assert torch.equal(y.view(torch.int16), y_cluster.view(torch.int16))
+    assert torch.equal(y.view(torch.int16), y_wide.view(torch.int16))
     want_hat, _ = orc.sample_fwd(bits_of(w), bt.numpy(), n, k, 1, 128, seed=d.seed, step=0)
     rows = np.concatenate([np.arange(0, 8), np.random.default_rng(1).choice(m, 40, replace=False), np.arange(m - 8, m)])
     rows = torch.from_numpy(np.unique(rows))

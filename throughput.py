@@ -158,6 +158,11 @@ def run_gemm(reps: int, dev) -> dict:
         line[f"fused_{rpb}_rows_per_block_us"] = timed(lambda i: gws.gemm_fused(d.with_step(i), x, w, bt, y=y, status=status, rows_per_block=rpb))
     for c in (1, 2, 4):
         line[f"fused_cluster_of_{c}_us"] = timed(lambda i: gws.gemm_fused(d.with_step(i), x, w, bt, y=y, status=status, cluster=c))
+    for c in (1, 2, 4):
+        line[f"fused_wide_cluster_of_{c}_us"] = timed(lambda i: gws.gemm_fused(d.with_step(i), x, w, bt, y=y, status=status, cluster=c, wide=True))
+    best_wide = min(line[f"fused_wide_cluster_of_{c}_us"] for c in (1, 2, 4))
+    line["fused_wide_best_TFLOP/s"] = line["flops"] / (best_wide * 1e-6) / 1e12
+    line["overhead_fused_wide_best_pct"] = 100.0 * (best_wide / line["plain_gemm_us"] - 1.0)
     line["status"] = int(status.item())
     line["fused_TFLOP/s"] = line["flops"] / (line["fused_512_rows_per_block_us"] * 1e-6) / 1e12
     line["fused_cluster_of_4_TFLOP/s"] = line["flops"] / (line["fused_cluster_of_4_us"] * 1e-6) / 1e12
