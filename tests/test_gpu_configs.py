@@ -2,8 +2,8 @@
 (one multi-tensor launch per kernel class), against the oracle.  Whole weight sets and whole matrices are
 compared element by element and group by group: the oracle runs as one single-threaded process per host
 core over disjoint tensors or row bands (oracle/pool.py; a row band with elem_offset = first_row * cols
-reproduces the noise stream of the full tensor).  Only the 28672 x 8192 matrix of the stress sweep and the
-intermediate step counters of the ten-step run are checked on row slices."""
+reproduces the noise stream of the full tensor).  Only the intermediate step counters of the ten-step run and the MX
+outputs are checked on row slices."""
 import numpy as np
 import pytest
 import torch
@@ -148,7 +148,6 @@ def test_config3_llama2_1b_ten_steps_whole_set_at_steps_0_and_9():
 @pytest.mark.parametrize("shape", syn.STRESS_SHAPES)
 def test_config4_stress_sweep(shape):
     rows, cols = shape
-    rng = np.random.default_rng(rows)
     case = 0
     for sigma in syn.STRESS_SIGMAS:
         base = syn.TensorSpec("stress", rows, cols, 1, 0)
@@ -164,14 +163,9 @@ def test_config4_stress_sweep(shape):
                 _, sc = gws.sample_fwd(d, w, bt, w_hat=w_hat)
                 _, gbt = gws.sample_bwd(d, g, sc)
                 torch.cuda.synchronize()
-                if rows * cols <= (1 << 26):
-                    # 4096^2 and 8192^2: the whole matrix, cut into row bands for the oracle processes
-                    with OraclePool() as pool:
-                        assert _whole_check(pool, [spec], [d.seed], case, [w], [bt], [w_hat], [sc], [g], [gbt]) == rows * cols
-                else:
-                    nrows = 8
-                    for r0 in (0, rows - nrows, int(rng.integers(0, rows - nrows))):
-                        _slice_check(spec, d.seed, case, w, bt, w_hat, sc, g, gbt, r0, nrows)
+                # the whole matrix (up to 234,881,024 elements), cut into row bands for the oracle processes
+                with OraclePool() as pool:
+                    assert _whole_check(pool, [spec], [d.seed], case, [w], [bt], [w_hat], [sc], [g], [gbt]) == rows * cols
                 # the outliers are there and the absmax sees them
                 am = gws.group_absmax(d, w)
                 assert float(am.max()) >= 7.9 * sigma
@@ -179,7 +173,7 @@ def test_config4_stress_sweep(shape):
 
 def test_config5_sample_then_gemm_unfused():
     # Up-projection of the Llama2-1B shape: W 5632 x 2048 (rows = outputs), groups of 128, 6 bits; X 16384 x 2048.
-    # The sampled weight is checked bit for bit on row slices; Y = X W_hat^T (the stock BF16 GEMM the paper keeps) is
+    # The sampled weight is checked bit for bit, whole; Y = X W_hat^T (the stock BF16 GEMM the paper keeps) is
     # checked on sampled outputs against a float64 dot product with the oracle's W_hat.
     spec = syn.TensorSpec("up", 5632, 2048, 1, 128)
     w = syn.weights(spec, 0, device=DEV)
@@ -190,8 +184,9 @@ def test_config5_sample_then_gemm_unfused():
     y = torch.matmul(x, w_hat.t())
     torch.cuda.synchronize()
     rng = np.random.default_rng(5)
-    for r0 in (0, spec.rows - 16, int(rng.integers(0, spec.rows - 16))):
-        _slice_check(spec, d.seed, 0, w, bt, w_hat, sc, None, None, r0, 16)
+    hat_all, sc_all = orc.sample_fwd(bits_of(w), bt.cpu().numpy(), spec.rows, spec.cols, 1, 128, seed=d.seed, step=0)
+    assert np.array_equal(bits_of(w_hat).ravel(), hat_all)                      # all 11,534,336 elements
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), sc_all.view(np.uint32))
     rows = sorted({0, spec.rows - 1, *[int(v) for v in rng.integers(0, spec.rows, 6)]})
     for n in rows:
         hat, _ = orc.sample_fwd(bits_of(w[n:n + 1]), bt[n * 16:(n + 1) * 16].cpu().numpy(), 1, spec.cols, 1, 128, seed=d.seed,
