@@ -489,6 +489,11 @@ def main():
                 gws.sample_bwd(d, G[i], SC[i], None, GBT[i], stream=stream)
 
         per_layer_ms = timed(per_layer, 5)
+        previous_overlap = gws.set_launch_overlap(True)     # the same 308 launches, each allowed to start while the one before drains
+        try:
+            per_layer_overlap_ms = timed(per_layer, 5)
+        finally:
+            gws.set_launch_overlap(previous_overlap)
         GW = [torch.empty_like(t) for t in G]
         copy_plan = gws.MultiPlan(descs, scale=SC, grad_w_hat=G, grad_w=GW, grad_bt=GBT)
         bwd_copy_ms = timed(lambda k: copy_plan.sample_bwd_multi(k), 10)
@@ -531,7 +536,9 @@ def main():
                                         "bwd_GB/s": sh_elems * BWD_BYTES_PER_ELEM / (sh_bwd_ms * 1e-3) / 1e9,
                                         "note": "each pass reads %.2f GB, more than L2; a real job adds two all-reduces of %d floats" % (sh_elems * 2 / 1e9, len(specs) * (shard_world + 1))},
             "per_layer_launches": {"ms_per_pass": per_layer_ms, "launches_per_pass": 2 * len(specs),
-                                   "GB/s": bytes_per_pass / (per_layer_ms * 1e-3) / 1e9},
+                                   "GB/s": bytes_per_pass / (per_layer_ms * 1e-3) / 1e9,
+                                   "ms_per_pass_overlapping_launches": per_layer_overlap_ms,
+                                   "GB/s_overlapping_launches": bytes_per_pass / (per_layer_overlap_ms * 1e-3) / 1e9},
             "bwd_with_grad_w_copy": {"ms_per_launch": bwd_copy_ms, "GB/s": n_elem * (4 + 8 / 128) / (bwd_copy_ms * 1e-3) / 1e9,
                                      "bytes_per_element": 4 + 8 / 128},
             "arithmetic_budget": alu,
