@@ -7,22 +7,29 @@
 // columns of FP32) take all 512 columns of tensor memory.
 //
 // A cluster is C blocks stacked along M (C = 1, 2, 4).  Per 128 elements along K (one sampling group per row of W) every
-// block samples 256 / C rows of the 256-row tile of W and stores them with st.async into the shared memory of all blocks
-// of the cluster; X arrives by TMA in steps of 64 along K.  Shared memory: two stages of W (256 rows x 128 along K = 64 KiB
-// each, as two 128-byte-swizzled halves of 64 along K) and three stages of X (2 x 128 rows x 64 along K = 32 KiB each).
-// Roles as in the cluster form: 16 sampling warps, a TMA thread, a relay thread (waits for the bytes of a W stage, fences
-// the generic-proxy stores against the tensor core's async-proxy reads), two MMA-issuing threads (one per accumulator).
+// block samples 256 / C rows of the 256-row tile of W into its OWN shared memory (64-byte chunks per thread, plain stores:
+// the arithmetic of the flat-group forward kernel), and one thread then copies that share into the same place of every
+// other block of the cluster with cp.async.bulk (shared memory to shared memory of the cluster, signalling the bytes on the
+// destination's mbarrier); X arrives by TMA in steps of 64 along K.  Shared memory: two stages of W (256 rows x 128 along
+// K = 64 KiB each, as two 128-byte-swizzled halves of 64 along K) and three stages of X (2 x 128 rows x 64 along K = 32 KiB
+// each).  Roles: 16 sampling warps, a TMA thread, a relay thread (waits for the block's own share, fences the generic-proxy
+// stores against async-proxy reads, starts the bulk copies, waits for the other blocks' shares, hands the stage to the
+// tensor core), two MMA-issuing threads (one per accumulator).
 //
-// What it showed (B200, 16384 x 2048 by 5632 x 2048): 595-601 us for clusters of 2 against 617 us for the 128-column form,
-// so shared-memory bandwidth and instruction issue were not what held that form back.  Cycle stamps in a copy of this
-// kernel: of the 122,000 cycles a block spends on its tile, the 16 steps of 128 along K take 98,000 (6,100 each against
-// 2,048 of tensor-core work), and for 44 % of them the MMA threads wait for W: sampling a block's share of a stage (2,048
-// vectors for clusters of 2) takes the 16 sampling warps 4,900 cycles, about 2.4 cycles per element and SM, which is what
-// the integer pipes of an SM deliver for Philox4x32-10 plus the decode with this code around them.  First operands are
-// ready 10,000 cycles after the block starts, the epilogue takes 10,000 and the last cluster barrier 3,000.
+// What it showed (B200, 16384 x 2048 by 5632 x 2048): 593 us for clusters of 2 against 617 us for the 128-column form, so
+// shared-memory bandwidth and instruction issue were not what held that form back; and an earlier version of this kernel
+// whose sampling threads stored every vector into every block with st.async (twice the sampling cost per stage) took
+// 595 us, so the sampling rate is not it either.  Cycle stamps in a copy of this kernel: a block spends about 120,000 cycles
+// on its tile, 95,000 of them in the 16 steps of 128 along K (5,900 each against 2,048 of tensor-core work).  A stage of W
+// goes round in about 12,000 cycles (wait for the tensor cores of every block of the cluster to release it, sample 4,300,
+// fence and copy 2,000 to 3,000, two MMA steps 2,500), and only two such stages fit beside three of X in 227 KiB: the
+// tensor core is fed a third of the time.  First operands are ready 10,000 cycles after the block starts, the epilogue
+// takes 10,000 and the last cluster barrier 3,000 to 4,000.
 //
-// No load is multicast.  Every mbarrier wait is bounded; a wait that runs out sets the status word and the block skips the
-// rest of its work.  No block leaves before all blocks of its cluster have passed the final cluster barrier.
+// No load from global memory is multicast and no TMA load touches another block's memory: the only transfers between blocks
+// are the bulk copies from a block's own shared memory, and the multicast of tcgen05.commit.  Every mbarrier wait is bounded;
+// a wait that runs out sets the status word and the block skips the rest of its work.  No block leaves before all blocks of
+// its cluster have passed the final cluster barrier.
 #pragma once
 
 namespace {
@@ -68,7 +75,7 @@ __global__ void __launch_bounds__(kClThreads, 1) k_gemm_wide(const __grid_consta
   const uint32_t raw = smem_u32(smem_raw);
   uint8_t* smem_x = smem_raw + (((raw + 1023u) & ~1023u) - raw);   // the same offset in every block of the cluster
   uint8_t* smem_w = smem_x + kWdStagesX * kWdStageXBytes;
-  __shared__ uint64_t x_full[kWdStagesX], x_empty[kWdStagesX], w_full[kWdStagesW], w_ready[kWdStagesW], w_empty[kWdStagesW], acc_full;
+  __shared__ uint64_t x_full[kWdStagesX], x_empty[kWdStagesX], w_full[kWdStagesW], w_ready[kWdStagesW], w_empty[kWdStagesW], w_local[kWdStagesW], acc_full;
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int failed;
 
@@ -91,6 +98,7 @@ __global__ void __launch_bounds__(kClThreads, 1) k_gemm_wide(const __grid_consta
       mbar_init(&w_full[s], 1);
       mbar_init(&w_ready[s], 1);
       mbar_init(&w_empty[s], kWdMT * C);
+      mbar_init(&w_local[s], kClSamplerWarps);   // one arrival per sampling warp: this block's share of the stage is in its own shared memory
     }
     mbar_init(&acc_full, kWdMT);
     failed = 0;
@@ -108,53 +116,75 @@ __global__ void __launch_bounds__(kClThreads, 1) k_gemm_wide(const __grid_consta
   uint32_t copies_started = 0;
 
   if (warp < kClSamplerWarps) {
-    // ---- samplers: rows [rank * 256 / C, (rank + 1) * 256 / C) of the W tile; a thread takes 16-byte vectors (8 elements, one
-    // Philox call), the 16 lanes of a row form its group of 128.  (Whole 64-byte chunks per thread, as in the flat-group
-    // kernel, were measured too: a stage is complete only when its slowest thread is, and the longer per-thread chain made
-    // every stage later: 887 us against 595 us for clusters of 2.) ----
+    // ---- samplers: rows [rank * 256 / C, (rank + 1) * 256 / C) of the W tile into this block's OWN shared memory with plain
+    // stores; the relay thread then copies the share to the other blocks of the cluster in bulk.  A thread takes kVecs
+    // neighbouring 16-byte vectors of a row (4 = a 64-byte chunk for C <= 2, 2 for C = 4), 16 / kVecs lanes form the group ----
     constexpr uint32_t kRowsPerBlock = static_cast<uint32_t>(kWdN) / C;
-    constexpr uint32_t kVecsPerThread = kRowsPerBlock * 16u / kSamplers;   // 8 (C = 1), 4, 2
-    uint32_t r[kVecsPerThread], vec0[kVecsPerThread], grp0[kVecsPerThread];
-    uint4 w_next[kVecsPerThread];
-    float bt_next[kVecsPerThread];
-    const uint32_t unit = tid & 15u;             // which 16 bytes of the row's 256; units 0..7 are the first half along K
+    constexpr uint32_t kVecs = C == 4 ? 2u : 4u;
+    constexpr uint32_t kLanesPerRow = 16u / kVecs;                       // 4 or 8
+    constexpr uint32_t kRowsPerPass = kSamplers / kLanesPerRow;          // 128 or 64
+    constexpr uint32_t kItems = kRowsPerBlock / kRowsPerPass;            // 2 (C = 1), 1, 1
+    static_assert(kItems * kRowsPerPass == kRowsPerBlock, "share of the tile");
+    const uint32_t part = tid % kLanesPerRow, unit0 = part * kVecs;      // first 16-byte unit of the row's 16
+    uint32_t r[kItems], vec0[kItems], grp0[kItems];
+    uint32_t x_next[kItems][4 * kVecs];
+    float bt_next[kItems];
+    auto load_item = [&](uint32_t (&x)[4 * kVecs], uint32_t vec) {
 #pragma unroll
-    for (uint32_t q = 0; q < kVecsPerThread; ++q) {
-      r[q] = rank * kRowsPerBlock + q * (kSamplers / 16u) + (tid >> 4);
+      for (uint32_t h = 0; h < kVecs / 2u; ++h) {
+        const gws::Vec32 v = gws::ld_vec32(a.w, static_cast<uint64_t>(vec + 2u * h) * 16u);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[8 * h + i] = v.v[i];
+      }
+    };
+#pragma unroll
+    for (uint32_t q = 0; q < kItems; ++q) {
+      r[q] = rank * kRowsPerBlock + q * kRowsPerPass + tid / kLanesPerRow;
       const uint32_t row = n0 + r[q];
-      vec0[q] = (row * a.k) / 8u + unit;         // pair j: + 16 * j
+      vec0[q] = (row * a.k) / 8u + unit0;        // pair j: + 16 * j
       grp0[q] = row * pairs;                     // pair j: + j
-      w_next[q] = gws::ld_vec(a.w, vec0[q]);
+      load_item(x_next[q], vec0[q]);
       bt_next[q] = gws::ld_f32(a.bt, grp0[q]);
     }
     for (uint32_t j = 0; j < pairs; ++j) {
       const uint32_t s = j % kWdStagesW;
       if (j >= kWdStagesW && !mbar_wait_cluster<true>(&w_empty[s], ((j / kWdStagesW) - 1u) & 1u)) failed = 1;
       if (__any_sync(0xFFFFFFFFu, failed != 0)) break;   // a whole warp stays or leaves: the shuffles below need all lanes
-      const uint32_t stage_w = smem_u32(smem_w + s * kWdStageWBytes), bar = smem_u32(&w_full[s]);
+      uint8_t* stage_w = smem_w + s * kWdStageWBytes;
 #pragma unroll
-      for (uint32_t q = 0; q < kVecsPerThread; ++q) {
+      for (uint32_t q = 0; q < kItems; ++q) {
         const uint32_t vec = vec0[q] + 16u * j;
-        const uint4 wv = w_next[q];
+        uint32_t x[4 * kVecs];
+#pragma unroll
+        for (uint32_t i = 0; i < 4 * kVecs; ++i) x[i] = x_next[q][i];
         const float bits = bt_next[q];
         if (j + 1u < pairs) {
-          w_next[q] = gws::ld_vec(a.w, vec + 16u);
+          load_item(x_next[q], vec + 16u);
           bt_next[q] = gws::ld_f32(a.bt, grp0[q] + j + 1u);
         }
-        uint32_t m = gws::absmax_vec(wv);
+        uint32_t m = gws::absmax_words4(x);
 #pragma unroll
-        for (uint32_t o = 1; o < 16u; o <<= 1) m = gws::maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        for (uint32_t i = 1; i < kVecs; ++i) m = gws::maxabs2(m, gws::absmax_words4(x + 4 * i));
+#pragma unroll
+        for (uint32_t o = 1; o < kLanesPerRow; o <<= 1) m = gws::maxabs2(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
         const gws::Scale sc = gws::make_scale(__fmul_rn(gws::absmax_finish(m), gws::pow2_one_minus(bits)));
-        const uint4 y = gws::sample_vec(wv, gws::philox4x32_10_pre(a.vec_lo + vec, a.k0, a.k1, a.pre), sc);
-        const uint32_t dst = stage_w + (unit >> 3) * kWdHalfWBytes + (r[q] >> 3) * 1024u + (r[q] & 7u) * 128u + (((unit & 7u) ^ (r[q] & 7u)) << 4);
+        uint32_t y[4 * kVecs];
+        if (kVecs == 4u) gws::sample_chunk(x, a.vec_lo + vec, a.k0, a.k1, a.pre, sc, y);
+        else gws::sample_half(x, a.vec_lo + vec, a.k0, a.k1, a.pre, sc, y);
+        uint8_t* row_base = stage_w + (unit0 >> 3) * kWdHalfWBytes + (r[q] >> 3) * 1024u + (r[q] & 7u) * 128u;
 #pragma unroll
-        for (uint32_t d = 0; d < static_cast<uint32_t>(C); ++d)
-          st_async_v4(C > 1 ? map_to_rank(dst, d) : dst, C > 1 ? map_to_rank(bar, d) : bar, y.x, y.y, y.z, y.w);
+        for (uint32_t i = 0; i < kVecs; ++i)
+          *reinterpret_cast<uint4*>(row_base + ((((unit0 + i) & 7u) ^ (r[q] & 7u)) << 4)) = make_uint4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
         if (blockIdx.y < static_cast<uint32_t>(C)) {   // the first cluster along M exports the sampled weights
-          if (a.w_hat_out != nullptr) gws::st_vec(a.w_hat_out, vec, y);
-          if (a.scale_out != nullptr && unit == 0u) gws::st_f32(a.scale_out, grp0[q] + j, sc.s);
+          if (a.w_hat_out != nullptr) {
+#pragma unroll
+            for (uint32_t h = 0; h < kVecs / 2u; ++h) gws::st_vec32(a.w_hat_out, static_cast<uint64_t>(vec + 2u * h) * 16u, y + 8 * h);
+          }
+          if (a.scale_out != nullptr && part == 0u) gws::st_f32(a.scale_out, grp0[q] + j, sc.s);
         }
       }
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&w_local[s])) : "memory");
     }
   } else if (warp == kClSamplerWarps) {
     // ---- X by TMA: a stage is kWdMT tiles of 128 rows x 64 along K ----
@@ -201,13 +231,33 @@ __global__ void __launch_bounds__(kClThreads, 1) k_gemm_wide(const __grid_consta
       else mma_commit(&acc_full);
     }
   } else if (warp == kClSamplerWarps + 2) {
-    // ---- W relay ----
+    // ---- W relay: when this block's share of a stage is complete in its own shared memory, orders those generic-proxy stores
+    // before async-proxy reads, copies the share in bulk into the same place of every other block of the cluster (two copies per
+    // block: the share is contiguous in each half along K), waits for the other blocks' shares and hands the stage on ----
     if (lane == 0) {
+      constexpr uint32_t kRowsPerBlock = static_cast<uint32_t>(kWdN) / C;
+      constexpr uint32_t kShareBytes = kRowsPerBlock * 128u;    // per half along K
       for (uint32_t j = 0; j < pairs; ++j) {
         const uint32_t s = j % kWdStagesW, ph = (j / kWdStagesW) & 1u;
-        mbar_expect_tx(&w_full[s], kWdStageWBytes);
-        if (!mbar_wait_cluster<false>(&w_full[s], ph)) { failed = 1; break; }
+        if (C > 1) mbar_expect_tx(&w_full[s], (C - 1) * 2u * kShareBytes);
+        if (!mbar_wait(&w_local[s], ph)) { failed = 1; break; }
         asm volatile("fence.proxy.async;" ::: "memory");
+        if (C > 1) {
+          const uint32_t src0 = smem_u32(smem_w + s * kWdStageWBytes) + rank * kShareBytes, bar = smem_u32(&w_full[s]);
+#pragma unroll
+          for (uint32_t d = 0; d < static_cast<uint32_t>(C); ++d) {
+            if (d == rank) continue;
+            const uint32_t rbar = map_to_rank(bar, d);
+#pragma unroll
+            for (uint32_t h = 0; h < 2; ++h) {
+              const uint32_t src = src0 + h * kWdHalfWBytes;
+              asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(map_to_rank(src, d)),
+                           "r"(src), "r"(kShareBytes), "r"(rbar)
+                           : "memory");
+            }
+          }
+          if (!mbar_wait_cluster<false>(&w_full[s], ph)) { failed = 1; break; }
+        }
         asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&w_ready[s])) : "memory");
       }
     }
