@@ -243,8 +243,9 @@ int gws_gemm_fused_cluster(const gws_desc* wdesc, int64_t m, const void* x, cons
 /* The cluster form with 256 x 256 tiles of Y per thread block: tcgen05.mma instructions of N = 256 read a third less
  * shared memory per unit of tensor-core work than those of N = 128 (the X operand is read once for twice the columns) and
  * halve the number of instructions to issue; both accumulators of a block take all 512 columns of an SM's tensor memory.
- * `cluster_blocks` (1, 2 or 4) blocks stacked along M sample 256 / cluster_blocks rows of each 256 x 128 tile of W each and
- * store them into the shared memory of all blocks of the cluster; X arrives by TMA in steps of 64 along K (three stages).
+ * `cluster_blocks` (1, 2 or 4) blocks stacked along M sample 256 / cluster_blocks rows of each 256 x 128 tile of W each, into
+ * their own shared memory, and copy that share in bulk into the shared memory of the other blocks of the cluster; X arrives
+ * by TMA in steps of 64 along K (three stages).
  * Arguments, results, bits of w_hat_out / scale_out and error behaviour as for gws_gemm_fused; wdesc->rows must be a
  * multiple of 256 and m a multiple of 256 * cluster_blocks.  No load is multicast; every wait is bounded as above. */
 int gws_gemm_fused_wide(const gws_desc* wdesc, int64_t m, const void* x, const void* w, const float* bt, void* y,
