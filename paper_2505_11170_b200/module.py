@@ -45,6 +45,19 @@ class _SampledWeight(torch.autograd.Function):
         return g, grad_bi, None, None, None, None, None
 
 
+class _PresampledWeight(torch.autograd.Function):
+    """w -> the w_hat a GaussWSSet has already written for this update; dL/dw = dL/dw_hat (Eq. 4).  The gradient of b_i is
+    formed once per update by GaussWSSet.finish_backward from the accumulated dL/dw."""
+
+    @staticmethod
+    def forward(ctx, w, w_hat):
+        return w_hat.view_as(w_hat)
+
+    @staticmethod
+    def backward(ctx, grad_w_hat):
+        return grad_w_hat, None
+
+
 class GaussWSLinear(torch.nn.Module):
     """Linear layer trained with Gaussian weight sampling.
 
@@ -67,6 +80,7 @@ class GaussWSLinear(torch.nn.Module):
         self.seed = binding.layer_seed(user_seed, layer_index)
         self.step = 0
         self._update = {"lambda_term_due": True}
+        self._set = None
         n_groups = binding.n_groups(self._desc())
         self.b_i = torch.nn.Parameter(torch.ones(n_groups, dtype=torch.float32, device=device))   # Eq. 11: starts at 1
 
@@ -79,6 +93,8 @@ class GaussWSLinear(torch.nn.Module):
         self._update["lambda_term_due"] = True
 
     def sampled_weight(self) -> torch.Tensor:
+        if self._set is not None:                       # sampled together with the other layers of a GaussWSSet
+            return _PresampledWeight.apply(self.weight, self._set.w_hat_of(self))
         return _SampledWeight.apply(self.weight, self.b_i, self._desc(), self.b_init, self.b_target, self.lam, self._update)
 
     def bitwidth(self) -> torch.Tensor:
@@ -90,3 +106,105 @@ class GaussWSLinear(torch.nn.Module):
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
         return torch.nn.functional.linear(x, self.sampled_weight(), self.bias)
+
+
+class GaussWSSet:
+    """All GaussWSLinear layers of a model sampled together: the whole sampling pass of an update is one multi-tensor
+    launch set forward (gws_sample_fwd_multi) and one backward (gws_sample_bwd_multi) instead of two launches per layer.
+
+        layers = [m for m in model.modules() if isinstance(m, GaussWSLinear)]
+        sampler = GaussWSSet(layers)
+        for each update:
+            sampler.sample()                    # Eq. 11 per layer, then Eq. 3 + cast for every layer at once
+            for each micro-batch: loss(model(x)).backward()      # dL/dw accumulates in weight.grad (dL/dw = dL/dw_hat)
+            sampler.finish_backward()           # Eq. 4 for every layer at once, then Eq. 11 / Eq. 12 into b_i.grad
+            optimizer.step(); optimizer.zero_grad(); sampler.advance()
+
+    Eq. 4's sum is linear in dL/dw_hat and all micro-batches of an update share R and the scale, so dL/db_t is taken once,
+    from the accumulated weight.grad, instead of once per micro-batch (with one micro-batch the two are the same numbers; with
+    several, weight.grad carries the BF16 rounding of its accumulation).  The Eq. 12 term is added once per
+    update.  The layers keep their parameters; the set owns the sampled weights, bit-widths, scales and dL/db_t buffers.
+    Every step of the pass runs in the library's kernels; this class only holds tensors and the launch plans.
+    """
+
+    def __init__(self, layers):
+        self.layers = list(layers)
+        if not self.layers:
+            raise ValueError("gws: a GaussWSSet needs at least one layer")
+        for layer in self.layers:
+            if layer._set is not None:
+                raise ValueError("gws: a layer belongs to one GaussWSSet at most")
+        dev = self.layers[0].weight.device
+        self._w_hat = [torch.empty_like(l.weight) for l in self.layers]
+        self._bt = [torch.empty(l.b_i.numel(), dtype=torch.float32, device=dev) for l in self.layers]
+        self._scale = [torch.empty_like(t) for t in self._bt]
+        self._grad_bt = [torch.empty_like(t) for t in self._bt]
+        self._index = {id(l): k for k, l in enumerate(self.layers)}
+        self._fwd_plan = None
+        self._fwd_key = None
+        self._bwd_plan = None
+        self._bwd_key = None
+        self._sampled_step = None
+        for layer in self.layers:
+            layer._set = self
+
+    def _descs(self):
+        return [l._desc() for l in self.layers]
+
+    def w_hat_of(self, layer) -> torch.Tensor:
+        if self._sampled_step != self._step():
+            raise RuntimeError("gws: call GaussWSSet.sample() once per update before the forward passes")
+        return self._w_hat[self._index[id(layer)]]
+
+    def _step(self) -> int:
+        steps = {l.step for l in self.layers}
+        if len(steps) != 1:
+            raise RuntimeError("gws: the layers of a GaussWSSet advance together (GaussWSSet.advance)")
+        return steps.pop()
+
+    def sample(self, stream=None) -> None:
+        """Eq. 11 for every layer, then Eq. 3 + the BF16 cast for all of them in one launch per kernel class."""
+        step = self._step()
+        for layer, bt in zip(self.layers, self._bt):
+            binding.bitwidth(layer.b_i.detach(), layer.b_init, layer.b_target, bt=bt, stream=stream)
+        key = tuple(l.weight.data_ptr() for l in self.layers)
+        if key != self._fwd_key:                        # the plan holds the addresses of the weights
+            self._fwd_plan = binding.MultiPlan(self._descs(), w=[l.weight.detach() for l in self.layers], bt=self._bt, w_hat=self._w_hat,
+                                               scale=self._scale, stream=stream)
+            self._fwd_key = key
+        self._fwd_plan.sample_fwd_multi(step, stream=stream)
+        self._sampled_step = step
+
+    def finish_backward(self, stream=None) -> None:
+        """Eq. 4 for every layer from the accumulated dL/dw (one launch per kernel class), then Eq. 11 / Eq. 12: adds
+        dL'/db_i of this update to every layer's ``b_i.grad``.  Call once per update, after the last backward pass."""
+        step = self._step()
+        if self._sampled_step != step:
+            raise RuntimeError("gws: finish_backward() belongs to the update that sample() started")
+        grads = []
+        for layer in self.layers:
+            g = layer.weight.grad
+            if g is None or not g.is_contiguous() or g.dtype != torch.bfloat16:
+                raise RuntimeError("gws: every layer needs a contiguous BF16 weight.grad before finish_backward()")
+            grads.append(g)
+        key = tuple(g.data_ptr() for g in grads)
+        if key != self._bwd_key:                        # the plan holds the addresses of the gradients
+            self._bwd_plan = binding.MultiPlan(self._descs(), scale=self._scale, grad_w_hat=grads, grad_bt=self._grad_bt, stream=stream)
+            self._bwd_key = key
+        self._bwd_plan.sample_bwd_multi(step, stream=stream)
+        for layer, bt, grad_bt in zip(self.layers, self._bt, self._grad_bt):
+            grad_bi = binding.bitwidth_grad(grad_bt, bt, layer.b_init, layer.b_target, layer.lam, stream=stream)
+            if layer.b_i.grad is None:
+                layer.b_i.grad = grad_bi
+            else:
+                layer.b_i.grad.add_(grad_bi)
+
+    def advance(self) -> None:
+        """One gradient update has been applied to every layer: the next sample() draws new noise."""
+        for layer in self.layers:
+            layer.advance()
+
+    @property
+    def launches_per_pass(self) -> int:
+        return self._fwd_plan.launches_per_pass if self._fwd_plan is not None else 0
+

@@ -1,6 +1,6 @@
 """Throughput of the sampling pass on the other workload shapes of the paper (one JSON line each).
 
-    python throughput.py [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [issue] [compare] [--reps N] [--blocks B]
+    python throughput.py [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [issue] [compare] [module] [--reps N] [--blocks B]
 
 gpt2         all GPT2-124M linear weights, one group per row (and the same set with groups of 128)
 gpt2_single  one GPT2-124M MLP weight, both orientations
@@ -11,6 +11,7 @@ mx           the same set with w_hat written as MX FP8 / FP6 instead of BF16
 gemm         sampling fused into a tcgen05 GEMM against sampling + library GEMM against the plain library GEMM
 compare      forward pass with the method's noise against the same kernel shape with Box-Muller and with BF16 uniform noise
              (the series "ours", "bm" and the DiffQ-style noise of the paper's forward benchmark), matrices of its range
+module       the sampling part of an update through the module wrappers: layer by layer against all layers at once (GaussWSSet)
 issue        cycles per warp instruction of the instruction kinds the passes are made of, and of the passes' arithmetic
              without memory traffic (gws_issue_probe): the terms of the arithmetic ceiling of the backward pass
 
@@ -246,6 +247,60 @@ def run_issue(reps: int, dev) -> list:
     return lines
 
 
+def run_module(reps: int, dev, n_blocks: int) -> dict:
+    """The module wrappers on the Llama2-1B-shaped layer set (the paper's 32 x 32 groups): the sampling part of an update
+    (Eq. 11, Eq. 3 forward; Eq. 4, Eq. 11 / Eq. 12 backward) layer by layer, as GaussWSLinear does on its own, against all
+    layers at once through GaussWSSet.  No GEMMs: weight.grad is filled with synthetic gradients.  Host time included (events
+    on the stream around the Python calls)."""
+    from paper_2505_11170_b200.module import GaussWSLinear, GaussWSSet
+    specs = syn.llama2_1b(n_blocks=n_blocks)
+
+    def build():
+        layers = [GaussWSLinear(s.cols, s.rows, bias=False, group=(32, 32), lam=0.1, layer_index=k, device=dev) for k, s in enumerate(specs)]
+        for k, (layer, s) in enumerate(zip(layers, specs)):
+            layer.weight.grad = syn.upstream_grad(s, k, device=dev)
+        return layers
+    alone, together = build(), build()
+    sampler = GaussWSSet(together)
+
+    def timed(fn):
+        total = 0.0
+        for i in range(3 + reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                total += a.elapsed_time(b)
+        return total / reps
+
+    def alone_fwd():
+        for layer in alone:
+            layer.sampled_weight()
+
+    saved = []
+    for layer in alone:                                   # what a layer's forward pass keeps for its backward pass
+        bt = layer.bitwidth()
+        saved.append((bt, gws.sample_fwd(layer._desc(), layer.weight.detach(), bt)[1]))
+
+    def alone_bwd():
+        for layer, (bt, scale) in zip(alone, saved):
+            _, grad_bt = gws.sample_bwd(layer._desc(), layer.weight.grad, scale)
+            gws.bitwidth_grad(grad_bt, bt, layer.b_init, layer.b_target, layer.lam)
+    n = syn.total_elements(specs)
+    with torch.no_grad():
+        fwd_alone = timed(alone_fwd)
+    bwd_alone = timed(alone_bwd)
+    fwd_set = timed(sampler.sample)
+    bwd_set = timed(sampler.finish_backward)
+    line = {"workload": f"module wrappers, llama2_1b {n_blocks} blocks, 32x32 groups", "layers": len(specs), "elements": n,
+            "forward_layer_by_layer_ms": fwd_alone, "forward_set_ms": fwd_set, "backward_layer_by_layer_ms": bwd_alone, "backward_set_ms": bwd_set,
+            "launches_per_pass_set": sampler.launches_per_pass, "reps": reps}
+    print(json.dumps(line), flush=True)
+    return line
+
+
 def main(argv=None) -> None:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("which", nargs="*", default=["gpt2", "stress"])
@@ -274,6 +329,8 @@ def main(argv=None) -> None:
             run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev)
         elif w == "gemm":
             run_gemm(args.reps, dev)
+        elif w == "module":
+            run_module(args.reps, dev, args.blocks)
         elif w == "issue":
             run_issue(args.reps, dev)
         elif w == "compare":
