@@ -378,6 +378,31 @@ int gws_bitwidth_loss(int64_t m, const float* bt, float b_target, float* loss_ou
 int gws_bitwidth_grad(int64_t m, const float* grad_bt, const float* bt, float b_init, float b_target, double lambda,
                       float* grad_bi, void* stream);
 
+/* Eq. 11 and the chain rule above for many layers at once.  A model has one b_i vector per linear layer, each a few
+ * thousand floats: a launch per layer is all launch latency, so these two calls take a host array of items, one per
+ * layer, and run them in one launch per 64 layers (the items travel in the kernel parameters; nothing is allocated or
+ * copied).  Results are bit for bit those of gws_bitwidth / gws_bitwidth_grad called layer by layer.
+ *   gws_bitwidth_multi       uses bi, bt, n, b_init, b_target of every item:   bt = b_target + bi * (b_init - b_target)
+ *   gws_bitwidth_grad_multi  uses grad_bt, bt, grad_bi, n, b_init, b_target, lambda, accumulate:
+ *                            grad_bi (+)= (b_init - b_target) * (grad_bt + lambda / n * sign(bt - b_target));
+ *                            accumulate != 0 adds to what grad_bi holds (gradient accumulation), 0 overwrites it
+ * All pointers device, FP32 [n], 4-byte aligned; n is the layer's number of groups (Eq. 12's mean is over them); items with
+ * n == 0 are skipped.  items: host memory, read during the call.  Every item is validated before the first launch
+ * (GWS_ERR_NULL, GWS_ERR_SHAPE for n < 0, GWS_ERR_LIMIT for n >= 2^31, GWS_ERR_ALIGN). */
+typedef struct gws_bitwidth_item {
+  const float* bi;
+  float* bt;
+  const float* grad_bt;
+  float* grad_bi;
+  int64_t n;
+  float b_init, b_target;
+  double lambda;
+  int32_t accumulate;
+  int32_t reserved;
+} gws_bitwidth_item;
+int gws_bitwidth_multi(int n_items, const gws_bitwidth_item* items, void* stream);
+int gws_bitwidth_grad_multi(int n_items, const gws_bitwidth_item* items, void* stream);
+
 /* Host only.  The seed of layer `layer` under the user's seed: the first 64 output bits of
  * Philox4x32-10 with counter (lo32(layer), hi32(layer), 0, 0) and key (lo32(user_seed), hi32(user_seed)).
  * The per-update change of a layer's PRNG state is the `step` of its descriptor. */

@@ -10,7 +10,7 @@ CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libgws.so")
 SOURCES = [os.path.join(CSRC, "gws_api.cu")]
-HEADERS = [os.path.join(CSRC, "gws_kernels.cuh"), os.path.join(CSRC, "gws_math.cuh"), os.path.join(CSRC, "gws_gemm.cuh"), os.path.join(CSRC, "gws_probe.cuh"), os.path.join(CSRC, "gws_compare.cuh"), os.path.join(CSRC, "gws_gemm_cluster.cuh"), os.path.join(CSRC, "gws_gemm_wide.cuh"),
+HEADERS = [os.path.join(CSRC, "gws_kernels.cuh"), os.path.join(CSRC, "gws_math.cuh"), os.path.join(CSRC, "gws_gemm.cuh"), os.path.join(CSRC, "gws_probe.cuh"), os.path.join(CSRC, "gws_compare.cuh"), os.path.join(CSRC, "gws_gemm_cluster.cuh"), os.path.join(CSRC, "gws_gemm_wide.cuh"), os.path.join(CSRC, "gws_train.cuh"),
            os.path.join(INCLUDE, "gws.h")]
 
 # -fmad=false: the add-then-cast path must round the multiply and the add separately.

@@ -88,6 +88,8 @@ _SIGNATURES = {
     "gws_bitwidth": (c_int, [c_int64, c_void_p, c_float, c_float, c_void_p, c_void_p]),
     "gws_bitwidth_loss": (c_int, [c_int64, c_void_p, c_float, c_void_p, c_void_p]),
     "gws_bitwidth_grad": (c_int, [c_int64, c_void_p, c_void_p, c_float, c_float, ctypes.c_double, c_void_p, c_void_p]),
+    "gws_bitwidth_multi": (c_int, [c_int, c_void_p, c_void_p]),
+    "gws_bitwidth_grad_multi": (c_int, [c_int, c_void_p, c_void_p]),
     "gws_layer_seed": (c_uint64, [c_uint64, c_uint64]),
     "gws_sample_fwd_multi_static": (c_int, [c_int, POINTER(Desc), POINTER(_MultiPtrs), c_uint64, c_void_p]),
     "gws_sample_step_host": (c_int, [POINTER(Desc)] + [c_void_p] * 13),
@@ -417,6 +419,39 @@ def bitwidth_grad(grad_bt: torch.Tensor, bt: torch.Tensor, b_init: float, b_targ
     _check(load_library().gws_bitwidth_grad(bt.numel(), _ptr(grad_bt), _ptr(bt), b_init, b_target, lam, _ptr(grad_bi),
                                             _stream(stream)))
     return grad_bi
+
+
+class BitwidthItem(Structure):
+    """``gws_bitwidth_item`` of include/gws.h: one layer of gws_bitwidth_multi / gws_bitwidth_grad_multi."""
+    _fields_ = [("bi", c_void_p), ("bt", c_void_p), ("grad_bt", c_void_p), ("grad_bi", c_void_p), ("n", c_int64),
+                ("b_init", c_float), ("b_target", c_float), ("lam", ctypes.c_double), ("accumulate", c_int32), ("reserved", c_int32)]
+
+
+def _bitwidth_items(layers) -> ctypes.Array:
+    """layers: dicts with bt, b_init, b_target and bi (forward) or grad_bt, grad_bi, lam, accumulate (gradient)."""
+    items = (BitwidthItem * len(layers))()
+    for k, it in enumerate(layers):
+        tensors = [it.get(name) for name in ("bi", "bt", "grad_bt", "grad_bi")]
+        _require_cuda(*tensors)
+        n = it["bt"].numel()
+        if any(t is not None and (t.numel() != n or t.dtype != torch.float32 or not t.is_contiguous()) for t in tensors):
+            raise ValueError("gws: the arrays of a layer are contiguous FP32 tensors of one length")
+        items[k] = BitwidthItem(*[None if t is None else t.data_ptr() for t in tensors], n, it["b_init"], it["b_target"], it.get("lam", 0.0),
+                                1 if it.get("accumulate") else 0, 0)
+    return items
+
+
+def bitwidth_multi(layers, stream=None) -> None:
+    """Eq. 11 for many layers in one launch per 64 layers: every dict gives bi, bt (written), b_init, b_target."""
+    items = _bitwidth_items(layers)
+    _check(load_library().gws_bitwidth_multi(len(layers), ctypes.cast(items, c_void_p), _stream(stream)))
+
+
+def bitwidth_grad_multi(layers, stream=None) -> None:
+    """dL'/db_i for many layers at once: every dict gives grad_bt, bt, grad_bi (written, or added to when ``accumulate``),
+    b_init, b_target, lam."""
+    items = _bitwidth_items(layers)
+    _check(load_library().gws_bitwidth_grad_multi(len(layers), ctypes.cast(items, c_void_p), _stream(stream)))
 
 
 def layer_seed(user_seed: int, layer: int) -> int:

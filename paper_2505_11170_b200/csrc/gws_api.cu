@@ -17,6 +17,7 @@
 #include "gws_kernels.cuh"
 #include "gws_probe.cuh"
 #include "gws_compare.cuh"
+#include "gws_train.cuh"
 
 namespace {
 
@@ -1267,6 +1268,58 @@ int gws_bitwidth_grad(int64_t m, const float* grad_bt, const float* bt, float b_
       grad_bt, bt, b_init - b_target, b_target, static_cast<float>(lambda / static_cast<double>(m)), grad_bi, m);
   return check_launch("bit-width gradient kernel");
 }
+
+// Shared by the two multi-layer calls: validation of every item first, then one launch per kBitwidthCap layers.
+static int bitwidth_multi(int n_items, const gws_bitwidth_item* items, bool grad, void* stream) {
+  if (n_items < 0) return GWS_ERR_SHAPE;
+  if (n_items == 0) return GWS_OK;
+  if (items == nullptr) return GWS_ERR_NULL;
+  for (int k = 0; k < n_items; ++k) {
+    const gws_bitwidth_item& it = items[k];
+    if (it.n < 0) return GWS_ERR_SHAPE;
+    if (it.n > 0x7FFFFFFFLL) return GWS_ERR_LIMIT;
+    if (it.n == 0) continue;
+    if (it.bt == nullptr || (grad ? (it.grad_bt == nullptr || it.grad_bi == nullptr) : it.bi == nullptr)) return GWS_ERR_NULL;
+    if (!aligned(it.bt, 4) || !aligned(it.bi, 4) || !aligned(it.grad_bt, 4) || !aligned(it.grad_bi, 4)) return GWS_ERR_ALIGN;
+  }
+  int k = 0;
+  while (k < n_items) {
+    gws::BitwidthBatch b;
+    std::memset(&b, 0, sizeof b);
+    uint64_t blocks = 0;
+    while (k < n_items && b.n < gws::kBitwidthCap) {
+      const gws_bitwidth_item& it = items[k++];
+      if (it.n == 0) continue;
+      const uint64_t need = (static_cast<uint64_t>(it.n) + gws::kBitwidthPerBlock - 1) / gws::kBitwidthPerBlock;
+      if (blocks + need > static_cast<uint64_t>(kMaxGrid)) { --k; break; }   // the next launch takes it
+      gws::BitwidthRec& r = b.e[b.n++];
+      r.bi = it.bi;
+      r.bt = it.bt;
+      r.grad_bt = it.grad_bt;
+      r.grad_bi = it.grad_bi;
+      r.n = static_cast<uint32_t>(it.n);
+      r.block_begin = static_cast<uint32_t>(blocks);
+      r.delta = it.b_init - it.b_target;
+      r.b_target = it.b_target;
+      r.lam_over_m = static_cast<float>(it.lambda / static_cast<double>(it.n));
+      r.accumulate = it.accumulate != 0 ? 1u : 0u;
+      blocks += need;
+    }
+    if (b.n == 0) {
+      if (k < n_items && blocks == 0) return GWS_ERR_LIMIT;   // a single layer beyond the grid limit
+      continue;
+    }
+    if (grad) gws::k_bitwidth_multi<true><<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(b);
+    else gws::k_bitwidth_multi<false><<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(b);
+    const int st = check_launch("multi-layer bit-width kernel");
+    if (st != GWS_OK) return st;
+  }
+  return GWS_OK;
+}
+
+int gws_bitwidth_multi(int n_items, const gws_bitwidth_item* items, void* stream) { return bitwidth_multi(n_items, items, false, stream); }
+
+int gws_bitwidth_grad_multi(int n_items, const gws_bitwidth_item* items, void* stream) { return bitwidth_multi(n_items, items, true, stream); }
 
 uint64_t gws_layer_seed(uint64_t user_seed, uint64_t layer) {
   const gws::Words4 w = gws::philox4x32_10(static_cast<uint32_t>(layer), static_cast<uint32_t>(layer >> 32), 0u, 0u,

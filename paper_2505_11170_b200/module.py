@@ -115,7 +115,7 @@ class GaussWSSet:
         layers = [m for m in model.modules() if isinstance(m, GaussWSLinear)]
         sampler = GaussWSSet(layers)
         for each update:
-            sampler.sample()                    # Eq. 11 per layer, then Eq. 3 + cast for every layer at once
+            sampler.sample()                    # Eq. 11, then Eq. 3 + cast, for every layer at once
             for each micro-batch: loss(model(x)).backward()      # dL/dw accumulates in weight.grad (dL/dw = dL/dw_hat)
             sampler.finish_backward()           # Eq. 4 for every layer at once, then Eq. 11 / Eq. 12 into b_i.grad
             optimizer.step(); optimizer.zero_grad(); sampler.advance()
@@ -163,10 +163,11 @@ class GaussWSSet:
         return steps.pop()
 
     def sample(self, stream=None) -> None:
-        """Eq. 11 for every layer, then Eq. 3 + the BF16 cast for all of them in one launch per kernel class."""
+        """Eq. 11 for every layer (one launch per 64 layers), then Eq. 3 + the BF16 cast for all of them in one launch per kernel
+        class."""
         step = self._step()
-        for layer, bt in zip(self.layers, self._bt):
-            binding.bitwidth(layer.b_i.detach(), layer.b_init, layer.b_target, bt=bt, stream=stream)
+        binding.bitwidth_multi([dict(bi=l.b_i.detach(), bt=bt, b_init=l.b_init, b_target=l.b_target) for l, bt in zip(self.layers, self._bt)],
+                               stream=stream)
         key = tuple(l.weight.data_ptr() for l in self.layers)
         if key != self._fwd_key:                        # the plan holds the addresses of the weights
             self._fwd_plan = binding.MultiPlan(self._descs(), w=[l.weight.detach() for l in self.layers], bt=self._bt, w_hat=self._w_hat,
@@ -192,12 +193,14 @@ class GaussWSSet:
             self._bwd_plan = binding.MultiPlan(self._descs(), scale=self._scale, grad_w_hat=grads, grad_bt=self._grad_bt, stream=stream)
             self._bwd_key = key
         self._bwd_plan.sample_bwd_multi(step, stream=stream)
+        items = []
         for layer, bt, grad_bt in zip(self.layers, self._bt, self._grad_bt):
-            grad_bi = binding.bitwidth_grad(grad_bt, bt, layer.b_init, layer.b_target, layer.lam, stream=stream)
-            if layer.b_i.grad is None:
-                layer.b_i.grad = grad_bi
-            else:
-                layer.b_i.grad.add_(grad_bi)
+            fresh = layer.b_i.grad is None
+            if fresh:
+                layer.b_i.grad = torch.empty_like(layer.b_i)
+            items.append(dict(grad_bt=grad_bt, bt=bt, grad_bi=layer.b_i.grad, b_init=layer.b_init, b_target=layer.b_target, lam=layer.lam,
+                              accumulate=not fresh))
+        binding.bitwidth_grad_multi(items, stream=stream)
 
     def advance(self) -> None:
         """One gradient update has been applied to every layer: the next sample() draws new noise."""

@@ -201,3 +201,22 @@ def test_launch_overlap_setting_is_off_at_load_and_returns_the_previous_value(li
     assert lib.gws_set_launch_overlap(1) == 1          # ... and is reported as 1
     assert gws.set_launch_overlap(False) is True
     assert gws.set_launch_overlap(False) is False
+
+
+def test_multi_layer_bitwidth_calls_validate_every_item_before_any_launch(lib):
+    Item = binding.BitwidthItem
+    assert lib.gws_bitwidth_multi(0, None, None) == binding.OK
+    assert lib.gws_bitwidth_multi(-1, None, None) == binding.ERR_SHAPE
+    assert lib.gws_bitwidth_multi(1, None, None) == binding.ERR_NULL
+    items = (Item * 2)(Item(256, 512, None, None, 0, 6.0, 4.0, 0.0, 0, 0), Item(None, 512, None, None, 8, 6.0, 4.0, 0.0, 0, 0))
+    assert lib.gws_bitwidth_multi(2, ctypes.cast(items, ctypes.c_void_p), None) == binding.ERR_NULL      # second item: no b_i
+    items[1] = Item(256, 514, None, None, 8, 6.0, 4.0, 0.0, 0, 0)
+    assert lib.gws_bitwidth_multi(2, ctypes.cast(items, ctypes.c_void_p), None) == binding.ERR_ALIGN
+    items[1] = Item(256, 512, None, None, -3, 6.0, 4.0, 0.0, 0, 0)
+    assert lib.gws_bitwidth_multi(2, ctypes.cast(items, ctypes.c_void_p), None) == binding.ERR_SHAPE
+    items[1] = Item(256, 512, None, None, 1 << 31, 6.0, 4.0, 0.0, 0, 0)
+    assert lib.gws_bitwidth_multi(2, ctypes.cast(items, ctypes.c_void_p), None) == binding.ERR_LIMIT
+    items[1] = Item(256, 512, 768, None, 8, 6.0, 4.0, 0.0, 0, 0)
+    assert lib.gws_bitwidth_grad_multi(2, ctypes.cast(items, ctypes.c_void_p), None) == binding.ERR_NULL # no grad_bi
+    items[1] = Item(None, None, None, None, 0, 6.0, 4.0, 0.0, 0, 0)
+    assert lib.gws_bitwidth_grad_multi(2, ctypes.cast(items, ctypes.c_void_p), None) == binding.OK       # empty layers only

@@ -128,3 +128,28 @@ def test_module_adds_the_bitwidth_loss_term_once_per_update():
     layer(x).backward(upstream)
     single = layer.b_i.grad.detach().cpu().numpy().astype(np.float64)
     assert np.abs(acc - (2.0 * single - term)).max() <= 1e-5 * np.abs(single).max()
+
+
+def test_multi_layer_calls_give_the_bits_of_the_layer_by_layer_calls():
+    # 150 layers (more than one launch carries), sizes from 1 to 100003, different hyper-parameters, one empty layer
+    g = torch.Generator().manual_seed(9)
+    sizes = [1, 255, 1024, 1025, 4096, 100003, 0] + [int(v) for v in torch.randint(1, 5000, (143,), generator=g)]
+    layers = []
+    for k, n in enumerate(sizes):
+        layers.append(dict(bi=torch.empty(n).uniform_(-0.5, 1.5, generator=g).to(DEV), bt=torch.empty(n, device=DEV),
+                           grad_bt=(torch.randn(n, generator=g) * 1e-3).to(DEV), grad_bi=torch.full((n,), 0.5, device=DEV),
+                           b_init=6.0 + 0.25 * (k % 5), b_target=4.0 - 0.5 * (k % 3), lam=0.1 * (k % 4), accumulate=(k % 2 == 1)))
+    gws.bitwidth_multi(layers)
+    gws.bitwidth_grad_multi(layers)
+    torch.cuda.synchronize()
+    for it in layers:
+        want_bt = gws.bitwidth(it["bi"], it["b_init"], it["b_target"])
+        assert torch.equal(it["bt"].view(torch.int32), want_bt.view(torch.int32))
+        want = gws.bitwidth_grad(it["grad_bt"], want_bt, it["b_init"], it["b_target"], it["lam"])
+        if it["accumulate"]:
+            want = torch.full_like(want, 0.5) + want
+        assert torch.equal(it["grad_bi"].view(torch.int32), want.view(torch.int32))
+    # and one layer against the oracle
+    it = layers[5]
+    want = orc.bitwidth(it["bi"].cpu().numpy(), it["b_init"], it["b_target"])
+    assert (it["bt"].cpu().numpy().view(np.uint32) == want.view(np.uint32)).all()
