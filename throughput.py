@@ -1,6 +1,6 @@
 """Throughput of the sampling pass on the other workload shapes of the paper (one JSON line each).
 
-    python throughput.py [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [issue] [compare] [module] [--reps N] [--blocks B]
+    python throughput.py [gpt2] [gpt2_single] [stress] [square] [llama] [mx] [gemm] [issue] [compare] [module] [overhead] [--reps N] [--blocks B]
 
 gpt2         all GPT2-124M linear weights, one group per row (and the same set with groups of 128)
 gpt2_single  one GPT2-124M MLP weight, both orientations
@@ -12,6 +12,7 @@ gemm         sampling fused into a tcgen05 GEMM against sampling + library GEMM 
 compare      forward pass with the method's noise against the same kernel shape with Box-Muller and with BF16 uniform noise
              (the series "ours", "bm" and the DiffQ-style noise of the paper's forward benchmark), matrices of its range
 module       the sampling part of an update through the module wrappers: layer by layer against all layers at once (GaussWSSet)
+overhead     the three GEMMs of every linear layer for one micro-batch, with and without the sampling pass around them
 issue        cycles per warp instruction of the instruction kinds the passes are made of, and of the passes' arithmetic
              without memory traffic (gws_issue_probe): the terms of the arithmetic ceiling of the backward pass
 
@@ -301,6 +302,61 @@ def run_module(reps: int, dev, n_blocks: int) -> dict:
     return line
 
 
+def run_overhead(reps: int, dev, n_blocks: int, tokens: int = 16384) -> dict:
+    """What the sampling pass adds to the linear layers of a training step (the kind of number Table 1 of the paper gives for
+    whole steps): for every Llama2-1B-shaped linear layer the three BF16 GEMMs of a micro-batch of `tokens` tokens (y = x W^T,
+    dx = dy W, dW = dy^T x; torch's GEMMs on synthetic activations), once on the master weights and once on weights sampled
+    by GaussWSSet with Eq. 4 / Eq. 11 / Eq. 12 at the end of the step.  No attention, norms or optimizer: the percentage is
+    an upper bound on the overhead of a full step."""
+    from paper_2505_11170_b200.module import GaussWSLinear, GaussWSSet
+    specs = syn.llama2_1b(n_blocks=n_blocks)
+    layers = [GaussWSLinear(s.cols, s.rows, bias=False, group=(32, 32), lam=0.1, layer_index=k, device=dev) for k, s in enumerate(specs)]
+    sampler = GaussWSSet(layers)
+    gen = torch.Generator(device=dev).manual_seed(1)
+    xs = {c: torch.randn(tokens, c, generator=gen, device=dev).to(torch.bfloat16) for c in {s.cols for s in specs}}
+    dys = {r: (torch.randn(tokens, r, generator=gen, device=dev) * 1e-2).to(torch.bfloat16) for r in {s.rows for s in specs}}
+    ys = {r: torch.empty(tokens, r, dtype=torch.bfloat16, device=dev) for r in dys}
+    dxs = {c: torch.empty(tokens, c, dtype=torch.bfloat16, device=dev) for c in xs}
+    for layer in layers:
+        layer.weight.grad = torch.empty_like(layer.weight)
+
+    def gemms(weights):
+        for layer, s, w in zip(layers, specs, weights):
+            torch.mm(xs[s.cols], w.t(), out=ys[s.rows])
+            torch.mm(dys[s.rows], w, out=dxs[s.cols])
+            torch.mm(dys[s.rows].t(), xs[s.cols], out=layer.weight.grad)
+
+    def plain():
+        gemms([l.weight.detach() for l in layers])
+
+    def sampled():
+        sampler.sample()
+        gemms([sampler.w_hat_of(l) for l in layers])
+        sampler.finish_backward()
+        sampler.advance()
+
+    def timed(fn):
+        total = 0.0
+        for i in range(2 + reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                total += a.elapsed_time(b)
+        return total / reps
+    with torch.no_grad():
+        t_plain, t_sampled, t_plain2 = timed(plain), timed(sampled), timed(plain)
+    base = 0.5 * (t_plain + t_plain2)
+    flops = 6.0 * syn.total_elements(specs) * tokens
+    line = {"workload": f"linear layers of llama2_1b ({n_blocks} blocks), one micro-batch of {tokens} tokens, 32x32 groups",
+            "gemms_only_ms": base, "gemms_with_sampling_ms": t_sampled, "overhead_pct": 100.0 * (t_sampled / base - 1.0),
+            "gemm_TFLOP/s": flops / (base * 1e-3) / 1e12, "reps": reps}
+    print(json.dumps(line), flush=True)
+    return line
+
+
 def main(argv=None) -> None:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("which", nargs="*", default=["gpt2", "stress"])
@@ -329,6 +385,8 @@ def main(argv=None) -> None:
             run(f"llama2_1b {args.blocks} blocks, groups of 128", syn.llama2_1b(n_blocks=args.blocks), args.reps, dev)
         elif w == "gemm":
             run_gemm(args.reps, dev)
+        elif w == "overhead":
+            run_overhead(max(1, args.reps // 4), dev, args.blocks)
         elif w == "module":
             run_module(args.reps, dev, args.blocks)
         elif w == "issue":
